@@ -1,0 +1,202 @@
+/*
+ * q8 -- 8-bit quantized CNN inference primitives for NVIDIA B200 (sm_100a).
+ *
+ * C ABI of the library.  Every entry point returns a q8_status.  No exception
+ * crosses this boundary, nothing aborts, no kernel traps.
+ *
+ * Conventions
+ *  - "device pointer" = memory reachable from the current CUDA device; the
+ *    caller owns every buffer, the library allocates no device memory.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  All
+ *    device work is enqueued on it asynchronously; only q8_read_status blocks.
+ *  - Activations are NHWC, weights are KRSC (Cout, R, S, Cin), both contiguous
+ *    in the channel dimension.  Quantized payloads are u8, s8 or s32; the
+ *    quantization factor q of a tensor is one host-side fp32 number.
+ *  - Rounding is round-half-to-even everywhere; every fp32 step is a single
+ *    IEEE operation (no fused multiply-add), so results are reproducible bit
+ *    for bit.
+ */
+#ifndef Q8_H_
+#define Q8_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum q8_status {
+  Q8_OK = 0,
+  Q8_ERR_INVALID_ARG = 1, /* null pointer, non-positive extent, unknown enum */
+  Q8_ERR_UNSUPPORTED = 2, /* legal request that no kernel here can run */
+  Q8_ERR_ALIGNMENT = 3,   /* pointer or stride not aligned as documented */
+  Q8_ERR_WORKSPACE = 4,   /* workspace missing or too small */
+  Q8_ERR_CUDA = 5,        /* CUDA runtime/driver error; text in q8_last_error() */
+  Q8_ERR_TIMEOUT = 6,     /* a bounded device-side wait gave up (status word set) */
+  Q8_ERR_NONFINITE = 7    /* NaN/Inf where a finite value is required */
+} q8_status;
+
+typedef enum q8_dtype { Q8_U8 = 0, Q8_S8 = 1, Q8_S32 = 2, Q8_F32 = 3 } q8_dtype;
+
+/* Which convolution kernel to use. */
+typedef enum q8_conv_algo {
+  Q8_ALGO_AUTO = 0,   /* tensor-core kernel when the shape allows it, else direct */
+  Q8_ALGO_UMMA = 1,   /* tcgen05 implicit GEMM; Q8_ERR_UNSUPPORTED if not eligible */
+  Q8_ALGO_DIRECT = 2  /* CUDA-core direct convolution, any shape */
+} q8_conv_algo;
+
+/* ------------------------------------------------------------------------
+ * Library info and errors (host only).
+ * ---------------------------------------------------------------------- */
+const char* q8_version(void);
+/* Text of the last error raised on the calling thread ("" if none). */
+const char* q8_last_error(void);
+/* Blocks until `stream` is idle, then reads and clears the device status word.
+ * Returns Q8_ERR_TIMEOUT if a kernel gave up on a bounded wait since the last
+ * call (its outputs are then undefined), Q8_OK otherwise. */
+int q8_read_status(void* stream);
+
+/* ------------------------------------------------------------------------
+ * Calibration (Sec. "8-bit Low Precision Inference", calibration paragraph:
+ * each tensor's factor is max|r| / (2^p - 1)).
+ * ---------------------------------------------------------------------- */
+
+/* *d_running_max = max(*d_running_max, max_i |x[i]|).
+ * x: device, n fp32 values (n may be 0).  d_running_max: device, one fp32 the
+ * caller sets to 0 before the first batch.  A NaN/Inf in x makes the result
+ * NaN/Inf (largest bit pattern wins); q8_factor then reports it. */
+int q8_calibrate_maxabs(const float* x, size_t n, float* d_running_max, void* stream);
+
+/* Host helper: *q = maxabs / (2^p - 1) as one fp32 division; *q = 1 when
+ * maxabs == 0.  p in [1,31].  Q8_ERR_NONFINITE if maxabs is NaN/Inf/negative. */
+int q8_factor(float maxabs, int p, float* q);
+
+/* Host helper: *s = fp32(q_x * q_w / q_y) formed in fp64 -- the single
+ * requantisation multiplier of Eq. (int8_affine) (accumulator factor q_W q_x by
+ * the product rule of Eq. (arithmetics), re-expressed at q_y). */
+int q8_requant_scale(float q_x, float q_w, float q_y, float* s);
+
+/* Host helper: *q_b = q_x * q_w (one fp32 multiply), the factor at which the
+ * int32 bias is quantized so that it can be added to the accumulator. */
+int q8_bias_factor(float q_x, float q_w, float* q_b);
+
+/* ------------------------------------------------------------------------
+ * Eq. (Q): z = clamp(Round(x / q)), and Eq. (D): r = q * z.
+ * ---------------------------------------------------------------------- */
+
+/* z[i] = clamp(Round(x[i] / q), lo, hi) with (lo,hi) = (0,255) for Q8_U8,
+ * (-128,127) for Q8_S8, (-2^31, 2^31-1) for Q8_S32.  fp32 IEEE division.  NaN
+ * maps to 0.  x, z: device, n elements, same layout.  q must be finite, > 0. */
+int q8_quantize(const float* x, size_t n, float q, int out_type, void* z, void* stream);
+
+/* As q8_quantize for an NHWC tensor of `pixels` x C values, but the output has
+ * C_pad >= C channels per pixel and channels C..C_pad-1 are written as 0 (the
+ * exact code of 0.0 under a symmetric quantizer).  Lets a 3-channel image feed
+ * kernels that need 16-byte aligned pixels.  out_type: Q8_U8 or Q8_S8. */
+int q8_quantize_pad_channels(const float* x, size_t pixels, int C, int C_pad, float q, int out_type,
+                             void* z, void* stream);
+
+/* r[i] = q * float(z[i]).  in_type: Q8_U8, Q8_S8 or Q8_S32. */
+int q8_dequantize(const void* z, int in_type, size_t n, float q, float* r, void* stream);
+
+/* ------------------------------------------------------------------------
+ * Batch-norm folding (Sec. "Model Optimization"):
+ *   a = gamma / sqrt(var + eps);  w' = a w;  b' = a (b - mean) + beta,
+ * evaluated in fp64 and rounded once to fp32.
+ * w, w_out: device [K][elems_per_k] (may alias).  b: device [K] or NULL (= 0).
+ * gamma, beta, mean, var, b_out: device [K].
+ * ---------------------------------------------------------------------- */
+int q8_fold_bn(const float* w, const float* b, const float* gamma, const float* beta, const float* mean,
+               const float* var, double eps, int K, size_t elems_per_k, float* w_out, float* b_out,
+               void* stream);
+
+/* ------------------------------------------------------------------------
+ * Quantized convolution with fused epilogue (Eq. int8_affine,
+ * Eq. int8_affine_fused; "+" and "x" of Eq. arithmetics; conv+ReLU and
+ * conv+eltwise-sum fusion of Sec. "Model Optimization"):
+ *
+ *   acc[n,p,q,k] = sum_{r,s,c} x[n, p*stride_h - pad_h + r*dil_h,
+ *                                   q*stride_w - pad_w + s*dil_w, c] * w[k,r,s,c]
+ *                  + bias[k]                          (int32, zero padding)
+ *   v = float(acc) * scale[k or 0]                    (one fp32 multiply)
+ *   v = v + float(residual[n,p,q,k]) * residual_scale (product, then sum)
+ *   v = max(v, 0)                                     (if relu)
+ *   y = clamp(Round(v)) as u8 [0,255] or s8 [-128,127]; or v (Q8_F32); or
+ *       acc (Q8_S32, raw accumulator, scale/residual/relu ignored)
+ * with P = (H + 2 pad_h - dil_h (R-1) - 1) / stride_h + 1 (floor), same for Q.
+ *
+ * y is written at y[((n*P + p)*Q + q) * y_ldc + y_c_offset + k]: with
+ * y_ldc > K the layer writes a channel slice of a wider tensor (concatenation
+ * in place).  y_ldc = 0 means K.
+ * ---------------------------------------------------------------------- */
+typedef struct q8_conv_desc {
+  int32_t N, H, W, C;       /* input  NHWC */
+  int32_t K, R, S;          /* filter KRSC (C shared) */
+  int32_t stride_h, stride_w;
+  int32_t pad_h, pad_w;
+  int32_t dil_h, dil_w;
+  int32_t x_type;           /* Q8_U8 or Q8_S8 */
+  int32_t res_type;         /* Q8_U8 or Q8_S8 (ignored without residual) */
+  int32_t y_type;           /* Q8_U8, Q8_S8, Q8_F32 or Q8_S32 */
+  int32_t relu;             /* 0/1 */
+  int32_t scale_count;      /* 1 (per tensor) or K (per output channel) */
+  int32_t y_ldc;            /* channels per output pixel in memory, 0 = K */
+  int32_t y_c_offset;       /* first channel written */
+  int32_t algo;             /* q8_conv_algo */
+} q8_conv_desc;
+
+/* Bytes of device scratch q8_conv2d needs for `d` (0 for most shapes; split-K
+ * partial sums otherwise).  Host only. */
+int q8_conv2d_workspace_bytes(const q8_conv_desc* d, size_t* bytes);
+
+/* Which kernel q8_conv2d would pick for `d`: writes Q8_ALGO_UMMA or
+ * Q8_ALGO_DIRECT.  Host only. */
+int q8_conv2d_query_algo(const q8_conv_desc* d, int* algo);
+
+/* x: device NHWC (x_type).  w: device KRSC s8.  bias: device s32[K] or NULL.
+ * scale: device fp32[scale_count].  residual: device [N,P,Q,K] dense (res_type)
+ * or NULL.  y: device, see above.  workspace: device, >= workspace_bytes (may be
+ * NULL when 0 are needed); contents undefined afterwards.
+ * Alignment: the tensor-core kernel needs x, w, y, residual 16-byte aligned, C
+ * a multiple of 16, and for u8/s8 output y_ldc and y_c_offset multiples of 16;
+ * Q8_ALGO_AUTO falls back to the direct kernel otherwise.
+ * Errors: Q8_ERR_INVALID_ARG (null/extent/enum, R*S*C > 65793 which could
+ * overflow int32), Q8_ERR_UNSUPPORTED (Q8_ALGO_UMMA on an ineligible shape),
+ * Q8_ERR_WORKSPACE, Q8_ERR_CUDA.  Nothing is launched on error. */
+int q8_conv2d(const q8_conv_desc* d, const void* x, const int8_t* w, const int32_t* bias,
+              const float* scale, const void* residual, float residual_scale, void* y,
+              void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------
+ * Channel concatenation of quantized branches under one factor (the paper
+ * gives no rule; the caller passes the shared factor, normally the largest
+ * branch factor as in the "+" rule of Eq. arithmetics).  Branch i is written
+ * as clamp(Round(float(z) * fp32(q_i / q_out))) (ratio formed in fp64), or
+ * copied unchanged when that ratio is exactly 1.
+ * xs: host array of n_in device pointers, branch i is [pixels][channels[i]].
+ * channels, in_factors: host arrays.  y: device [pixels][sum channels].
+ * t: Q8_U8 or Q8_S8.  n_in <= 8.
+ * ---------------------------------------------------------------------- */
+int q8_concat(int n_in, const void* const* xs, const int* channels, const float* in_factors,
+              float out_factor, int t, size_t pixels, void* y, void* stream);
+
+/* ------------------------------------------------------------------------
+ * Pooling between quantized layers (not described in the paper; needed to
+ * run whole networks in int8).  The factor is unchanged.
+ * max: maximum over the in-image cells of the window.
+ * avg: clamp(Round(float(sum of in-image cells) * fp32(1/(kh*kw)))) -- full
+ *      window divisor, padding counts as zero.
+ * ceil_mode: output extent rounds up (last window may hang over the edge).
+ * x: device NHWC, y: device [N,P,Q,C]; t: Q8_U8 or Q8_S8.
+ * ---------------------------------------------------------------------- */
+int q8_pool_out_extent(int H, int k, int stride, int pad, int ceil_mode, int* out);
+int q8_maxpool2d(const void* x, int t, int N, int H, int W, int C, int kh, int kw, int stride_h,
+                 int stride_w, int pad_h, int pad_w, int ceil_mode, void* y, void* stream);
+int q8_avgpool2d(const void* x, int t, int N, int H, int W, int C, int kh, int kw, int stride_h,
+                 int stride_w, int pad_h, int pad_w, int ceil_mode, void* y, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* Q8_H_ */

@@ -1,0 +1,525 @@
+// Bandwidth-bound kernels around the quantized convolution: max-abs calibration,
+// quantize (Eq. Q), dequantize (Eq. D), BN folding, concat, pooling.
+//
+// All of them stream their operands once with 16-byte accesses; grids are sized
+// as a multiple of the SM count so every SM keeps several loads in flight.
+#include <cmath>
+
+#include "q8_internal.h"
+
+namespace q8 {
+namespace {
+
+constexpr int kThreads = 512;
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 148;
+  }
+  return n;
+}
+
+int grid_for(size_t work_items, int per_block, int blocks_per_sm) {
+  size_t need = (work_items + per_block - 1) / per_block;
+  size_t cap = (size_t)sm_count() * blocks_per_sm;
+  if (need < 1) need = 1;
+  return (int)(need < cap ? need : cap);
+}
+
+// ---------------------------------------------------------------------------------------------
+// max |x|: bits of a non-negative float order like unsigned integers, and NaN/Inf patterns sit
+// above every finite value, so an unsigned atomicMax both reduces and propagates non-finite input.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned int abs_bits(float v) { return __float_as_uint(v) & 0x7fffffffu; }
+
+__global__ void __launch_bounds__(kThreads) maxabs_kernel(const float* __restrict__ x, size_t n,
+                                                          unsigned int* __restrict__ running) {
+  unsigned int m = 0;
+  // head: scalar until 16-byte aligned
+  size_t head = ((16 - (reinterpret_cast<uintptr_t>(x) & 15u)) & 15u) / 4;
+  if (head > n) head = n;
+  const size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  if (tid < head) m = abs_bits(x[tid]);
+  const float4* x4 = reinterpret_cast<const float4*>(x + head);
+  const size_t n4 = (n - head) / 4;
+  size_t i = tid;
+  // four independent 16-byte loads in flight per thread
+  for (; i + 3 * nthreads < n4; i += 4 * nthreads) {
+    float4 a = __ldcs(x4 + i), b = __ldcs(x4 + i + nthreads), c = __ldcs(x4 + i + 2 * nthreads),
+           d = __ldcs(x4 + i + 3 * nthreads);
+    m = max(m, max(max(abs_bits(a.x), abs_bits(a.y)), max(abs_bits(a.z), abs_bits(a.w))));
+    m = max(m, max(max(abs_bits(b.x), abs_bits(b.y)), max(abs_bits(b.z), abs_bits(b.w))));
+    m = max(m, max(max(abs_bits(c.x), abs_bits(c.y)), max(abs_bits(c.z), abs_bits(c.w))));
+    m = max(m, max(max(abs_bits(d.x), abs_bits(d.y)), max(abs_bits(d.z), abs_bits(d.w))));
+  }
+  for (; i < n4; i += nthreads) {
+    float4 a = __ldcs(x4 + i);
+    m = max(m, max(max(abs_bits(a.x), abs_bits(a.y)), max(abs_bits(a.z), abs_bits(a.w))));
+  }
+  const size_t tail0 = head + n4 * 4;
+  if (tail0 + tid < n) m = max(m, abs_bits(x[tail0 + tid]));
+
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+  __shared__ unsigned int warp_max[kThreads / 32];
+  if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    m = threadIdx.x < kThreads / 32 ? warp_max[threadIdx.x] : 0u;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if (threadIdx.x == 0 && m != 0) atomicMax(running, m);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Eq. (Q).  One fp32 IEEE division, round-to-nearest-even conversion (saturating, NaN -> 0), clamp.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ int quant1(float v, float q, int lo, int hi) {
+  int z = __float2int_rn(__fdiv_rn(v, q));
+  return min(max(z, lo), hi);
+}
+
+__device__ __forceinline__ unsigned int pack4(int a, int b, int c, int d) {
+  return (unsigned int)(a & 0xff) | ((unsigned int)(b & 0xff) << 8) | ((unsigned int)(c & 0xff) << 16) |
+         ((unsigned int)(d & 0xff) << 24);
+}
+
+// 16 floats in, 16 bytes out per thread and step.  Requires x and z 16-byte aligned.
+__global__ void __launch_bounds__(kThreads) quantize8_vec_kernel(const float4* __restrict__ x, size_t n16,
+                                                                 float q, int lo, int hi,
+                                                                 uint4* __restrict__ z) {
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += nthreads) {
+    float4 a = __ldcs(x + 4 * i), b = __ldcs(x + 4 * i + 1), c = __ldcs(x + 4 * i + 2), d = __ldcs(x + 4 * i + 3);
+    uint4 o;
+    o.x = pack4(quant1(a.x, q, lo, hi), quant1(a.y, q, lo, hi), quant1(a.z, q, lo, hi), quant1(a.w, q, lo, hi));
+    o.y = pack4(quant1(b.x, q, lo, hi), quant1(b.y, q, lo, hi), quant1(b.z, q, lo, hi), quant1(b.w, q, lo, hi));
+    o.z = pack4(quant1(c.x, q, lo, hi), quant1(c.y, q, lo, hi), quant1(c.z, q, lo, hi), quant1(c.w, q, lo, hi));
+    o.w = pack4(quant1(d.x, q, lo, hi), quant1(d.y, q, lo, hi), quant1(d.z, q, lo, hi), quant1(d.w, q, lo, hi));
+    __stcs(z + i, o);
+  }
+}
+
+template <typename OutT>
+__global__ void __launch_bounds__(kThreads) quantize_scalar_kernel(const float* __restrict__ x, size_t begin,
+                                                                   size_t n, float q, int lo, int hi,
+                                                                   OutT* __restrict__ z) {
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = begin + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += nthreads)
+    z[i] = (OutT)quant1(x[i], q, lo, hi);
+}
+
+__global__ void __launch_bounds__(kThreads) quantize32_vec_kernel(const float4* __restrict__ x, size_t n4, float q,
+                                                                  int4* __restrict__ z) {
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += nthreads) {
+    float4 a = __ldcs(x + i);
+    int4 o;
+    o.x = __float2int_rn(__fdiv_rn(a.x, q));
+    o.y = __float2int_rn(__fdiv_rn(a.y, q));
+    o.z = __float2int_rn(__fdiv_rn(a.z, q));
+    o.w = __float2int_rn(__fdiv_rn(a.w, q));
+    __stcs(z + i, o);
+  }
+}
+
+// NHWC pixels with C real channels -> C_pad channels, zeros appended.  One thread per pixel group.
+template <typename OutT>
+__global__ void __launch_bounds__(kThreads) quantize_pad_kernel(const float* __restrict__ x, size_t pixels, int C,
+                                                                int C_pad, float q, int lo, int hi,
+                                                                OutT* __restrict__ z) {
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  const size_t total = pixels * (size_t)C_pad;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += nthreads) {
+    size_t px = i / C_pad;
+    int c = (int)(i - px * C_pad);
+    z[i] = c < C ? (OutT)quant1(x[px * C + c], q, lo, hi) : (OutT)0;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Eq. (D): r = q * float(z), one fp32 multiply.
+// ---------------------------------------------------------------------------------------------
+template <bool kSigned>
+__device__ __forceinline__ float4 deq4(unsigned int w, float q) {
+  float4 r;
+  if (kSigned) {
+    r.x = __fmul_rn(q, (float)(int)(signed char)(w & 0xff));
+    r.y = __fmul_rn(q, (float)(int)(signed char)((w >> 8) & 0xff));
+    r.z = __fmul_rn(q, (float)(int)(signed char)((w >> 16) & 0xff));
+    r.w = __fmul_rn(q, (float)(int)(signed char)(w >> 24));
+  } else {
+    r.x = __fmul_rn(q, (float)(w & 0xff));
+    r.y = __fmul_rn(q, (float)((w >> 8) & 0xff));
+    r.z = __fmul_rn(q, (float)((w >> 16) & 0xff));
+    r.w = __fmul_rn(q, (float)(w >> 24));
+  }
+  return r;
+}
+
+template <bool kSigned>
+__global__ void __launch_bounds__(kThreads) dequantize8_vec_kernel(const uint4* __restrict__ z, size_t n16, float q,
+                                                                   float4* __restrict__ r) {
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += nthreads) {
+    uint4 v = __ldcs(z + i);
+    __stcs(r + 4 * i, deq4<kSigned>(v.x, q));
+    __stcs(r + 4 * i + 1, deq4<kSigned>(v.y, q));
+    __stcs(r + 4 * i + 2, deq4<kSigned>(v.z, q));
+    __stcs(r + 4 * i + 3, deq4<kSigned>(v.w, q));
+  }
+}
+
+template <typename InT>
+__global__ void __launch_bounds__(kThreads) dequantize_scalar_kernel(const InT* __restrict__ z, size_t begin,
+                                                                     size_t n, float q, float* __restrict__ r) {
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = begin + (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += nthreads)
+    r[i] = __fmul_rn(q, (float)z[i]);
+}
+
+// ---------------------------------------------------------------------------------------------
+// BN folding in fp64, rounded once to fp32.  grid = (chunks, K).
+// ---------------------------------------------------------------------------------------------
+__global__ void fold_bn_kernel(const float* __restrict__ w, const float* __restrict__ b,
+                               const float* __restrict__ gamma, const float* __restrict__ beta,
+                               const float* __restrict__ mean, const float* __restrict__ var, double eps,
+                               size_t elems_per_k, float* __restrict__ w_out, float* __restrict__ b_out) {
+  const int k = blockIdx.y;
+  const double a = __ddiv_rn((double)gamma[k], __dsqrt_rn(__dadd_rn((double)var[k], eps)));
+  const size_t base = (size_t)k * elems_per_k;
+  for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < elems_per_k; e += (size_t)gridDim.x * blockDim.x)
+    w_out[base + e] = (float)__dmul_rn(a, (double)w[base + e]);
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    double b0 = b ? (double)b[k] : 0.0;
+    b_out[k] = (float)__dadd_rn(__dmul_rn(a, __dsub_rn(b0, (double)mean[k])), (double)beta[k]);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Concat: one launch per branch; re-expresses the branch at the shared factor.
+// ---------------------------------------------------------------------------------------------
+template <bool kSigned>
+__device__ __forceinline__ int requant_byte(unsigned int b, float s) {
+  float v = kSigned ? (float)(int)(signed char)b : (float)b;
+  int z = __float2int_rn(__fmul_rn(v, s));
+  return kSigned ? min(max(z, -128), 127) : min(max(z, 0), 255);
+}
+
+template <bool kSigned>
+__device__ __forceinline__ unsigned int requant_word(unsigned int w, float s) {
+  return pack4(requant_byte<kSigned>(w & 0xff, s), requant_byte<kSigned>((w >> 8) & 0xff, s),
+               requant_byte<kSigned>((w >> 16) & 0xff, s), requant_byte<kSigned>(w >> 24, s));
+}
+
+// vec path: channels, c_total and c_off multiples of 16, pointers 16-byte aligned
+template <bool kSigned>
+__global__ void __launch_bounds__(kThreads) concat_vec_kernel(const uint4* __restrict__ x, size_t pixels, int cvec,
+                                                              int ctot_vec, int coff_vec, float s, int copy_only,
+                                                              uint4* __restrict__ y) {
+  const size_t total = pixels * (size_t)cvec;
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += nthreads) {
+    size_t px = i / cvec;
+    int c = (int)(i - px * cvec);
+    uint4 v = __ldcs(x + i);
+    if (!copy_only) {
+      v.x = requant_word<kSigned>(v.x, s);
+      v.y = requant_word<kSigned>(v.y, s);
+      v.z = requant_word<kSigned>(v.z, s);
+      v.w = requant_word<kSigned>(v.w, s);
+    }
+    y[px * ctot_vec + coff_vec + c] = v;
+  }
+}
+
+template <bool kSigned>
+__global__ void __launch_bounds__(kThreads) concat_scalar_kernel(const unsigned char* __restrict__ x, size_t pixels,
+                                                                 int ch, int ctot, int coff, float s, int copy_only,
+                                                                 unsigned char* __restrict__ y) {
+  const size_t total = pixels * (size_t)ch;
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += nthreads) {
+    size_t px = i / ch;
+    int c = (int)(i - px * ch);
+    unsigned int b = x[i];
+    y[px * ctot + coff + c] = copy_only ? (unsigned char)b : (unsigned char)requant_byte<kSigned>(b, s);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Pooling: one thread per output pixel and group of 4 channels (C % 4 == 0) or single channel.
+// ---------------------------------------------------------------------------------------------
+template <bool kSigned, bool kAvg, int kVec>
+__global__ void __launch_bounds__(256) pool_kernel(const unsigned char* __restrict__ x, int N, int H, int W, int C,
+                                                   int kh, int kw, int st_h, int st_w, int pad_h, int pad_w, int P,
+                                                   int Q, float inv, unsigned char* __restrict__ y) {
+  const int cg = C / kVec;
+  const size_t total = (size_t)N * P * Q * cg;
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += nthreads) {
+    int c = (int)(i % cg) * kVec;
+    size_t t = i / cg;
+    int q = (int)(t % Q);
+    t /= Q;
+    int p = (int)(t % P);
+    int n = (int)(t / P);
+    int acc[kVec];
+#pragma unroll
+    for (int j = 0; j < kVec; ++j) acc[j] = kAvg ? 0 : (kSigned ? -128 : 0);
+    for (int r = 0; r < kh; ++r) {
+      int h = p * st_h - pad_h + r;
+      if (h < 0 || h >= H) continue;
+      for (int s = 0; s < kw; ++s) {
+        int w = q * st_w - pad_w + s;
+        if (w < 0 || w >= W) continue;
+        const unsigned char* px = x + (((size_t)n * H + h) * W + w) * C + c;
+        unsigned int word;
+        if (kVec == 4) word = *reinterpret_cast<const unsigned int*>(px);
+        else word = *px;
+#pragma unroll
+        for (int j = 0; j < kVec; ++j) {
+          unsigned int b = (word >> (8 * j)) & 0xff;
+          int v = kSigned ? (int)(signed char)b : (int)b;
+          acc[j] = kAvg ? acc[j] + v : max(acc[j], v);
+        }
+      }
+    }
+    unsigned char* out = y + (((size_t)n * P + p) * Q + q) * C + c;
+    int o[kVec];
+#pragma unroll
+    for (int j = 0; j < kVec; ++j) {
+      if (kAvg) {
+        int z = __float2int_rn(__fmul_rn((float)acc[j], inv));
+        o[j] = kSigned ? min(max(z, -128), 127) : min(max(z, 0), 255);
+      } else {
+        o[j] = acc[j];
+      }
+    }
+    if (kVec == 4) *reinterpret_cast<unsigned int*>(out) = pack4(o[0], o[1], o[2], o[3]);
+    else *out = (unsigned char)o[0];
+  }
+}
+
+int pool_extent(int H, int k, int st, int pad, int ceil_mode) {
+  int num = H + 2 * pad - k;
+  int o = (ceil_mode ? (num + st - 1) / st : num / st) + 1;
+  if (ceil_mode && (o - 1) * st >= H + pad) --o;
+  return o;
+}
+
+template <bool kAvg>
+int launch_pool(const void* x, int t, int N, int H, int W, int C, int kh, int kw, int st_h, int st_w, int pad_h,
+                int pad_w, int ceil_mode, void* y, void* stream) {
+  clear_error();
+  if (!x || !y) return fail(Q8_ERR_INVALID_ARG, "pool: null pointer");
+  if (t != Q8_U8 && t != Q8_S8) return fail(Q8_ERR_INVALID_ARG, "pool: type must be Q8_U8 or Q8_S8");
+  if (N <= 0 || H <= 0 || W <= 0 || C <= 0 || kh <= 0 || kw <= 0 || st_h <= 0 || st_w <= 0 || pad_h < 0 || pad_w < 0 ||
+      pad_h >= kh || pad_w >= kw)
+    return fail(Q8_ERR_INVALID_ARG, "pool: bad extents");
+  int P = pool_extent(H, kh, st_h, pad_h, ceil_mode), Q = pool_extent(W, kw, st_w, pad_w, ceil_mode);
+  if (P <= 0 || Q <= 0) return fail(Q8_ERR_INVALID_ARG, "pool: empty output");
+  float inv = 1.0f / (float)(kh * kw);
+  bool vec = (C % 4 == 0) && ((reinterpret_cast<uintptr_t>(x) & 3u) == 0) && ((reinterpret_cast<uintptr_t>(y) & 3u) == 0);
+  size_t total = (size_t)N * P * Q * (vec ? C / 4 : C);
+  int grid = grid_for(total, 256, 8);
+  cudaStream_t s = as_stream(stream);
+  const unsigned char* xp = static_cast<const unsigned char*>(x);
+  unsigned char* yp = static_cast<unsigned char*>(y);
+#define Q8_POOL(SG, V) pool_kernel<SG, kAvg, V><<<grid, 256, 0, s>>>(xp, N, H, W, C, kh, kw, st_h, st_w, pad_h, pad_w, P, Q, inv, yp)
+  if (t == Q8_S8) { if (vec) Q8_POOL(true, 4); else Q8_POOL(true, 1); }
+  else { if (vec) Q8_POOL(false, 4); else Q8_POOL(false, 1); }
+#undef Q8_POOL
+  return check_launch("pool_kernel");
+}
+
+}  // namespace
+}  // namespace q8
+
+using namespace q8;
+
+extern "C" {
+
+int q8_calibrate_maxabs(const float* x, size_t n, float* d_running_max, void* stream) {
+  clear_error();
+  if (!d_running_max || (!x && n)) return fail(Q8_ERR_INVALID_ARG, "q8_calibrate_maxabs: null pointer");
+  if (reinterpret_cast<uintptr_t>(x) & 3u) return fail(Q8_ERR_ALIGNMENT, "q8_calibrate_maxabs: x not 4-byte aligned");
+  if (n == 0) return Q8_OK;
+  int grid = grid_for((n + 3) / 4, kThreads * 4, 4);
+  maxabs_kernel<<<grid, kThreads, 0, as_stream(stream)>>>(x, n, reinterpret_cast<unsigned int*>(d_running_max));
+  return check_launch("maxabs_kernel");
+}
+
+int q8_factor(float maxabs, int p, float* q) {
+  clear_error();
+  if (!q || p < 1 || p > 31) return fail(Q8_ERR_INVALID_ARG, "q8_factor: bad argument");
+  if (!(maxabs >= 0.0f) || std::isinf(maxabs)) return fail(Q8_ERR_NONFINITE, "q8_factor: max-abs is not a finite non-negative number");
+  if (maxabs == 0.0f) { *q = 1.0f; return Q8_OK; }
+  volatile float denom = (float)((1ll << p) - 1);
+  volatile float r = maxabs / denom;
+  *q = r;
+  return Q8_OK;
+}
+
+int q8_requant_scale(float q_x, float q_w, float q_y, float* s) {
+  clear_error();
+  if (!s) return fail(Q8_ERR_INVALID_ARG, "q8_requant_scale: null pointer");
+  if (!(q_x > 0.f) || !(q_w > 0.f) || !(q_y > 0.f) || std::isinf(q_x) || std::isinf(q_w) || std::isinf(q_y))
+    return fail(Q8_ERR_NONFINITE, "q8_requant_scale: factors must be finite and positive");
+  volatile double prod = (double)q_x * (double)q_w;
+  volatile double quo = prod / (double)q_y;
+  *s = (float)quo;
+  return Q8_OK;
+}
+
+int q8_bias_factor(float q_x, float q_w, float* q_b) {
+  clear_error();
+  if (!q_b) return fail(Q8_ERR_INVALID_ARG, "q8_bias_factor: null pointer");
+  volatile float r = q_x * q_w;
+  *q_b = r;
+  return Q8_OK;
+}
+
+int q8_quantize(const float* x, size_t n, float q, int out_type, void* z, void* stream) {
+  clear_error();
+  if ((!x || !z) && n) return fail(Q8_ERR_INVALID_ARG, "q8_quantize: null pointer");
+  if (!(q > 0.f) || std::isinf(q)) return fail(Q8_ERR_NONFINITE, "q8_quantize: factor must be finite and positive");
+  if (out_type != Q8_U8 && out_type != Q8_S8 && out_type != Q8_S32) return fail(Q8_ERR_INVALID_ARG, "q8_quantize: bad out_type");
+  if (n == 0) return Q8_OK;
+  cudaStream_t s = as_stream(stream);
+  if (out_type == Q8_S32) {
+    if (aligned16(x) && aligned16(z)) {
+      size_t n4 = n / 4;
+      if (n4) quantize32_vec_kernel<<<grid_for(n4, kThreads, 8), kThreads, 0, s>>>(reinterpret_cast<const float4*>(x), n4, q, static_cast<int4*>(z));
+      if (n4 * 4 < n) quantize_scalar_kernel<int><<<1, kThreads, 0, s>>>(x, n4 * 4, n, q, INT32_MIN, INT32_MAX, static_cast<int*>(z));
+    } else {
+      quantize_scalar_kernel<int><<<grid_for(n, kThreads, 8), kThreads, 0, s>>>(x, 0, n, q, INT32_MIN, INT32_MAX, static_cast<int*>(z));
+    }
+    return check_launch("quantize32");
+  }
+  const int lo = out_type == Q8_U8 ? 0 : -128, hi = out_type == Q8_U8 ? 255 : 127;
+  if (aligned16(x) && aligned16(z)) {
+    size_t n16 = n / 16;
+    if (n16) quantize8_vec_kernel<<<grid_for(n16, kThreads, 4), kThreads, 0, s>>>(reinterpret_cast<const float4*>(x), n16, q, lo, hi, static_cast<uint4*>(z));
+    if (n16 * 16 < n) quantize_scalar_kernel<unsigned char><<<1, kThreads, 0, s>>>(x, n16 * 16, n, q, lo, hi, static_cast<unsigned char*>(z));
+  } else {
+    quantize_scalar_kernel<unsigned char><<<grid_for(n, kThreads, 8), kThreads, 0, s>>>(x, 0, n, q, lo, hi, static_cast<unsigned char*>(z));
+  }
+  return check_launch("quantize8");
+}
+
+int q8_quantize_pad_channels(const float* x, size_t pixels, int C, int C_pad, float q, int out_type, void* z, void* stream) {
+  clear_error();
+  if ((!x || !z) && pixels) return fail(Q8_ERR_INVALID_ARG, "q8_quantize_pad_channels: null pointer");
+  if (C <= 0 || C_pad < C) return fail(Q8_ERR_INVALID_ARG, "q8_quantize_pad_channels: need 0 < C <= C_pad");
+  if (!(q > 0.f) || std::isinf(q)) return fail(Q8_ERR_NONFINITE, "q8_quantize_pad_channels: factor must be finite and positive");
+  if (out_type != Q8_U8 && out_type != Q8_S8) return fail(Q8_ERR_INVALID_ARG, "q8_quantize_pad_channels: bad out_type");
+  if (pixels == 0) return Q8_OK;
+  const int lo = out_type == Q8_U8 ? 0 : -128, hi = out_type == Q8_U8 ? 255 : 127;
+  quantize_pad_kernel<unsigned char><<<grid_for(pixels * C_pad, kThreads, 8), kThreads, 0, as_stream(stream)>>>(
+      x, pixels, C, C_pad, q, lo, hi, static_cast<unsigned char*>(z));
+  return check_launch("quantize_pad_kernel");
+}
+
+int q8_dequantize(const void* z, int in_type, size_t n, float q, float* r, void* stream) {
+  clear_error();
+  if ((!z || !r) && n) return fail(Q8_ERR_INVALID_ARG, "q8_dequantize: null pointer");
+  if (in_type != Q8_U8 && in_type != Q8_S8 && in_type != Q8_S32) return fail(Q8_ERR_INVALID_ARG, "q8_dequantize: bad in_type");
+  if (!std::isfinite(q)) return fail(Q8_ERR_NONFINITE, "q8_dequantize: factor must be finite");
+  if (n == 0) return Q8_OK;
+  cudaStream_t s = as_stream(stream);
+  if (in_type == Q8_S32) {
+    dequantize_scalar_kernel<int><<<grid_for(n, kThreads, 8), kThreads, 0, s>>>(static_cast<const int*>(z), 0, n, q, r);
+    return check_launch("dequantize32");
+  }
+  size_t done = 0;
+  if (aligned16(z) && aligned16(r)) {
+    size_t n16 = n / 16;
+    if (n16) {
+      int grid = grid_for(n16, kThreads, 4);
+      if (in_type == Q8_S8) dequantize8_vec_kernel<true><<<grid, kThreads, 0, s>>>(static_cast<const uint4*>(z), n16, q, reinterpret_cast<float4*>(r));
+      else dequantize8_vec_kernel<false><<<grid, kThreads, 0, s>>>(static_cast<const uint4*>(z), n16, q, reinterpret_cast<float4*>(r));
+    }
+    done = n16 * 16;
+  }
+  if (done < n) {
+    int grid = grid_for(n - done, kThreads, 8);
+    if (in_type == Q8_S8) dequantize_scalar_kernel<signed char><<<grid, kThreads, 0, s>>>(static_cast<const signed char*>(z), done, n, q, r);
+    else dequantize_scalar_kernel<unsigned char><<<grid, kThreads, 0, s>>>(static_cast<const unsigned char*>(z), done, n, q, r);
+  }
+  return check_launch("dequantize8");
+}
+
+int q8_fold_bn(const float* w, const float* b, const float* gamma, const float* beta, const float* mean,
+               const float* var, double eps, int K, size_t elems_per_k, float* w_out, float* b_out, void* stream) {
+  clear_error();
+  if (!w || !gamma || !beta || !mean || !var || !w_out || !b_out) return fail(Q8_ERR_INVALID_ARG, "q8_fold_bn: null pointer");
+  if (K <= 0 || K > 65535 || elems_per_k == 0) return fail(Q8_ERR_INVALID_ARG, "q8_fold_bn: need 0 < K <= 65535 and elems_per_k > 0");
+  if (!(eps >= 0.0)) return fail(Q8_ERR_INVALID_ARG, "q8_fold_bn: eps must be >= 0");
+  int chunks = (int)((elems_per_k + 255) / 256);
+  if (chunks > 64) chunks = 64;
+  fold_bn_kernel<<<dim3(chunks, K), 256, 0, as_stream(stream)>>>(w, b, gamma, beta, mean, var, eps, elems_per_k, w_out, b_out);
+  return check_launch("fold_bn_kernel");
+}
+
+int q8_concat(int n_in, const void* const* xs, const int* channels, const float* in_factors, float out_factor,
+              int t, size_t pixels, void* y, void* stream) {
+  clear_error();
+  if (n_in <= 0 || n_in > 8 || !xs || !channels || !in_factors || !y) return fail(Q8_ERR_INVALID_ARG, "q8_concat: bad argument");
+  if (t != Q8_U8 && t != Q8_S8) return fail(Q8_ERR_INVALID_ARG, "q8_concat: type must be Q8_U8 or Q8_S8");
+  if (!(out_factor > 0.f) || std::isinf(out_factor)) return fail(Q8_ERR_NONFINITE, "q8_concat: out_factor must be finite and positive");
+  long long ctot = 0;
+  for (int i = 0; i < n_in; ++i) {
+    if (!xs[i] || channels[i] <= 0) return fail(Q8_ERR_INVALID_ARG, "q8_concat: branch %d null or empty", i);
+    if (!(in_factors[i] > 0.f) || std::isinf(in_factors[i])) return fail(Q8_ERR_NONFINITE, "q8_concat: factor %d not finite positive", i);
+    ctot += channels[i];
+  }
+  if (pixels == 0) return Q8_OK;
+  cudaStream_t s = as_stream(stream);
+  int off = 0;
+  for (int i = 0; i < n_in; ++i) {
+    volatile double ratio = (double)in_factors[i] / (double)out_factor;
+    float sc = (float)ratio;
+    int copy_only = sc == 1.0f;
+    int ch = channels[i];
+    bool vec = (ch % 16 == 0) && (ctot % 16 == 0) && (off % 16 == 0) && aligned16(xs[i]) && aligned16(y);
+    if (vec) {
+      int grid = grid_for(pixels * (ch / 16), kThreads, 4);
+      if (t == Q8_S8) concat_vec_kernel<true><<<grid, kThreads, 0, s>>>(static_cast<const uint4*>(xs[i]), pixels, ch / 16, (int)(ctot / 16), off / 16, sc, copy_only, static_cast<uint4*>(y));
+      else concat_vec_kernel<false><<<grid, kThreads, 0, s>>>(static_cast<const uint4*>(xs[i]), pixels, ch / 16, (int)(ctot / 16), off / 16, sc, copy_only, static_cast<uint4*>(y));
+    } else {
+      int grid = grid_for(pixels * ch, kThreads, 8);
+      if (t == Q8_S8) concat_scalar_kernel<true><<<grid, kThreads, 0, s>>>(static_cast<const unsigned char*>(xs[i]), pixels, ch, (int)ctot, off, sc, copy_only, static_cast<unsigned char*>(y));
+      else concat_scalar_kernel<false><<<grid, kThreads, 0, s>>>(static_cast<const unsigned char*>(xs[i]), pixels, ch, (int)ctot, off, sc, copy_only, static_cast<unsigned char*>(y));
+    }
+    int rc = check_launch("concat_kernel");
+    if (rc != Q8_OK) return rc;
+    off += ch;
+  }
+  return Q8_OK;
+}
+
+int q8_pool_out_extent(int H, int k, int stride, int pad, int ceil_mode, int* out) {
+  clear_error();
+  if (!out || H <= 0 || k <= 0 || stride <= 0 || pad < 0) return fail(Q8_ERR_INVALID_ARG, "q8_pool_out_extent: bad argument");
+  *out = pool_extent(H, k, stride, pad, ceil_mode);
+  return Q8_OK;
+}
+
+int q8_maxpool2d(const void* x, int t, int N, int H, int W, int C, int kh, int kw, int stride_h, int stride_w,
+                 int pad_h, int pad_w, int ceil_mode, void* y, void* stream) {
+  return launch_pool<false>(x, t, N, H, W, C, kh, kw, stride_h, stride_w, pad_h, pad_w, ceil_mode, y, stream);
+}
+
+int q8_avgpool2d(const void* x, int t, int N, int H, int W, int C, int kh, int kw, int stride_h, int stride_w,
+                 int pad_h, int pad_w, int ceil_mode, void* y, void* stream) {
+  return launch_pool<true>(x, t, N, H, W, C, kh, kw, stride_h, stride_w, pad_h, pad_w, ceil_mode, y, stream);
+}
+
+}  // extern "C"

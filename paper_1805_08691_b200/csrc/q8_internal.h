@@ -1,0 +1,54 @@
+// Internal declarations shared by the translation units of libq8 (host side).
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include <cstdarg>
+#include <cstddef>
+#include <cstdint>
+
+#include "q8.h"
+
+namespace q8 {
+
+// Records the message returned by q8_last_error() on this thread and returns `code`.
+int fail(int code, const char* fmt, ...);
+void clear_error();
+
+// Returns Q8_OK or records the CUDA error text and returns Q8_ERR_CUDA.
+int check_cuda(cudaError_t e, const char* what);
+int check_launch(const char* kernel);
+
+// Device status word (bit mask of timeout sites), zero when healthy.
+unsigned int* status_word_device_ptr();
+
+inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline int conv_out_extent(int H, int pad, int dil, int R, int stride) {
+  return (H + 2 * pad - dil * (R - 1) - 1) / stride + 1;
+}
+
+struct ConvArgs {
+  q8_conv_desc d;
+  int P, Q;
+  long long M;  // N*P*Q
+  const void* x;
+  const int8_t* w;
+  const int32_t* bias;
+  const float* scale;
+  const void* residual;
+  float residual_scale;
+  void* y;
+  int ldc, c_off;
+  void* workspace;
+  size_t workspace_bytes;
+  cudaStream_t stream;
+};
+
+// Eligibility of the tensor-core kernel for a descriptor (pointer alignment checked at launch).
+bool umma_shape_eligible(const q8_conv_desc& d, const char** why);
+int launch_conv_umma(const ConvArgs& a);
+int launch_conv_direct(const ConvArgs& a);
+
+}  // namespace q8

@@ -1,0 +1,113 @@
+"""GPU parity of the bandwidth-bound kernels against the CPU oracle (bit-exact)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as o
+
+pytestmark = pytest.mark.gpu
+
+
+def _cuda(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+@pytest.mark.parametrize("n", [0, 1, 5, 16, 1000, 4099, 1 << 20, (1 << 22) + 13])
+def test_maxabs_matches_sequential_scan(q8, n):
+    g = np.random.default_rng(n)
+    r = (g.standard_normal(n) * 3).astype(np.float32)
+    slot = torch.zeros(1, dtype=torch.float32, device="cuda")
+    q8.q8_calibrate_maxabs(_cuda(r), slot)
+    assert slot.item() == o.maxabs(r)
+    # running maximum over a second batch, and an unaligned view
+    r2 = (g.standard_normal(n + 3) * 2).astype(np.float32)
+    t2 = _cuda(r2)
+    q8.q8_calibrate_maxabs(t2[1:], slot)
+    assert slot.item() == o.maxabs(r2[1:], init=o.maxabs(r))
+
+
+@pytest.mark.parametrize("out_type,otype", [(0, o.U8), (1, o.S8), (2, o.S32)])
+@pytest.mark.parametrize("n", [1, 15, 16, 17, 4099, (1 << 20) + 7])
+def test_quantize_bit_exact(q8, out_type, otype, n):
+    g = np.random.default_rng(n + out_type)
+    r = (g.standard_normal(n) * 50).astype(np.float32)
+    r[: min(n, 8)] = np.array([0.5, 1.5, 2.5, -0.5, -1.5, 1e30, -1e30, 254.5], dtype=np.float32)[: min(n, 8)]
+    for qf in (1.0, 0.0437, 0.25):
+        got = q8.q8_quantize(_cuda(r), qf, out_type).cpu().numpy()
+        assert np.array_equal(got, o.quantize(r, qf, otype))
+    # unaligned input view takes the scalar path
+    t = _cuda(np.concatenate([[0], r]).astype(np.float32))
+    got = q8.q8_quantize(t[1:], 0.0437, out_type).cpu().numpy()
+    assert np.array_equal(got, o.quantize(r, 0.0437, otype))
+
+
+def test_quantize_calibrated_extremes(q8):
+    g = np.random.default_rng(3)
+    r = np.maximum(g.standard_normal(100000), 0).astype(np.float32)
+    slot = torch.zeros(1, dtype=torch.float32, device="cuda")
+    q8.q8_calibrate_maxabs(_cuda(r), slot)
+    qf = q8.q8_factor(slot.item(), 8)
+    assert qf == o.factor(o.maxabs(r), 8)
+    z = q8.q8_quantize(_cuda(r), qf, 0)
+    assert int(z.max()) == 255 and np.array_equal(z.cpu().numpy(), o.quantize(r, qf, o.U8))
+
+
+def test_quantize_pad_channels(q8):
+    g = np.random.default_rng(4)
+    x = g.standard_normal((2, 9, 7, 3)).astype(np.float32)
+    got = q8.q8_quantize_pad_channels(_cuda(x), 16, 0.02, 1).cpu().numpy()
+    assert got.shape == (2, 9, 7, 16)
+    assert np.array_equal(got[..., :3], o.quantize(x, 0.02, o.S8)) and np.all(got[..., 3:] == 0)
+
+
+@pytest.mark.parametrize("dt", [np.uint8, np.int8, np.int32])
+@pytest.mark.parametrize("n", [1, 16, 33, 100003])
+def test_dequantize_bit_exact(q8, dt, n):
+    g = np.random.default_rng(n)
+    info = np.iinfo(dt)
+    z = g.integers(max(info.min, -10 ** 6), min(info.max, 10 ** 6) + 1, n).astype(dt)
+    got = q8.q8_dequantize(_cuda(z), 0.0371).cpu().numpy()
+    assert np.array_equal(got, o.dequantize(z, 0.0371))
+
+
+def test_fold_bn_bit_exact(q8):
+    g = np.random.default_rng(5)
+    K, R, S, C = 37, 3, 3, 20
+    w = g.standard_normal((K, R, S, C)).astype(np.float32)
+    b = g.standard_normal(K).astype(np.float32)
+    gamma = g.uniform(0.5, 1.5, K).astype(np.float32)
+    beta = g.standard_normal(K).astype(np.float32)
+    mean = g.standard_normal(K).astype(np.float32)
+    var = g.uniform(0.5, 1.5, K).astype(np.float32)
+    for bias in (b, None):
+        wf, bf = q8.q8_fold_bn(_cuda(w), _cuda(bias) if bias is not None else None, _cuda(gamma), _cuda(beta),
+                               _cuda(mean), _cuda(var), 1e-5)
+        wo, bo = o.fold_bn(w, bias, gamma, beta, mean, var, 1e-5)
+        assert np.array_equal(wf.cpu().numpy(), wo) and np.array_equal(bf.cpu().numpy(), bo)
+
+
+@pytest.mark.parametrize("chans", [(16, 32), (64, 96, 32), (5, 7), (48,)])
+@pytest.mark.parametrize("signed", [False, True])
+def test_concat_bit_exact(q8, chans, signed):
+    g = np.random.default_rng(sum(chans))
+    dt = np.int8 if signed else np.uint8
+    lo, hi = (-128, 128) if signed else (0, 256)
+    xs = [g.integers(lo, hi, (2, 5, 6, c)).astype(dt) for c in chans]
+    fac = [float(np.float32(0.01 * (i + 1))) for i in range(len(chans))]
+    out_f = max(fac)
+    got = q8.q8_concat([_cuda(a) for a in xs], fac, out_f).cpu().numpy()
+    assert np.array_equal(got, o.concat(xs, fac, out_f))
+
+
+@pytest.mark.parametrize("k,st,pad,ceil", [(3, 2, 1, False), (2, 2, 0, True), (3, 1, 1, False), (3, 2, 0, False), (7, 1, 0, False)])
+@pytest.mark.parametrize("C", [64, 5])
+def test_pools_bit_exact(q8, k, st, pad, ceil, C):
+    g = np.random.default_rng(k * 10 + C)
+    x = g.integers(0, 256, (2, 15, 13, C), dtype=np.uint8)
+    got = q8.q8_maxpool2d(_cuda(x), (k, k), (st, st), (pad, pad), ceil).cpu().numpy()
+    assert np.array_equal(got, o.pool(x, "max", (k, k), (st, st), (pad, pad), ceil))
+    got = q8.q8_avgpool2d(_cuda(x), (k, k), (st, st), (pad, pad), ceil).cpu().numpy()
+    assert np.array_equal(got, o.pool(x, "avg", (k, k), (st, st), (pad, pad), ceil))
+    xs = x.view(np.int8)
+    got = q8.q8_maxpool2d(_cuda(xs), (k, k), (st, st), (pad, pad), ceil).cpu().numpy()
+    assert np.array_equal(got, o.pool(xs, "max", (k, k), (st, st), (pad, pad), ceil))
