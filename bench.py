@@ -1,0 +1,338 @@
+#!/usr/bin/env python
+"""Benchmark of the int8 quantized-convolution hot path on the ResNet-50 bottleneck workload.
+
+    python bench.py --gpus N --steps K --warmup W [--impl reference]
+
+One step = one int8 forward of the bottleneck block (1x1 256->64, 3x3 64->64, 1x1 64->256 with fused
+bias, requantisation, ReLU and residual sum) over a batch of 32 56x56x256 u8 images: three launches
+of the tcgen05 convolution kernel through the C ABI.  Prints ONE JSON line (rank 0).
+
+* value      : int8 conv TOPS (2 * MACs / time), inputs resident in HBM, steps replayed as CUDA
+               graphs over rotating buffer sets whose total size exceeds L2.
+* e2e        : same metric with the u8 input copied from pinned host memory and the u8 output copied
+               back inside the timed region.
+* roofline   : dominant kernel, algorithmic bytes / CUDA-event duration against the measured copy peak.
+* cpu_baseline: the CPU oracle timed on a bounded sample of the same workload on the host cores.
+* --impl reference: the oracle alone (there is no reference implementation to install for this paper).
+With N > 1 every rank runs its own batch (weak scaling, replicated weights, no data-path collective).
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+BATCH, H, W, C, MID = 32, 56, 56, 256, 64
+MACS_PER_IMAGE = H * W * (C * MID + 9 * MID * MID + MID * C)
+METRIC = "int8_conv_tops_resnet50_bottleneck_b32"
+UNIT = "TOPS"
+CONFIG = {"workload": "configs[1]: ResNet-50 bottleneck, batch 32, 56x56x256 u8 in, 1x1 256->64 / 3x3 64->64 / "
+                      "1x1 64->256 + identity residual, BN folded, ReLU fused, max-abs factors from 4 seeded batches",
+          "global_batch_per_gpu": BATCH, "parallelism": "replicas"}
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel from
+# the ncu capture summarised under profiles/; None until a capture exists for the current kernel.
+NCU_TRAFFIC_BYTES = {}
+
+
+def layer_bytes(M, Cin, K, R, S, out_bytes=1, residual=False):
+    """Algorithmic bytes of one conv launch: input once, weights, bias, output, residual."""
+    return M * Cin + K * R * S * Cin + 4 * K + M * K * out_bytes + (M * K if residual else 0)
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"], source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, source="fallback")
+
+
+class ClockMonitor:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------ CPU oracle legs
+def oracle_setup(n_images, seed=2000):
+    """Oracle-side preparation of the block on a reduced calibration set; returns (factors, x_q)."""
+    import oracle as o
+    import workloads as wl
+    from oracle import net as oracle_net
+    cfg = wl.config2(seed=seed, batch=n_images, calib_batches=4, calib_batch=2)
+    folded = [o.fold_bn(sp.w, sp.b, sp.gamma, sp.beta, sp.mean, sp.var, 1e-5) for sp in cfg["convs"]]
+    per_batch = []
+    for xb in cfg["calib"]:
+        s = wl.bottleneck_fp32(xb, folded)
+        per_batch.append({k: s[k] for k in ("x", "a", "b", "c")})
+    f = oracle_net.bottleneck_prepare(folded, oracle_net.calib_maxima(per_batch))
+    return f, o.quantize(cfg["x"], f["q_x"], o.U8)
+
+
+def oracle_time_steps(steps, warmup, budget_s=150.0):
+    """Times the oracle's bottleneck forward.  A step is a bounded sample of the batch: one image per
+    host thread when a step of that size fits the time budget, else a single image."""
+    from oracle import net as oracle_net
+    cores = os.cpu_count() or 1
+    threads = min(cores, BATCH)
+    f, xq = oracle_setup(threads)
+    t0 = time.perf_counter()
+    oracle_net.bottleneck_forward(f, xq[:1], threads=1)
+    t1 = time.perf_counter() - t0
+    n = threads if t1 * 1.5 * (steps + warmup) <= budget_s else 1
+    xq = xq[:n]
+    times = []
+    for i in range(warmup + steps):
+        t0 = time.perf_counter()
+        oracle_net.bottleneck_forward(f, xq, threads=n)
+        dt = time.perf_counter() - t0
+        if i >= warmup:
+            times.append(dt)
+    per_step = sum(times) / len(times)
+    tops = 2.0 * MACS_PER_IMAGE * n / per_step / 1e12
+    return dict(value=tops, per_step_s=per_step, images=n, threads=n, total_cores=cores)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    r = oracle_time_steps(args.steps, args.warmup)
+    sample = f"{r['images']} of {BATCH} images per step, one image per thread, oracle loop nest unchanged"
+    line = {"impl": "reference", "metric": METRIC, "value": r["value"], "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": r["per_step_s"] * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "s32", "data": "synthetic",
+            "config": CONFIG,
+            "cpu_baseline": {"value": r["value"], "unit": UNIT, "cores": r["threads"], "kind": "oracle", "sample": sample},
+            "e2e": {"value": r["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------ GPU arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    import paper_1805_08691_b200 as q8
+    from paper_1805_08691_b200 import pipeline
+    import workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the q8 library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def cuda(a):
+        return torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+
+    # ---- preparation (untimed): fold BN, calibrate on 4 seeded batches, quantize weights/bias
+    cfg = wl.config2(seed=2000 + rank, batch=BATCH, calib_batches=4, calib_batch=8)
+    folded = []
+    for sp in cfg["convs"]:
+        folded.append(q8.q8_fold_bn(cuda(sp.w), None, cuda(sp.gamma), cuda(sp.beta), cuda(sp.mean), cuda(sp.var), 1e-5))
+    names = ["x", "a", "b", "c"]
+    cal = pipeline.Calibrator(names, device=dev)
+    folded_np = [(w.cpu().numpy(), b.cpu().numpy()) for w, b in folded]
+    for xb in cfg["calib"]:
+        s = wl.bottleneck_fp32(xb, folded_np, device=dev)
+        for k in names:
+            cal.observe(k, cuda(s[k]))
+    maxima = pipeline.sync_maxima(cal.maxima(), dev if world > 1 else None)
+    shape = (BATCH, H, W, C)
+    x_f32 = cuda(cfg["x"])
+    n_sets = max(2, args.sets)
+    blocks = [pipeline.Bottleneck(folded, maxima, shape) for _ in range(n_sets)]
+    xs = [q8.q8_quantize(x_f32.roll(i, dims=0), blocks[0].q_x, q8.Q8_U8) for i in range(n_sets)]
+    ys = [torch.empty(shape, dtype=torch.uint8, device=dev) for _ in range(n_sets)]
+    del x_f32
+    set_bytes = 2 * BATCH * H * W * C + 2 * BATCH * H * W * MID
+    for lay in (blocks[0].a, blocks[0].b, blocks[0].c):
+        assert q8.q8_conv2d_query_algo(lay.desc) == q8.Q8_ALGO_UMMA
+
+    # eager warm-up (loads kernels, sets attributes) then one CUDA graph per buffer set
+    for i in range(n_sets):
+        blocks[i](xs[i], out=ys[i])
+    torch.cuda.synchronize()
+    q8.q8_read_status()
+    graphs = []
+    for i in range(n_sets):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            blocks[i](xs[i], out=ys[i])
+        graphs.append(g)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(3, args.warmup)):
+        graphs[i % n_sets].replay()
+    barrier()
+    mon = ClockMonitor(local)
+    if rank == 0:
+        mon.start()
+    # keep the monitor sampling for a moment under load before the timed region
+    t_end = time.time() + 0.3
+    i = 0
+    while time.time() < t_end:
+        graphs[i % n_sets].replay()
+        i += 1
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        graphs[i % n_sets].replay()
+    e1.record()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+
+    # ---- per-kernel durations: eager launches bracketed by events, queued behind a delay kernel so
+    # that the GPU never waits for the host between an event and its kernel.
+    ksteps = min(args.steps, 60)
+    evs = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(3)]
+           for _ in range(ksteps)]
+    torch.cuda._sleep(int(2e7))
+    for i in range(ksteps):
+        blk, xq, yq = blocks[i % n_sets], xs[i % n_sets], ys[i % n_sets]
+        evs[i][0][0].record(); blk.a(xq, out=blk.ya); evs[i][0][1].record()
+        evs[i][1][0].record(); blk.b(blk.ya, out=blk.yb); evs[i][1][1].record()
+        evs[i][2][0].record(); blk.c(blk.yb, residual=xq, out=yq); evs[i][2][1].record()
+    barrier()
+    clocks = mon.stop() if rank == 0 else None
+    kms = [statistics.mean(evs[i][j][0].elapsed_time(evs[i][j][1]) for i in range(ksteps)) for j in range(3)]
+
+    # ---- end to end: u8 input from pinned host memory, u8 result back to pinned host memory
+    hx = torch.from_numpy(np.ascontiguousarray(xs[0].cpu().numpy())).pin_memory()
+    hy = torch.empty(shape, dtype=torch.uint8).pin_memory()
+    esteps = max(3, min(args.steps, 20))
+    for i in range(2):
+        xs[i % n_sets].copy_(hx, non_blocking=True)
+        blocks[i % n_sets](xs[i % n_sets], out=ys[i % n_sets])
+        hy.copy_(ys[i % n_sets], non_blocking=True)
+    barrier()
+    e0.record()
+    for i in range(esteps):
+        k = i % n_sets
+        xs[k].copy_(hx, non_blocking=True)
+        blocks[k](xs[k], out=ys[k])
+        hy.copy_(ys[k], non_blocking=True)
+    e1.record()
+    barrier()
+    ms_e2e = e0.elapsed_time(e1) / esteps
+    q8.q8_read_status()
+
+    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, ms_e2e = t.tolist()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    ms_step = ms_total / args.steps
+    ops_step = 2.0 * MACS_PER_IMAGE * BATCH * world
+    peaks = measured_peaks()
+    M = BATCH * H * W
+    kinfo = [("conv_umma 1x1 256->64", layer_bytes(M, C, MID, 1, 1), 2.0 * M * C * MID),
+             ("conv_umma 3x3 64->64", layer_bytes(M, MID, MID, 3, 3), 2.0 * M * 9 * MID * MID),
+             ("conv_umma 1x1 64->256 +res", layer_bytes(M, MID, C, 1, 1, residual=True), 2.0 * M * MID * C)]
+    int8_peak = peaks["bf16_tflops"] * 2.0  # nominal int8:bf16 dense ratio 4.5 : 2.25
+    kernels = []
+    for (name, nbytes, ops), ms in zip(kinfo, kms):
+        kernels.append({"kernel": name, "ms": ms, "GB/s": nbytes / ms / 1e6, "TOPS": ops / ms / 1e9,
+                        "roofline_ms": max(nbytes / peaks["hbm_gbs"] / 1e6, ops / int8_peak / 1e9)})
+    dom = max(range(3), key=lambda j: kms[j])
+    achieved = kinfo[dom][1] / kms[dom] / 1e6
+    roofline = {"bound": "hbm", "kernel": kinfo[dom][0], "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                "algorithmic_bytes_per_launch": kinfo[dom][1], "traffic": NCU_TRAFFIC_BYTES.get(kinfo[dom][0])}
+    line = {"metric": METRIC, "value": ops_step / ms_step / 1e9, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "s32", "data": "synthetic",
+            "config": dict(CONFIG, l2="rotating %d buffer sets of %.0f MB (> 126 MB L2)" % (n_sets, set_bytes / 1e6),
+                           launch="one CUDA graph replay per step"),
+            "clocks": clocks,
+            "e2e": {"value": ops_step / ms_e2e / 1e9, "unit": UNIT, "ms_per_step": ms_e2e,
+                    "h2d_bytes_per_step": BATCH * H * W * C, "d2h_bytes_per_step": BATCH * H * W * C},
+            "gpu_launches": 3 * args.steps,
+            "roofline": roofline, "kernels": kernels,
+            "images_per_s": BATCH * world / ms_step * 1e3}
+    if world == 1 and not args.skip_cpu_baseline:
+        r = oracle_time_steps(steps=2, warmup=1)
+        line["cpu_baseline"] = {"value": r["value"], "unit": UNIT, "cores": r["threads"], "kind": "oracle",
+                                "sample": f"{r['images']} of {BATCH} images per step x 2 steps, one image per thread"}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sets", type=int, default=6, help="rotating buffer sets (working set must exceed L2)")
+    ap.add_argument("--skip-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,7 +1,10 @@
-"""Oracle-side assembly of quantized layers (mirrors the paper's workflow with oracle calls only)."""
+"""Oracle-side assembly of quantized layers: the paper's workflow (fold, calibrate, quantize, run) with oracle calls only.
+
+TEST INFRASTRUCTURE like the rest of this package.
+"""
 import numpy as np
 
-import oracle as o
+from . import q8_oracle as o
 
 
 def prepare_conv(w, b, q_x, q_y, y_type=o.U8, q_res=None):

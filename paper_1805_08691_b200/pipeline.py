@@ -102,3 +102,28 @@ class Bottleneck:
         self.a(x_q, out=self.ya)
         self.b(self.ya, out=self.yb)
         return self.c(self.yb, residual=x_q, out=out)
+
+
+def sync_maxima(maxima: Dict[str, float], device=None) -> Dict[str, float]:
+    """Element-wise MAX of the calibration maxima over all ranks of the default process group.
+
+    The only exchange the data-parallel path needs: with replicated weights and images sharded over
+    GPUs, equal factors on every rank keep the outputs independent of the GPU count.  Returns the
+    input unchanged when no process group is initialised.  `device`: CUDA device for NCCL, None for
+    a CPU (gloo) group.
+    """
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return dict(maxima)
+    names = sorted(maxima)
+    t = torch.tensor([maxima[n] for n in names], dtype=torch.float32, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    vals = t.cpu().tolist()
+    return {n: v for n, v in zip(names, vals)}
+
+
+def shard_batch(n_images: int, rank: int, world: int) -> Tuple[int, int]:
+    """Contiguous [begin, end) slice of a batch owned by `rank` (images are independent units)."""
+    base, extra = divmod(n_images, world)
+    begin = rank * base + min(rank, extra)
+    return begin, begin + base + (1 if rank < extra else 0)
