@@ -2,59 +2,105 @@
 //
 //   D[M = N*P*Q pixels, Cout] (int32, in TMEM) = A[M, R*S*C] (u8/s8) x B[Cout, R*S*C]^T (s8)
 //
-// Persistent kernel: one CTA per SM walks over 128 x BN output tiles.
-//   warp 0    : TMA producer.  A tiles come from the NHWC activation tensor through an im2col tensor
-//               map (one filter tap (r,s) and one channel block per load; padding is the map's zero
-//               fill, the exact code of 0.0 under a symmetric quantizer) or, for 1x1 / stride 1 / no
-//               padding, through a 2-D tiled map.  B tiles come from the KRSC weights through a 3-D
-//               tiled map.  Both land in the K-major swizzled layout tcgen05.mma reads.  The residual
-//               tile of the fused eltwise sum is fetched by TMA as well, ahead of its epilogue.
-//   warp 1    : allocates TMEM (two accumulator buffers), one lane issues tcgen05.mma.kind::i8
-//               (128 x BN x 32 per instruction); tcgen05.commit releases smem stages and publishes
-//               each finished accumulator.
-//   warps 2-9 : epilogue.  tcgen05.ld (one accumulator row per thread), + bias, requantise,
-//               + residual, ReLU, round, clamp, into a swizzled smem tile that one thread hands to a
-//               TMA store.  The epilogue of tile i overlaps the loads and MMAs of tile i+1.
-// Every mbarrier wait is bounded in wall-clock time; on expiry a bit of the library's status word
-// is set and all roles drain instead of hanging.
+// Persistent kernel: one CTA per SM walks over output tiles of 128 accumulator rows x BN channels.
+// A lone control warp executes roughly one instruction every 6-10 cycles and every TMA operation
+// occupies the SM's copy engine for at least ~370 cycles whatever its size, so the pipeline moves
+// few, large pieces:
+//
+//   A operand, three sources
+//     plain  : 1x1 / stride 1 / no padding.  The activation tensor is the [M][C] matrix itself; a
+//              stage holds several consecutive 128 x BK channel blocks (2-D tiled loads).
+//     halo   : stride 1 filters.  A tile is TH x TW output pixels of one image.  One 4-D tiled load
+//              brings the (TH + halo) x (TW + halo) input patch of a channel block, zero filled
+//              outside the image (the exact code of 0.0 under a symmetric quantizer).  Every filter
+//              tap (r, s) is then the same patch read from a start address shifted by
+//              (r*dil_h * patch width + s*dil_w) pixels: accumulator row i = pp * patch width + qq
+//              is output pixel (pp, qq); rows with qq >= TW are computed and dropped.  Each input
+//              byte crosses the L2 port about 1.5 times instead of R*S times.
+//     im2col : everything else (strided, tiny images): one im2col-mode load per tap and channel
+//              block, several of them per stage.
+//   B operand (KRSC weights), three sources
+//     resident : the whole layer's weights sit in shared memory for the CTA's lifetime;
+//     ring     : (halo) one BN x BK tile per tap and channel block through its own ring;
+//     stage    : (plain, im2col) one BN x BK tile next to each A block of a stage.
+//
+// Roles (one lane each unless noted):
+//   thread 0   : TMA producer of A patches / blocks and of B tiles;
+//   thread 32  : tcgen05.mma.kind::i8 issue (128 x BN x 32 per instruction, int32 accumulators in a
+//                ring of up to four TMEM buffers); tcgen05.commit releases stages and publishes
+//                accumulators.  Warp 1 also owns the TMEM allocation;
+//   thread 64  : hands 8-bit tile buffers to the epilogue groups, filled by TMA with the residual
+//                tile of the fused eltwise sum when there is one;
+//   thread 96  : sends finished 8-bit tiles to global memory with TMA stores, recycles the buffers;
+//   warps 4..  : G epilogue groups of four warps; group g owns every G-th tile of the CTA.  A thread
+//                owns one accumulator row: tcgen05.ld, + bias, requantise, + residual, ReLU, round,
+//                clamp; the 16 bytes go back into the buffer the residual came from (same swizzled
+//                position), which then is the source of the TMA store.
+// All hand-offs are mbarriers, there is no block-wide barrier after the prologue.  Every wait is
+// bounded in wall-clock time; on expiry a bit of the library's status word is set and all roles drain
+// instead of hanging.
 #include <cuda.h>
 
+#include <cstdlib>
 #include <cstring>
 #include <initializer_list>
 
-#include "q8_epilogue.cuh"
 #include "q8_internal.h"
 
 namespace q8 {
 namespace {
 
 constexpr int kBM = 128;
-constexpr int kEpiWarps = 8;
-constexpr int kEpiThreads = kEpiWarps * 32;
-constexpr int kUmmaThreads = 64 + kEpiThreads;
+constexpr int kCtrlThreads = 128;       // warps 0-3
+constexpr int kGroupThreads = 128;      // one epilogue group
+constexpr int kMaxStages = 8;           // A stages
+constexpr int kMaxBStages = 8;          // weight ring
+constexpr int kMaxAcc = 4;
+constexpr int kMaxSlots = 8;            // 8-bit tile buffers over all groups
+constexpr int kMaxGroups = 4;
+constexpr int kMaxTaps = 64;            // halo mode keeps a descriptor offset per tap in shared memory
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
 constexpr int kSmemLimit = 232448;                           // 227 KiB opt-in maximum per CTA
-constexpr int kStaticSmemReserve = 4096;                     // barriers, bias/scale staging
+constexpr int kStaticSmemReserve = 2048;                     // barriers, tap table and flags
 
 enum StatusBits : unsigned int {
   kTimeoutProducer = 1u,
   kTimeoutMma = 2u,
   kTimeoutEpilogue = 4u,
+  kTimeoutResidual = 8u,
+  kTimeoutStore = 16u,
 };
 
 enum ResMode : int { kResNone = 0, kResTma = 1, kResGlobal = 2 };
+enum AMode : int { kAPlain = 0, kAIm2col = 1, kAHalo = 2 };
+enum BMode : int { kBStage = 0, kBResident = 1, kBRing = 2 };
 
 struct UmmaParams {
   int M, K;                  // GEMM rows (pixels) and Cout
-  int PQ, Q;                 // pixels per image, output width
+  int P, Q, PQ;              // output height, width, pixels per image
   int stride_h, stride_w, pad_h, pad_w, dil_h, dil_w;
-  int S;                     // filter width
-  int c_blocks;              // ceil(C / BK)
-  int k_iters;               // R * S * c_blocks
-  int stages;                // smem stages in use (<= template maximum)
+  int R, S, taps;            // filter height, width, R * S
+  int C_pad, c_blocks;       // channels rounded up to whole K blocks, number of K blocks
+  int bn, bk, ksteps;        // tile width (multiple of 16), K bytes per block (32/64/128), bk / 32
+  int a_mode, b_mode;
+  int k_iters, kb;           // plain/im2col: taps * c_blocks (tap, block) iterations, kb of them per A stage
+  int tw, th, twb, hb;       // halo: tile and patch extents in pixels
+  int p_tiles, q_tiles;      // halo: tiles per image column / row
+  int stages, b_stages;      // A stages, weight-ring stages
+  int nacc, acc_stride, tmem_cols;  // TMEM accumulators, columns between them, allocation (power of two)
+  int nbuf;                  // 8-bit tile buffers per epilogue group (0: none)
   int m_tiles, n_tiles;
-  int a_im2col;              // 1: im2col tensor map, 0: 2-D tiled [M][C]
   unsigned int idesc;        // tcgen05 instruction descriptor
+  unsigned int desc_hi;      // high word of the shared-memory matrix descriptors
+  unsigned int a_sub_bytes;  // plain/im2col: one 128 x bk block; halo: bytes of one patch load
+  unsigned int b_tile_bytes; // bn * bk
+  unsigned int b_sub_bytes;  // b_tile_bytes rounded up to 1 KiB (placement inside a stage / the ring)
+  unsigned int a_stage_bytes;
+  unsigned int tile8_bytes;
+  unsigned int res_tx_bytes; // bytes one residual tile load delivers
+  unsigned int off_a, off_bring, off_bufs, off_chan;  // from the 1 KiB aligned base; resident weights at 0
+  int pw_shift, pmask, panels;  // 8-bit tiles live in smem as panels of 2^pw_shift bytes per row
+  int k_pad;                 // n_tiles * bn channels of bias/scale staged in smem
   const int* bias;
   const float* scale;
   int scale_count;
@@ -62,8 +108,48 @@ struct UmmaParams {
   int res_mode, res_signed;
   float res_scale;
   void* y;
-  int y_type, y_vec, y_tma, ldc, c_off, relu;
+  int y_type, y_vec, out8, ldc, c_off, relu;
   unsigned int* status;
+};
+
+// Walks the tiles of one role: tile = first, first + step, ...; tile -> (m tile, n tile) with the
+// n tiles of one m tile adjacent (they share the A operand through L2), and for halo tiles
+// m tile -> (image, tile row, tile column).  Only additions after init().
+struct TileIter {
+  int tile, step;
+  int mt, nt;        // m tile, n tile
+  int img, pt, qt;   // halo: image, tile row, tile column
+  int d_mt, d_nt, d_img, d_pt, d_qt;
+
+  __device__ __forceinline__ void init(const UmmaParams& p, int first, int step_) {
+    tile = first; step = step_;
+    mt = first / p.n_tiles; nt = first - mt * p.n_tiles;
+    d_mt = step_ / p.n_tiles; d_nt = step_ - d_mt * p.n_tiles;
+    img = pt = qt = d_img = d_pt = d_qt = 0;
+    if (p.a_mode == kAHalo) {
+      const int per_img = p.p_tiles * p.q_tiles;
+      img = mt / per_img;
+      int r = mt - img * per_img;
+      pt = r / p.q_tiles; qt = r - pt * p.q_tiles;
+      d_img = d_mt / per_img;
+      r = d_mt - d_img * per_img;
+      d_pt = r / p.q_tiles; d_qt = r - d_pt * p.q_tiles;
+    }
+  }
+  __device__ __forceinline__ void next(const UmmaParams& p) {
+    tile += step;
+    int carry = 0;
+    nt += d_nt;
+    if (nt >= p.n_tiles) { nt -= p.n_tiles; carry = 1; }
+    mt += d_mt + carry;
+    if (p.a_mode == kAHalo) {
+      qt += d_qt + carry; carry = 0;
+      if (qt >= p.q_tiles) { qt -= p.q_tiles; carry = 1; }
+      pt += d_pt + carry; carry = 0;
+      if (pt >= p.p_tiles) { pt -= p.p_tiles; carry = 1; }
+      img += d_img + carry;
+    }
+  }
 };
 
 // ------------------------------------------------------------------------------------------ PTX
@@ -99,19 +185,26 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Waits for the phase with the given parity.  Gives up after kWaitLimitNs or when another role of
-// this CTA has already given up; the caller then records the site and leaves its loop.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_timer_ns();
+// Slow path of a wait, out of line to keep the role loops small.  Gives up after about
+// kWaitLimitNs or when another role of this CTA has already given up; the caller then records the
+// site and leaves its loop.  The wall clock is only read once the wait has lasted a while.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  unsigned long long t0 = 0;
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
-    if ((++spins & 0xffu) == 0) {
+    if ((++spins & 0x3ffu) == 0) {
       if (*abort_flag) return false;
-      if (global_timer_ns() - t0 > kWaitLimitNs) return false;
+      const unsigned long long now = global_timer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) return false;
     }
   }
   return true;
+}
+
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag);
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
@@ -139,6 +232,19 @@ __device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const CUtensorM
       : "memory");
 }
 
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+               ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+               : "memory");
+}
+
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
                ::"l"(map), "r"(src), "r"(c0), "r"(c1)
@@ -147,7 +253,6 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t sr
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
@@ -167,14 +272,35 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
   asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
 }
 
-// D[tmem] (+)= A[smem desc] * B[smem desc]^T, 8-bit integer inputs, int32 accumulate.
-__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+// D[tmem] (+)= A[smem desc] * B[smem desc]^T, 8-bit integer inputs, int32 accumulate.  The 64-bit
+// shared-memory descriptors are handed over as (low, high) words: only the low word (start address)
+// changes between instructions.
+__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                        uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "mov.b64 da, {%1, %2};\n\t"
+      "mov.b64 db, {%3, %4};\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %5, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
       : "memory");
+}
+
+// kSteps instructions over one K block of kSteps * 32 bytes: +2 in 16-byte address units per step.
+template <int kSteps>
+__device__ __forceinline__ void umma_i8_block(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                              uint32_t idesc, uint32_t accumulate_first) {
+  umma_i8(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate_first);
+#pragma unroll
+  for (int k = 1; k < kSteps; ++k) umma_i8(d_tmem, a_lo + 2 * k, a_hi, b_lo + 2 * k, b_hi, idesc, 1u);
+}
+
+__device__ __forceinline__ void umma_i8_ksteps(int ksteps, uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
+                                               uint32_t b_hi, uint32_t idesc, uint32_t accumulate_first) {
+  if (ksteps == 4) umma_i8_block<4>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate_first);
+  else if (ksteps == 2) umma_i8_block<2>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate_first);
+  else umma_i8_block<1>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate_first);
 }
 
 // The mbarrier gets one arrival once every tcgen05.mma issued so far by this thread has completed.
@@ -190,85 +316,256 @@ __device__ __forceinline__ void tmem_ld_16(uint32_t taddr, int (&v)[16]) {
         "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
       : "r"(taddr));
 }
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
-
-// Shared-memory matrix descriptor of a K-major operand tile whose rows are BK bytes (= one swizzle
-// span): 8-row groups are 8*BK bytes apart (stride byte offset), the leading byte offset is unused
-// for swizzled K-major tiles and set to 1, descriptor version 1, swizzle mode from BK.
-template <int BK>
-__device__ __forceinline__ uint64_t make_kmajor_desc(uint32_t smem_addr) {
-  constexpr uint64_t layout = BK == 128 ? 2 : (BK == 64 ? 4 : 6);
-  return (uint64_t)((smem_addr >> 4) & 0x3fffu) | (1ull << 16) | ((uint64_t)((8 * BK) >> 4) << 32) | (1ull << 46) |
-         (layout << 61);
+// Waits for this thread's TMEM loads.  The registers are named as operands so that no use of them
+// can be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_ld_wait(int (&v)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]), "+r"(v[8]),
+                 "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15])
+               :
+               : "memory");
 }
 
-__device__ __forceinline__ unsigned int pack4(int a, int b, int c, int d) {
-  return (unsigned int)(a & 0xff) | ((unsigned int)(b & 0xff) << 8) | ((unsigned int)(c & 0xff) << 16) |
-         ((unsigned int)(d & 0xff) << 24);
+// {lo byte, next byte} = {sat(b), sat(a)}, upper half = low half of c.
+__device__ __forceinline__ unsigned int pack_sat_u8(int a, int b, unsigned int c) {
+  unsigned int d;
+  asm("cvt.pack.sat.u8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+__device__ __forceinline__ unsigned int pack_sat_s8(int a, int b, unsigned int c) {
+  unsigned int d;
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+// bytes (z0, z1, z2, z3), z0 lowest, each saturated to the 8-bit range
+template <bool kSigned>
+__device__ __forceinline__ unsigned int pack4_sat(int z0, int z1, int z2, int z3) {
+  return kSigned ? pack_sat_s8(z1, z0, pack_sat_s8(z3, z2, 0u)) : pack_sat_u8(z1, z0, pack_sat_u8(z3, z2, 0u));
 }
 
-// TMEM columns for two accumulator buffers of BN columns (power of two, at least 32).
-__host__ __device__ constexpr int tmem_cols_for(int bn) { return bn <= 16 ? 32 : (bn <= 32 ? 64 : (bn <= 64 ? 128 : (bn <= 128 ? 256 : 512))); }
-// 8-bit output / residual tiles are kept in smem as panels of at most one 128-byte swizzle span;
-// panel_mask is the XOR mask the TMA swizzle applies to 16-byte chunk indices.
-__host__ __device__ constexpr int panel_bytes_for(int bn) { return bn < 128 ? bn : 128; }
-__host__ __device__ constexpr int panel_mask_for(int pw) { return pw == 128 ? 7 : (pw == 64 ? 3 : (pw == 32 ? 1 : 0)); }
+// ------------------------------------------------------------------------------------------ epilogue
+struct EpiTile {
+  const int* s_bias;       // smem, k_pad entries
+  const float* s_scale;    // smem, k_pad entries
+  unsigned char* buf;      // this tile's 8-bit buffer (residual in, output out) or nullptr
+  long long m;             // output pixel (row of the [M][Cout] result) of this thread
+  int srow;                // row of this thread's pixel inside the 8-bit tile buffer
+  int n0;                  // first channel of the tile
+  bool row_ok;             // the pixel exists (inside the image and below M)
+  bool smem_ok;            // this accumulator row maps to a pixel of the tile (always, except halo tiles)
+};
+
+// One 16-column chunk of one accumulator row.  kOut: Q8_U8, Q8_S8, Q8_S32 or Q8_F32.
+//   v = float(acc + bias) * s;  v += float(res) * s_res;  v = max(v, 0);  y = clamp(Round(v))
+// Each step is one IEEE fp32 operation (the library is built without FMA contraction).
+template <int kOut, int kRes>
+__device__ __forceinline__ void epilogue_chunk(const UmmaParams& p, const EpiTile& t, int ch, const int (&raw)[16]) {
+  const int c16 = ch * 16;
+  const int nb = t.n0 + c16;
+  int acc[16];
+  {
+    const int4* bp = reinterpret_cast<const int4*>(t.s_bias + nb);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int4 b = bp[j];
+      acc[4 * j] = raw[4 * j] + b.x; acc[4 * j + 1] = raw[4 * j + 1] + b.y;
+      acc[4 * j + 2] = raw[4 * j + 2] + b.z; acc[4 * j + 3] = raw[4 * j + 3] + b.w;
+    }
+  }
+  if (kOut == Q8_S32) {
+    if (t.row_ok && nb < p.K) {
+      const int valid = min(16, p.K - nb);
+      int* yp = static_cast<int*>(p.y) + (size_t)t.m * p.ldc + p.c_off + nb;
+      if (p.y_vec && valid == 16) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) reinterpret_cast<int4*>(yp)[j] = make_int4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          if (j < valid) yp[j] = acc[j];
+      }
+    }
+    return;
+  }
+  // position of this thread's 16 bytes inside the swizzled 8-bit tile buffer
+  uint32_t off = 0;
+  if (kOut == Q8_U8 || kOut == Q8_S8 || kRes == kResTma) {
+    const int pn = c16 >> p.pw_shift;
+    off = ((uint32_t)t.srow << p.pw_shift) + (uint32_t)(c16 & ((1 << p.pw_shift) - 1));
+    off ^= ((off >> 7) & (uint32_t)p.pmask) << 4;
+    off += (uint32_t)pn * ((uint32_t)kBM << p.pw_shift);
+  }
+  float v[16];
+  {
+    const float4* sp = reinterpret_cast<const float4*>(t.s_scale + nb);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float4 s = sp[j];
+      v[4 * j] = __fmul_rn(__int2float_rn(acc[4 * j]), s.x);
+      v[4 * j + 1] = __fmul_rn(__int2float_rn(acc[4 * j + 1]), s.y);
+      v[4 * j + 2] = __fmul_rn(__int2float_rn(acc[4 * j + 2]), s.z);
+      v[4 * j + 3] = __fmul_rn(__int2float_rn(acc[4 * j + 3]), s.w);
+    }
+  }
+  if (kRes != kResNone) {
+    unsigned int rw[4] = {0u, 0u, 0u, 0u};
+    if (kRes == kResTma) {
+      const uint4 rv = *reinterpret_cast<const uint4*>(t.buf + off);
+      rw[0] = rv.x; rw[1] = rv.y; rw[2] = rv.z; rw[3] = rv.w;
+    } else if (t.row_ok && nb < p.K) {
+      const int valid = min(16, p.K - nb);
+      const unsigned char* rp = p.res + (size_t)t.m * p.K + nb;
+#pragma unroll
+      for (int j = 0; j < 16; ++j)
+        if (j < valid) rw[j >> 2] |= (unsigned int)rp[j] << (8 * (j & 3));
+    }
+    // byte b -> float without a conversion instruction: 0x4B0000bb is 2^23 + b exactly; a signed
+    // byte is first biased by 128
+    const unsigned int sign_mask = p.res_signed ? 0x80808080u : 0u;
+    const float magic = p.res_signed ? 8388736.0f : 8388608.0f;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const unsigned int w = rw[j >> 2] ^ sign_mask;
+      const float r = __fsub_rn(__uint_as_float(__byte_perm(w, 0x4B000000u, 0x7540u | (unsigned)(j & 3))), magic);
+      v[j] = __fadd_rn(v[j], __fmul_rn(r, p.res_scale));
+    }
+  }
+  if (kOut == Q8_F32) {
+    if (p.relu) {
+#pragma unroll
+      for (int j = 0; j < 16; ++j) v[j] = fmaxf(v[j], 0.0f);
+    }
+    if (t.row_ok && nb < p.K) {
+      const int valid = min(16, p.K - nb);
+      float* yp = static_cast<float*>(p.y) + (size_t)t.m * p.ldc + p.c_off + nb;
+      if (p.y_vec && valid == 16) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) reinterpret_cast<float4*>(yp)[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          if (j < valid) yp[j] = v[j];
+      }
+    }
+    return;
+  }
+  // 8-bit output: the saturating pack clamps to [0,255] (which also is the ReLU) or [-128,127]
+  if (kOut == Q8_S8 && p.relu) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v[j] = fmaxf(v[j], 0.0f);
+  }
+  int z[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) z[j] = __float2int_rn(v[j]);
+  uint4 o;
+  o.x = pack4_sat<kOut == Q8_S8>(z[0], z[1], z[2], z[3]);
+  o.y = pack4_sat<kOut == Q8_S8>(z[4], z[5], z[6], z[7]);
+  o.z = pack4_sat<kOut == Q8_S8>(z[8], z[9], z[10], z[11]);
+  o.w = pack4_sat<kOut == Q8_S8>(z[12], z[13], z[14], z[15]);
+  if (t.smem_ok) *reinterpret_cast<uint4*>(t.buf + off) = o;
+}
+
+// All chunks of one accumulator row, TMEM loads one chunk ahead of the arithmetic.  The accumulator
+// is released (acc_empty) as soon as its last chunk is in registers.
+template <int kOut, int kRes>
+__device__ __forceinline__ void epilogue_row(const UmmaParams& p, const EpiTile& t, uint32_t taddr, uint32_t acc_empty_bar,
+                                             int lane) {
+  const int nchunk = p.bn >> 4;
+  int ra[16], rb[16];
+  tmem_ld_16(taddr, ra);
+#pragma unroll 1
+  for (int ch = 0; ch < nchunk; ch += 2) {
+    tmem_ld_wait(ra);
+    const bool more1 = ch + 1 < nchunk;
+    if (more1) tmem_ld_16(taddr + (ch + 1) * 16, rb);
+    else {
+      // every accumulator value of this warp is in registers: hand the TMEM buffer back
+      tcgen05_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acc_empty_bar);
+    }
+    epilogue_chunk<kOut, kRes>(p, t, ch, ra);
+    if (more1) {
+      tmem_ld_wait(rb);
+      const bool more2 = ch + 2 < nchunk;
+      if (more2) tmem_ld_16(taddr + (ch + 2) * 16, ra);
+      else {
+        tcgen05_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acc_empty_bar);
+      }
+      epilogue_chunk<kOut, kRes>(p, t, ch + 1, rb);
+    }
+  }
+}
 
 // ------------------------------------------------------------------------------------------ kernel
-template <int BN, int BK, int MAX_STAGES>
-__global__ void __launch_bounds__(kUmmaThreads, 1) conv_umma_kernel(const __grid_constant__ CUtensorMap tmA,
-                                                                    const __grid_constant__ CUtensorMap tmB,
-                                                                    const __grid_constant__ CUtensorMap tmRes,
-                                                                    const __grid_constant__ CUtensorMap tmY,
-                                                                    const UmmaParams p) {
-  constexpr uint32_t A_BYTES = kBM * BK, B_BYTES = BN * BK, STAGE_BYTES = A_BYTES + B_BYTES;
-  constexpr uint32_t TMEM_COLS = tmem_cols_for(BN);
-  constexpr int PW = panel_bytes_for(BN), PANELS = BN / PW, PMASK = panel_mask_for(PW);
-  constexpr uint32_t TILE8_BYTES = kBM * BN;  // one 8-bit output / residual tile
-  constexpr int NCHUNK = BN / 16;
-
+// G epilogue groups; one instantiation per output type and residual source keeps a single epilogue
+// body in each kernel (several of them in one kernel made the register allocator spill).
+template <int G, int kOut, int kRes>
+__global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
+    conv_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                     const __grid_constant__ CUtensorMap tmRes, const __grid_constant__ CUtensorMap tmY,
+                     const __grid_constant__ UmmaParams p) {
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long full_bar[MAX_STAGES];
-  __shared__ __align__(8) unsigned long long empty_bar[MAX_STAGES];
-  __shared__ __align__(8) unsigned long long acc_full[2], acc_empty[2], res_full[2], res_empty[2];
+  __shared__ __align__(8) unsigned long long a_full[kMaxStages], a_empty[kMaxStages];
+  __shared__ __align__(8) unsigned long long b_full[kMaxBStages], b_empty[kMaxBStages];
+  __shared__ __align__(8) unsigned long long acc_full[kMaxAcc], acc_empty[kMaxAcc];
+  __shared__ __align__(8) unsigned long long buf_full[kMaxSlots], buf_empty[kMaxSlots];
+  __shared__ __align__(8) unsigned long long store_ready[kMaxGroups];
+  __shared__ __align__(8) unsigned long long bres_full;
+  __shared__ uint32_t tap_shift16[kMaxTaps];  // halo: descriptor start offset of a tap, in 16-byte units
   __shared__ uint32_t tmem_holder;
   __shared__ int abort_flag;
-  __shared__ int epi_ok;
-  __shared__ float s_scale[BN];
-  __shared__ int s_bias[BN];
 
-  // dynamic smem: [stages][A|B], then two 8-bit output staging tiles, then two residual tiles
+  // dynamic smem: [resident weights] [A stages] [weight ring] [G*nbuf 8-bit tile buffers] [bias, scale]
   const uint32_t raw_base = smem_u32(smem_raw);
-  const uint32_t tiles_base = (raw_base + 1023u) & ~1023u;
-  const int stages = p.stages;
-  const uint32_t out_base = (tiles_base + (uint32_t)stages * STAGE_BYTES + 1023u) & ~1023u;
-  const uint32_t res_base = out_base + (p.y_tma ? 2u * TILE8_BYTES : 0u);
+  const uint32_t base = (raw_base + 1023u) & ~1023u;
+  unsigned char* const base_ptr = smem_raw + (base - raw_base);
+  int* const s_bias = reinterpret_cast<int*>(base_ptr + p.off_chan);
+  float* const s_scale = reinterpret_cast<float*>(base_ptr + p.off_chan) + p.k_pad;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int total_tiles = p.m_tiles * p.n_tiles;
+  const int slots = G * p.nbuf;
 
   if (threadIdx.x == 0) {
     prefetch_tensormap(&tmA);
     prefetch_tensormap(&tmB);
     if (p.res_mode == kResTma) prefetch_tensormap(&tmRes);
-    if (p.y_tma) prefetch_tensormap(&tmY);
-    for (int s = 0; s < stages; ++s) {
-      mbar_init(smem_u32(&full_bar[s]), 1);
-      mbar_init(smem_u32(&empty_bar[s]), 1);
+    if (p.out8) prefetch_tensormap(&tmY);
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(smem_u32(&a_full[s]), 1);
+      mbar_init(smem_u32(&a_empty[s]), 1);
     }
-    for (int i = 0; i < 2; ++i) {
+    for (int s = 0; s < p.b_stages; ++s) {
+      mbar_init(smem_u32(&b_full[s]), 1);
+      mbar_init(smem_u32(&b_empty[s]), 1);
+    }
+    for (int i = 0; i < p.nacc; ++i) {
       mbar_init(smem_u32(&acc_full[i]), 1);
-      mbar_init(smem_u32(&acc_empty[i]), 1);
-      mbar_init(smem_u32(&res_full[i]), 1);
-      mbar_init(smem_u32(&res_empty[i]), 1);
+      mbar_init(smem_u32(&acc_empty[i]), 4);  // one arrival per epilogue warp of the owning group
     }
+    for (int i = 0; i < slots; ++i) {
+      mbar_init(smem_u32(&buf_full[i]), 1);
+      mbar_init(smem_u32(&buf_empty[i]), 1);
+    }
+    for (int g = 0; g < G; ++g) mbar_init(smem_u32(&store_ready[g]), kGroupThreads);
+    mbar_init(smem_u32(&bres_full), 1);
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(&tmem_holder), TMEM_COLS);
+    tmem_alloc(smem_u32(&tmem_holder), (uint32_t)p.tmem_cols);
     tmem_relinquish();
+  }
+  if (p.a_mode == kAHalo && threadIdx.x < p.taps) {
+    const int r = threadIdx.x / p.S, s = threadIdx.x - r * p.S;
+    tap_shift16[threadIdx.x] = (uint32_t)((r * p.dil_h * p.twb + s * p.dil_w) * p.bk) >> 4;
+  }
+  // bias and scale of every channel, once per CTA (zero beyond Cout; one scale replicated if per tensor)
+  for (int i = threadIdx.x; i < p.k_pad; i += blockDim.x) {
+    s_bias[i] = (p.bias && i < p.K) ? p.bias[i] : 0;
+    s_scale[i] = p.scale ? (p.scale_count == 1 ? p.scale[0] : (i < p.K ? p.scale[i] : 0.f)) : 0.f;
   }
   tcgen05_fence_before();
   __syncthreads();
@@ -277,43 +574,83 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) conv_umma_kernel(const __grid
   volatile int* abortp = &abort_flag;
 
   if (threadIdx.x == 0) {
-    // ------------------------------------------------------------------ TMA producer
-    int stage = 0;
-    uint32_t phase = 0;
-    int lt = 0;
+    // ------------------------------------------------------------------ A / B producer
+    TileIter ti;
+    ti.init(p, blockIdx.x, gridDim.x);
+    const uint32_t nstages = (uint32_t)p.stages, nbst = (uint32_t)p.b_stages;
+    const uint32_t afull0 = smem_u32(&a_full[0]), aempty0 = smem_u32(&a_empty[0]);
+    const uint32_t bfull0 = smem_u32(&b_full[0]), bempty0 = smem_u32(&b_empty[0]);
+    const uint32_t a0 = base + p.off_a, bring0 = base + p.off_bring;
+    uint32_t stage = 0, phase = 0, a_dst = a0;
+    uint32_t bs = 0, bphase = 0, b_dst = bring0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++lt) {
-      const int m0 = (tile / p.n_tiles) * kBM, n0 = (tile % p.n_tiles) * BN;
-      if (p.res_mode == kResTma) {
-        const int rb = lt & 1;
-        if (!mbar_wait(smem_u32(&res_empty[rb]), ((uint32_t)(lt >> 1) & 1u) ^ 1u, abortp)) { ok = false; break; }
-        const uint32_t bar = smem_u32(&res_full[rb]);
-        mbar_arrive_expect_tx(bar, TILE8_BYTES);
-#pragma unroll
-        for (int pn = 0; pn < PANELS; ++pn)
-          tma_load_2d(res_base + rb * TILE8_BYTES + pn * (kBM * PW), &tmRes, bar, n0 + pn * PW, m0);
+    if (p.b_mode == kBResident) {
+      // every weight tile of the layer, once: one load per (n tile, channel block) brings all taps,
+      // laid out [tap][bn rows][bk bytes], i.e. one K-major operand tile per tap
+      const uint32_t bar = smem_u32(&bres_full);
+      mbar_arrive_expect_tx(bar, (uint32_t)(p.n_tiles * p.c_blocks * p.taps) * p.b_tile_bytes);
+      uint32_t dst = base;
+      for (int nt = 0; nt < p.n_tiles; ++nt)
+        for (int c = 0; c < p.C_pad; c += p.bk, dst += (uint32_t)p.taps * p.b_tile_bytes) tma_load_3d(dst, &tmB, bar, c, nt * p.bn, 0);
+    }
+    if (p.a_mode == kAHalo) {
+      for (; ti.tile < total_tiles && ok; ti.next(p)) {
+        const int n0 = ti.nt * p.bn, q0 = ti.qt * p.tw - p.pad_w, p0 = ti.pt * p.th - p.pad_h;
+        for (int c = 0; c < p.C_pad && ok; c += p.bk) {
+          if (!mbar_wait(aempty0 + stage * 8u, phase ^ 1u, abortp)) { ok = false; break; }
+          const uint32_t bar = afull0 + stage * 8u;
+          mbar_arrive_expect_tx(bar, p.a_sub_bytes);
+          tma_load_4d(a_dst, &tmA, bar, c, q0, p0, ti.img);
+          a_dst += p.a_stage_bytes;
+          if (++stage == nstages) { stage = 0; phase ^= 1u; a_dst = a0; }
+          if (p.b_mode == kBRing) {
+            for (int tap = 0; tap < p.taps; ++tap) {
+              if (!mbar_wait(bempty0 + bs * 8u, bphase ^ 1u, abortp)) { ok = false; break; }
+              const uint32_t bbar = bfull0 + bs * 8u;
+              mbar_arrive_expect_tx(bbar, p.b_tile_bytes);
+              tma_load_3d(b_dst, &tmB, bbar, c, tap, n0);
+              b_dst += p.b_sub_bytes;
+              if (++bs == nbst) { bs = 0; bphase ^= 1u; b_dst = bring0; }
+            }
+          }
+        }
       }
-      int w0 = 0, h0 = 0, img = 0;
-      if (p.a_im2col) {
-        img = m0 / p.PQ;
-        const int rem = m0 - img * p.PQ;
-        const int p0 = rem / p.Q, q0 = rem - p0 * p.Q;
-        h0 = p0 * p.stride_h - p.pad_h;
-        w0 = q0 * p.stride_w - p.pad_w;
-      }
-      int r = 0, s = 0, cb = 0;
-      for (int it = 0; it < p.k_iters; ++it) {
-        if (!mbar_wait(smem_u32(&empty_bar[stage]), phase ^ 1u, abortp)) { ok = false; break; }
-        const uint32_t bar = smem_u32(&full_bar[stage]);
-        const uint32_t a_dst = tiles_base + stage * STAGE_BYTES, b_dst = a_dst + A_BYTES;
-        mbar_arrive_expect_tx(bar, STAGE_BYTES);
-        if (p.a_im2col)
-          tma_load_im2col_4d(a_dst, &tmA, bar, cb * BK, w0, h0, img, (unsigned short)(s * p.dil_w), (unsigned short)(r * p.dil_h));
-        else
-          tma_load_2d(a_dst, &tmA, bar, cb * BK, m0);
-        tma_load_3d(b_dst, &tmB, bar, cb * BK, r * p.S + s, n0);
-        if (++cb == p.c_blocks) { cb = 0; if (++s == p.S) { s = 0; ++r; } }
-        if (++stage == stages) { stage = 0; phase ^= 1u; }
+    } else {
+      const uint32_t sub_tx = p.a_sub_bytes + (p.b_mode == kBStage ? p.b_tile_bytes : 0u);
+      const uint32_t b_in_stage = (uint32_t)p.kb * p.a_sub_bytes;
+      for (; ti.tile < total_tiles && ok; ti.next(p)) {
+        const int m0 = ti.mt * kBM, n0 = ti.nt * p.bn;
+        int w0 = 0, h0 = 0, img = 0;
+        if (p.a_mode == kAIm2col) {
+          img = m0 / p.PQ;
+          const int rem = m0 - img * p.PQ;
+          const int pr = rem / p.Q, qc = rem - pr * p.Q;
+          h0 = pr * p.stride_h - p.pad_h;
+          w0 = qc * p.stride_w - p.pad_w;
+        }
+        int c = 0, tap = 0, s = 0, off_w = 0, off_h = 0;
+        for (int it = 0; it < p.k_iters;) {
+          const int nsub = min(p.kb, p.k_iters - it);
+          if (!mbar_wait(aempty0 + stage * 8u, phase ^ 1u, abortp)) { ok = false; break; }
+          const uint32_t bar = afull0 + stage * 8u;
+          mbar_arrive_expect_tx(bar, (uint32_t)nsub * sub_tx);
+          uint32_t dst = a_dst, bdst = a_dst + b_in_stage;
+          for (int j = 0; j < nsub; ++j) {
+            if (p.a_mode == kAIm2col) tma_load_im2col_4d(dst, &tmA, bar, c, w0, h0, img, (unsigned short)off_w, (unsigned short)off_h);
+            else tma_load_2d(dst, &tmA, bar, c, m0);
+            if (p.b_mode == kBStage) tma_load_3d(bdst, &tmB, bar, c, tap, n0);
+            dst += p.a_sub_bytes;
+            bdst += p.b_sub_bytes;
+            c += p.bk;
+            if (c >= p.C_pad) {  // next tap
+              c = 0; ++tap; ++s; off_w += p.dil_w;
+              if (s == p.S) { s = 0; off_w = 0; off_h += p.dil_h; }
+            }
+          }
+          it += nsub;
+          a_dst += p.a_stage_bytes;
+          if (++stage == nstages) { stage = 0; phase ^= 1u; a_dst = a0; }
+        }
       }
     }
     if (!ok) {
@@ -322,164 +659,221 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) conv_umma_kernel(const __grid
     }
   } else if (threadIdx.x == 32) {
     // ------------------------------------------------------------------ MMA issuer
-    int stage = 0;
-    uint32_t phase = 0;
-    int lt = 0;
+    TileIter ti;
+    ti.init(p, blockIdx.x, gridDim.x);
+    const uint32_t nstages = (uint32_t)p.stages, nbst = (uint32_t)p.b_stages;
+    const uint32_t afull0 = smem_u32(&a_full[0]), aempty0 = smem_u32(&a_empty[0]);
+    const uint32_t bfull0 = smem_u32(&b_full[0]), bempty0 = smem_u32(&b_empty[0]);
+    const uint32_t accf0 = smem_u32(&acc_full[0]), acce0 = smem_u32(&acc_empty[0]);
+    // low descriptor words: start address >> 4 (shared memory ends below 256 KiB, the 14-bit field never
+    // wraps) plus the leading-byte-offset field (bits 16-29), unused for swizzled K-major tiles and set to 1
+    const uint32_t lbo = 1u << 16;
+    const uint32_t a_lo0 = (((base + p.off_a) >> 4) & 0x3fffu) | lbo, bring_lo0 = (((base + p.off_bring) >> 4) & 0x3fffu) | lbo;
+    const uint32_t bres_lo0 = ((base >> 4) & 0x3fffu) | lbo;
+    const uint32_t stage16 = p.a_stage_bytes >> 4, asub16 = p.a_sub_bytes >> 4, bsub16 = p.b_sub_bytes >> 4, btile16 = p.b_tile_bytes >> 4;
+    const uint32_t hi = p.desc_hi;
+    const int ksteps = p.ksteps;
+    uint32_t stage = 0, phase = 0, a_lo = a_lo0;
+    uint32_t bs = 0, bphase = 0, bring_lo = bring_lo0;
+    uint32_t ab = 0, acc_par = 1;  // accumulator ring position and the parity to wait for on its empty barrier
     bool ok = true;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++lt) {
-      const int ab = lt & 1;
-      if (!mbar_wait(smem_u32(&acc_empty[ab]), ((uint32_t)(lt >> 1) & 1u) ^ 1u, abortp)) { ok = false; break; }
+    if (p.b_mode == kBResident) ok = mbar_wait(smem_u32(&bres_full), 0u, abortp);
+    for (; ti.tile < total_tiles && ok; ti.next(p)) {
+      if (!mbar_wait(acce0 + ab * 8u, acc_par, abortp)) { ok = false; break; }
       tcgen05_fence_after();
-      const uint32_t d_tmem = tmem_base + (uint32_t)(ab * BN);
-      for (int it = 0; it < p.k_iters; ++it) {
-        if (!mbar_wait(smem_u32(&full_bar[stage]), phase, abortp)) { ok = false; break; }
-        tcgen05_fence_after();
-        const uint32_t a_src = tiles_base + stage * STAGE_BYTES, b_src = a_src + A_BYTES;
-        const uint64_t a_desc = make_kmajor_desc<BK>(a_src), b_desc = make_kmajor_desc<BK>(b_src);
-#pragma unroll
-        for (int k = 0; k < BK / 32; ++k)  // 32 bytes of K per instruction: +2 in 16-byte address units
-          umma_i8(d_tmem, a_desc + 2 * k, b_desc + 2 * k, p.idesc, (it > 0 || k > 0) ? 1u : 0u);
-        umma_commit(smem_u32(&empty_bar[stage]));
-        if (++stage == stages) { stage = 0; phase ^= 1u; }
+      const uint32_t d_tmem = tmem_base + ab * (uint32_t)p.acc_stride;
+      uint32_t accum = 0;
+      // resident weights: tile (nt, cb, tap) sits at ((nt * c_blocks + cb) * taps + tap) * b_tile_bytes
+      const uint32_t bres_nt = bres_lo0 + (uint32_t)(ti.nt * p.c_blocks * p.taps) * btile16;
+      if (p.a_mode == kAHalo) {
+        uint32_t bres = bres_nt;  // (cb, tap) is exactly the order of the loops below
+        for (int cb = 0; cb < p.c_blocks && ok; ++cb) {
+          if (!mbar_wait(afull0 + stage * 8u, phase, abortp)) { ok = false; break; }
+          tcgen05_fence_after();
+          for (int tap = 0; tap < p.taps; ++tap) {
+            uint32_t b_lo = bres;
+            if (p.b_mode == kBRing) {
+              if (!mbar_wait(bfull0 + bs * 8u, bphase, abortp)) { ok = false; break; }
+              tcgen05_fence_after();
+              b_lo = bring_lo;
+            }
+            umma_i8_ksteps(ksteps, d_tmem, a_lo + tap_shift16[tap], hi, b_lo, hi, p.idesc, accum);
+            accum = 1;
+            if (p.b_mode == kBRing) {
+              umma_commit(bempty0 + bs * 8u);
+              bring_lo += bsub16;
+              if (++bs == nbst) { bs = 0; bphase ^= 1u; bring_lo = bring_lo0; }
+            } else {
+              bres += btile16;
+            }
+          }
+          umma_commit(aempty0 + stage * 8u);
+          a_lo += stage16;
+          if (++stage == nstages) { stage = 0; phase ^= 1u; a_lo = a_lo0; }
+        }
+      } else {
+        uint32_t bres_tap = bres_nt, bres = bres_nt;  // iterations run over taps with the channel blocks innermost
+        int cb = 0;
+        const uint32_t b_in_stage16 = (uint32_t)p.kb * asub16;
+        for (int it = 0; it < p.k_iters;) {
+          const int nsub = min(p.kb, p.k_iters - it);
+          if (!mbar_wait(afull0 + stage * 8u, phase, abortp)) { ok = false; break; }
+          tcgen05_fence_after();
+          uint32_t sa = a_lo, sb = a_lo + b_in_stage16;
+          for (int j = 0; j < nsub; ++j) {
+            umma_i8_ksteps(ksteps, d_tmem, sa, hi, p.b_mode == kBStage ? sb : bres, hi, p.idesc, accum);
+            accum = 1;
+            sa += asub16;
+            sb += bsub16;
+            bres += (uint32_t)p.taps * btile16;
+            if (++cb == p.c_blocks) { cb = 0; bres_tap += btile16; bres = bres_tap; }
+          }
+          umma_commit(aempty0 + stage * 8u);
+          it += nsub;
+          a_lo += stage16;
+          if (++stage == nstages) { stage = 0; phase ^= 1u; a_lo = a_lo0; }
+        }
       }
-      if (ok) umma_commit(smem_u32(&acc_full[ab]));
+      if (ok) umma_commit(accf0 + ab * 8u);
+      if (++ab == (uint32_t)p.nacc) { ab = 0; acc_par ^= 1u; }
     }
     if (!ok) {
       abort_flag = 1;
       atomicOr(p.status, kTimeoutMma);
     }
-  } else if (warp >= 2) {
-    // ------------------------------------------------------------------ epilogue (8 warps)
-    const int et = threadIdx.x - 64;
-    const int quad = warp & 3;         // TMEM lane quadrant this warp may read
-    const int half = (warp - 2) >> 2;  // which interleaved half of the 16-column chunks
-    const int row = quad * 32 + lane;
-    const bool leader = et == 0;
-    const bool out8 = p.y_type == Q8_U8 || p.y_type == Q8_S8;
-    unsigned char* const smem_tiles = smem_raw + (tiles_base - raw_base);  // generic pointer to tiles_base
-    int lt = 0;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++lt) {
-      const int m0 = (tile / p.n_tiles) * kBM, n0 = (tile % p.n_tiles) * BN;
-      const int ab = lt & 1;
-      const uint32_t par = (uint32_t)(lt >> 1) & 1u;
-      if (leader) {
-        bool ok = mbar_wait(smem_u32(&acc_full[ab]), par, abortp);
-        if (ok && p.res_mode == kResTma) ok = mbar_wait(smem_u32(&res_full[ab]), par, abortp);
-        if (!ok) {
+  } else if (threadIdx.x == 64) {
+    // ------------------------------------------------------------------ tile-buffer / residual producer
+    if (p.nbuf > 0) {
+      TileIter ti;
+      ti.init(p, blockIdx.x, gridDim.x);
+      const uint32_t bfull0 = smem_u32(&buf_full[0]), bempty0 = smem_u32(&buf_empty[0]);
+      const uint32_t nslots = (uint32_t)slots;
+      uint32_t slot = 0, par = 1;  // slots are used round robin over all groups: tile lt -> slot lt % (G*nbuf)
+      bool ok = true;
+      const int pw = 1 << p.pw_shift;
+      const uint32_t panel_bytes = (uint32_t)kBM << p.pw_shift;
+      for (; ti.tile < total_tiles; ti.next(p)) {
+        if (!mbar_wait(bempty0 + slot * 8u, par, abortp)) { ok = false; break; }
+        const uint32_t bar = bfull0 + slot * 8u;
+        if (p.res_mode == kResTma) {
+          uint32_t dst = base + p.off_bufs + slot * p.tile8_bytes;
+          mbar_arrive_expect_tx(bar, p.res_tx_bytes);
+          if (p.a_mode == kAHalo) {
+            for (int pn = 0, c = ti.nt * p.bn; pn < p.panels; ++pn, c += pw, dst += panel_bytes) tma_load_4d(dst, &tmRes, bar, c, ti.qt * p.tw, ti.pt * p.th, ti.img);
+          } else {
+            for (int pn = 0, c = ti.nt * p.bn; pn < p.panels; ++pn, c += pw, dst += panel_bytes) tma_load_2d(dst, &tmRes, bar, c, ti.mt * kBM);
+          }
+        } else {
+          mbar_arrive(bar);
+        }
+        if (++slot == nslots) { slot = 0; par ^= 1u; }
+      }
+      if (!ok) {
+        abort_flag = 1;
+        atomicOr(p.status, kTimeoutResidual);
+      }
+    }
+  } else if (threadIdx.x == 96) {
+    // ------------------------------------------------------------------ output store / buffer recycler
+    if (p.nbuf > 0) {
+      TileIter ti;
+      ti.init(p, blockIdx.x, gridDim.x);
+      const uint32_t bempty0 = smem_u32(&buf_empty[0]), ready0 = smem_u32(&store_ready[0]);
+      const uint32_t nslots = (uint32_t)slots;
+      uint32_t slot = 0, g = 0, gpar = 0;  // tile lt belongs to group lt % G, its j-th tile has parity j & 1
+      int prev_slot = -1;
+      bool ok = true;
+      const int pw = 1 << p.pw_shift;
+      const uint32_t panel_bytes = (uint32_t)kBM << p.pw_shift;
+      for (; ti.tile < total_tiles; ti.next(p)) {
+        if (!mbar_wait(ready0 + g * 8u, gpar, abortp)) { ok = false; break; }
+        if (p.out8) {
+          uint32_t src = base + p.off_bufs + slot * p.tile8_bytes;
+          if (p.a_mode == kAHalo) {
+            for (int pn = 0, c = p.c_off + ti.nt * p.bn; pn < p.panels; ++pn, c += pw, src += panel_bytes) tma_store_4d(&tmY, src, c, ti.qt * p.tw, ti.pt * p.th, ti.img);
+          } else {
+            for (int pn = 0, c = p.c_off + ti.nt * p.bn; pn < p.panels; ++pn, c += pw, src += panel_bytes) tma_store_2d(&tmY, src, c, ti.mt * kBM);
+          }
+          bulk_commit();
+          // the store before this one has read its buffer: hand that buffer back
+          bulk_wait_read<1>();
+          if (prev_slot >= 0) mbar_arrive(bempty0 + (uint32_t)prev_slot * 8u);
+          prev_slot = (int)slot;
+        } else {
+          mbar_arrive(bempty0 + slot * 8u);
+        }
+        if (++slot == nslots) slot = 0;
+        if (++g == (uint32_t)G) { g = 0; gpar ^= 1u; }
+      }
+      if (p.out8) {
+        bulk_wait_read<0>();  // the CTA's shared memory must outlive the reads of its last stores
+        if (prev_slot >= 0) mbar_arrive(bempty0 + (uint32_t)prev_slot * 8u);
+      }
+      if (!ok) {
+        abort_flag = 1;
+        atomicOr(p.status, kTimeoutStore);
+      }
+    }
+  } else if (warp >= 4) {
+    // ------------------------------------------------------------------ epilogue groups
+    const int g = (warp - 4) >> 2;
+    const int quad = warp & 3;  // TMEM lane quadrant this warp may read
+    const int row = quad * 32 + lane;  // accumulator row of this thread
+    EpiTile t;
+    t.s_bias = s_bias;
+    t.s_scale = s_scale;
+    // halo tiles: accumulator row -> pixel (pp, qq) of the patch grid; rows right of the tile are dropped
+    int pp = 0, qq = 0;
+    t.srow = row;
+    t.smem_ok = true;
+    if (p.a_mode == kAHalo) {
+      pp = row / p.twb;
+      qq = row - pp * p.twb;
+      t.smem_ok = pp < p.th && qq < p.tw;
+      t.srow = t.smem_ok ? pp * p.tw + qq : 0;
+    }
+    // this group's tiles are lt = g, g + G, ... of the CTA's sequence; ring positions advance by additions
+    const uint32_t accf0 = smem_u32(&acc_full[0]), acce0 = smem_u32(&acc_empty[0]);
+    const uint32_t bfull0 = smem_u32(&buf_full[0]), ready = smem_u32(&store_ready[g]);
+    const uint32_t nslots = (uint32_t)slots, nacc = (uint32_t)p.nacc;
+    uint32_t ab = (uint32_t)g % nacc, acc_par = ((uint32_t)g / nacc) & 1u;
+    uint32_t slot = (uint32_t)g, slot_par = 0;
+    TileIter ti;
+    ti.init(p, blockIdx.x + g * (int)gridDim.x, G * (int)gridDim.x);
+    for (; ti.tile < total_tiles; ti.next(p)) {
+      bool ok = mbar_wait(accf0 + ab * 8u, acc_par, abortp);
+      if (p.nbuf > 0 && ok) ok = mbar_wait(bfull0 + slot * 8u, slot_par, abortp);
+      ok = __all_sync(0xffffffffu, ok ? 1 : 0) != 0;
+      if (!ok) {
+        if (lane == 0) {
           abort_flag = 1;
           atomicOr(p.status, kTimeoutEpilogue);
         }
-        if (p.y_tma) bulk_wait_read<1>();  // the store that last used this staging tile has read it
-        epi_ok = ok ? 1 : 0;
+        break;
       }
-      for (int j = et; j < BN; j += kEpiThreads) {
-        const int n = n0 + j;
-        s_bias[j] = (p.bias && n < p.K) ? p.bias[n] : 0;
-        s_scale[j] = p.scale ? (p.scale_count == 1 ? p.scale[0] : (n < p.K ? p.scale[n] : 0.f)) : 0.f;
-      }
-      epi_bar_sync();
-      if (!epi_ok) break;
       tcgen05_fence_after();
-
-      const long long m = (long long)m0 + row;
-      const bool row_ok = m < p.M;
-      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(ab * BN);
-      unsigned char* const stage_out = smem_tiles + (out_base - tiles_base) + ab * TILE8_BYTES;
-      const unsigned char* const stage_res = smem_tiles + (res_base - tiles_base) + ab * TILE8_BYTES;
-      const bool has_res = p.res_mode != kResNone;
-#pragma unroll 1
-      for (int ch = half; ch < NCHUNK; ch += 2) {
-        int acc[16];
-        __syncwarp();
-        tmem_ld_16(taddr + ch * 16, acc);
-        tmem_ld_wait();
-        const int nb = n0 + ch * 16;
-        // 16-byte chunk (row, ch) of an 8-bit tile: panel, byte offset inside it, swizzled
-        const int pn = (ch * 16) / PW;
-        uint32_t off = (uint32_t)row * PW + (uint32_t)((ch * 16) % PW);
-        off ^= ((off >> 7) & PMASK) << 4;
-        off += pn * (kBM * PW);
-#pragma unroll
-        for (int j = 0; j < 16; ++j) acc[j] += s_bias[ch * 16 + j];
-
-        if (p.y_type == Q8_S32) {
-          if (row_ok && nb < p.K) {
-            const int valid = min(16, p.K - nb);
-            int* yp = static_cast<int*>(p.y) + (size_t)m * p.ldc + p.c_off + nb;
-            if (p.y_vec && valid == 16) {
-#pragma unroll
-              for (int j = 0; j < 4; ++j) reinterpret_cast<int4*>(yp)[j] = make_int4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
-            } else {
-#pragma unroll
-              for (int j = 0; j < 16; ++j)
-                if (j < valid) yp[j] = acc[j];
-            }
-          }
-          continue;
-        }
-        unsigned int rw[4] = {0u, 0u, 0u, 0u};
-        if (p.res_mode == kResTma) {
-          const uint4 rv = *reinterpret_cast<const uint4*>(stage_res + off);
-          rw[0] = rv.x; rw[1] = rv.y; rw[2] = rv.z; rw[3] = rv.w;
-        } else if (p.res_mode == kResGlobal) {
-          if (row_ok && nb < p.K) {
-            const int valid = min(16, p.K - nb);
-            const unsigned char* rp = p.res + (size_t)m * p.K + nb;
-#pragma unroll
-            for (int j = 0; j < 16; ++j)
-              if (j < valid) rw[j >> 2] |= (unsigned int)rp[j] << (8 * (j & 3));
-          }
-        }
-        float v[16];
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const unsigned int b = (rw[j >> 2] >> (8 * (j & 3))) & 0xffu;
-          const int rz = p.res_signed ? (int)(signed char)b : (int)b;
-          v[j] = requant_value(acc[j], s_scale[ch * 16 + j], has_res, rz, p.res_scale, p.relu != 0);
-        }
-        if (p.y_type == Q8_F32) {
-          if (row_ok && nb < p.K) {
-            const int valid = min(16, p.K - nb);
-            float* yp = static_cast<float*>(p.y) + (size_t)m * p.ldc + p.c_off + nb;
-            if (p.y_vec && valid == 16) {
-#pragma unroll
-              for (int j = 0; j < 4; ++j) reinterpret_cast<float4*>(yp)[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-            } else {
-#pragma unroll
-              for (int j = 0; j < 16; ++j)
-                if (j < valid) yp[j] = v[j];
-            }
-          }
-          continue;
-        }
-        int z[16];
-        if (p.y_type == Q8_U8) {
-#pragma unroll
-          for (int j = 0; j < 16; ++j) z[j] = round_clamp_u8(v[j]);
-        } else {
-#pragma unroll
-          for (int j = 0; j < 16; ++j) z[j] = round_clamp_s8(v[j]);
-        }
-        *reinterpret_cast<uint4*>(stage_out + off) =
-            make_uint4(pack4(z[0], z[1], z[2], z[3]), pack4(z[4], z[5], z[6], z[7]), pack4(z[8], z[9], z[10], z[11]),
-                       pack4(z[12], z[13], z[14], z[15]));
+      t.n0 = ti.nt * p.bn;
+      if (p.a_mode == kAHalo) {
+        const int pr = ti.pt * p.th + pp, qc = ti.qt * p.tw + qq;
+        t.row_ok = t.smem_ok && pr < p.P && qc < p.Q;
+        t.m = ((long long)ti.img * p.P + pr) * p.Q + qc;
+      } else {
+        t.m = (long long)ti.mt * kBM + row;
+        t.row_ok = t.m < p.M;
       }
-      // after this barrier every TMEM read, residual read and staging write of the tile is done
-      tcgen05_fence_before();
-      if (out8) fence_proxy_async_smem();
-      epi_bar_sync();
-      if (leader) {
-        mbar_arrive(smem_u32(&acc_empty[ab]));
-        if (p.res_mode == kResTma) mbar_arrive(smem_u32(&res_empty[ab]));
-        if (p.y_tma) {
-#pragma unroll
-          for (int pn = 0; pn < PANELS; ++pn)
-            tma_store_2d(&tmY, out_base + ab * TILE8_BYTES + pn * (kBM * PW), p.c_off + n0 + pn * PW, m0);
-          bulk_commit();
-        }
+      t.buf = p.nbuf > 0 ? base_ptr + p.off_bufs + (size_t)slot * p.tile8_bytes : nullptr;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + ab * (uint32_t)p.acc_stride;
+      epilogue_row<kOut, kRes>(p, t, taddr, acce0 + ab * 8u, lane);
+      if (p.nbuf > 0) {
+        // this thread's reads and writes of the buffer are done; the store thread takes over
+        if (p.out8) fence_proxy_async_smem();
+        mbar_arrive(ready);
       }
+      ab += (uint32_t)G;
+      while (ab >= nacc) { ab -= nacc; acc_par ^= 1u; }
+      slot += (uint32_t)G;
+      if (slot >= nslots) { slot -= nslots; slot_par ^= 1u; }
     }
-    if (leader && p.y_tma) bulk_wait_all();
   }
 
   tcgen05_fence_before();
@@ -487,7 +881,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) conv_umma_kernel(const __grid
   if (warp == 1) {
     __syncwarp();
     tcgen05_fence_after();
-    tmem_dealloc(tmem_base, TMEM_COLS);
+    tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
   }
 }
 
@@ -541,28 +935,22 @@ int pick_bk(int C) {
   return best;
 }
 
-int pick_bn(int K) {
-  if (K <= 16) return 16;
-  if (K <= 32) return 32;
-  if (K <= 64) return 64;
-  if (K <= 128) return 128;
-  // wider tiles re-read A less often; take 256 unless it pads Cout by more than 128 would
-  int pad128 = ((K + 127) / 128) * 128, pad256 = ((K + 255) / 256) * 256;
-  return pad256 <= pad128 ? 256 : 128;
-}
-
-constexpr int max_stages_for(int bn, int bk) {
-  int n = 200 * 1024 / ((kBM + bn) * bk);
-  return n < 2 ? 2 : (n > 12 ? 12 : n);
-}
-
-// Dynamic shared memory besides the A/B stages: alignment slack and the epilogue tiles.
-int fixed_smem_bytes(int bn, bool y_tma, bool res_tma) {
-  return 2048 + (y_tma ? 2 * kBM * bn : 0) + (res_tma ? 2 * kBM * bn : 0);
-}
-
-int stages_that_fit(int bn, int bk, bool y_tma, bool res_tma) {
-  return (kSmemLimit - kStaticSmemReserve - fixed_smem_bytes(bn, y_tma, res_tma)) / ((kBM + bn) * bk);
+// Tile width: the multiple of 16 (power-of-two panels keep the 8-bit tile layout simple) that pads
+// Cout least; short reductions are bandwidth bound and take narrower tiles, which leaves room for
+// four TMEM accumulators and more tile buffers.
+int pick_bn(int K, int kgemm) {
+  static const int widths[] = {16, 32, 48, 64, 96, 128, 192, 256};
+  const int cap = kgemm <= 640 ? 128 : 256;
+  int best = 16;
+  long long best_cost = -1;
+  for (int w : widths) {
+    if (w > cap) break;
+    const long long padded = (long long)((K + w - 1) / w) * w;
+    // padded columns are wasted MMA and epilogue work; every extra tile re-reads A once more
+    const long long cost = padded * 8 + (padded / w) * 24;
+    if (best_cost < 0 || cost <= best_cost) { best = w; best_cost = cost; }
+  }
+  return best;
 }
 
 CUtensorMapSwizzle swizzle_for_bytes(int row_bytes) {
@@ -571,19 +959,50 @@ CUtensorMapSwizzle swizzle_for_bytes(int row_bytes) {
                                              : (row_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE));
 }
 
-template <int BN, int BK>
-int launch_tile(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmRes, const CUtensorMap& tmY,
-                UmmaParams& p, cudaStream_t stream) {
-  constexpr int MAXS = max_stages_for(BN, BK);
-  constexpr int STAGE_BYTES = (kBM + BN) * BK;
-  auto kernel = conv_umma_kernel<BN, BK, MAXS>;
-  int stages = stages_that_fit(BN, BK, p.y_tma != 0, p.res_mode == kResTma);
-  if (stages > MAXS) stages = MAXS;
-  if (stages < 2) return fail(Q8_ERR_UNSUPPORTED, "conv_umma: tile does not fit in shared memory");
-  p.stages = stages;
-  // at least 120 KiB so that one CTA owns an SM and with it the whole TMEM
-  size_t dyn = (size_t)fixed_smem_bytes(BN, p.y_tma != 0, p.res_mode == kResTma) + (size_t)stages * STAGE_BYTES;
-  if (dyn < 120 * 1024) dyn = 120 * 1024;
+unsigned int round_up(unsigned int v, unsigned int a) { return (v + a - 1) / a * a; }
+
+int tune_env(const char* name, int dflt) {
+  const char* v = getenv(name);
+  return v && *v ? atoi(v) : dflt;
+}
+
+// Halo tiling of a stride-1 filter: TH x TW output pixels per tile, (TH + ext_h) x (TW + ext_w)
+// input pixels per patch, TH * (TW + ext_w) <= 128 accumulator rows.  Picks the extents that waste
+// the fewest accumulator rows, preferring less halo among near-equals.
+struct HaloTile {
+  int tw, th, twb, hb;
+  double eff;  // useful output pixels per computed accumulator row
+};
+
+bool choose_halo_tile(const q8_conv_desc& d, int P, int Q, HaloTile* out) {
+  if (d.stride_h != 1 || d.stride_w != 1) return false;
+  const int taps = d.R * d.S;
+  if (taps < 2 || taps > kMaxTaps) return false;
+  const int ext_w = (d.S - 1) * d.dil_w, ext_h = (d.R - 1) * d.dil_h;
+  HaloTile best = {0, 0, 0, 0, 0.0};
+  double best_score = 0.0;
+  for (int tw = 1; tw <= Q && tw + ext_w <= kBM; ++tw) {
+    const int twb = tw + ext_w;
+    int th = kBM / twb;
+    if (th > P) th = P;
+    if (th < 1) continue;
+    const int hb = th + ext_h;
+    if (hb > 256 || twb > 256) continue;
+    const long long tiles = (long long)((Q + tw - 1) / tw) * ((P + th - 1) / th);
+    const double eff = (double)P * Q / ((double)tiles * kBM);
+    const double halo = (double)hb * twb / ((double)th * tw);
+    const double score = eff / (1.0 + 0.04 * halo);
+    if (score > best_score) { best_score = score; best = {tw, th, twb, hb, eff}; }
+  }
+  if (best.eff < 0.5) return false;
+  *out = best;
+  return true;
+}
+
+template <int G, int kOut, int kRes>
+int launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmRes, const CUtensorMap& tmY,
+                   const UmmaParams& p, size_t dyn, int grid, cudaStream_t stream) {
+  auto kernel = conv_umma_kernel<G, kOut, kRes>;
   static bool configured = false;  // per instantiation
   if (!configured) {
     int rc = check_cuda(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit - kStaticSmemReserve),
@@ -591,22 +1010,31 @@ int launch_tile(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMa
     if (rc != Q8_OK) return rc;
     configured = true;
   }
-  p.m_tiles = (p.M + kBM - 1) / kBM;
-  p.n_tiles = (p.K + BN - 1) / BN;
-  const long long tiles = (long long)p.m_tiles * p.n_tiles;
-  const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
-  kernel<<<grid, kUmmaThreads, dyn, stream>>>(tmA, tmB, tmRes, tmY, p);
+  kernel<<<grid, kCtrlThreads + G * kGroupThreads, dyn, stream>>>(tmA, tmB, tmRes, tmY, p);
   return check_launch("conv_umma_kernel");
 }
 
-template <int BN>
-int launch_bk(int bk, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmRes, const CUtensorMap& tmY,
-              UmmaParams& p, cudaStream_t stream) {
-  switch (bk) {
-    case 128: return launch_tile<BN, 128>(tmA, tmB, tmRes, tmY, p, stream);
-    case 64: return launch_tile<BN, 64>(tmA, tmB, tmRes, tmY, p, stream);
-    default: return launch_tile<BN, 32>(tmA, tmB, tmRes, tmY, p, stream);
+template <int G>
+int launch_groups(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmRes, const CUtensorMap& tmY,
+                  const UmmaParams& p, size_t dyn, int grid, cudaStream_t stream) {
+#define Q8_LAUNCH(OUT, RES) return launch_variant<G, OUT, RES>(tmA, tmB, tmRes, tmY, p, dyn, grid, stream)
+  switch (p.y_type * 3 + p.res_mode) {
+    case Q8_U8 * 3 + kResNone: Q8_LAUNCH(Q8_U8, kResNone);
+    case Q8_U8 * 3 + kResTma: Q8_LAUNCH(Q8_U8, kResTma);
+    case Q8_U8 * 3 + kResGlobal: Q8_LAUNCH(Q8_U8, kResGlobal);
+    case Q8_S8 * 3 + kResNone: Q8_LAUNCH(Q8_S8, kResNone);
+    case Q8_S8 * 3 + kResTma: Q8_LAUNCH(Q8_S8, kResTma);
+    case Q8_S8 * 3 + kResGlobal: Q8_LAUNCH(Q8_S8, kResGlobal);
+    case Q8_F32 * 3 + kResNone: Q8_LAUNCH(Q8_F32, kResNone);
+    case Q8_F32 * 3 + kResTma: Q8_LAUNCH(Q8_F32, kResTma);
+    case Q8_F32 * 3 + kResGlobal: Q8_LAUNCH(Q8_F32, kResGlobal);
+    default: Q8_LAUNCH(Q8_S32, kResNone);
   }
+#undef Q8_LAUNCH
+}
+
+bool is_plain(const q8_conv_desc& d) {
+  return d.R == 1 && d.S == 1 && d.stride_h == 1 && d.stride_w == 1 && d.pad_h == 0 && d.pad_w == 0;
 }
 
 }  // namespace
@@ -615,15 +1043,17 @@ bool umma_shape_eligible(const q8_conv_desc& d, const char** why) {
   const char* dummy;
   if (!why) why = &dummy;
   if (d.C % 16) { *why = "C is not a multiple of 16"; return false; }
-  const bool plain = d.R == 1 && d.S == 1 && d.stride_h == 1 && d.stride_w == 1 && d.pad_h == 0 && d.pad_w == 0;
-  if (!plain) {
-    // im2col tensor maps: corners are 8-bit signed, tap offsets 8-bit unsigned, strides at most 8
-    const int up_w = d.pad_w - (d.S - 1) * d.dil_w, up_h = d.pad_h - (d.R - 1) * d.dil_h;
-    if (d.pad_w > 128 || d.pad_h > 128 || up_w < -128 || up_h < -128 || up_w > 127 || up_h > 127) { *why = "padding/dilation outside the im2col corner range"; return false; }
-    if ((d.S - 1) * d.dil_w > 255 || (d.R - 1) * d.dil_h > 255) { *why = "filter extent outside the im2col offset range"; return false; }
-    if (d.stride_h > 8 || d.stride_w > 8) { *why = "stride > 8"; return false; }
-    if ((long long)d.N * d.H * d.W * d.C < 131072) { *why = "activation tensor smaller than 128 KiB"; return false; }
-  }
+  if (d.K > 4096) { *why = "more than 4096 output channels"; return false; }
+  if (is_plain(d)) return true;
+  HaloTile ht;
+  const int P = conv_out_extent(d.H, d.pad_h, d.dil_h, d.R, d.stride_h), Q = conv_out_extent(d.W, d.pad_w, d.dil_w, d.S, d.stride_w);
+  if (choose_halo_tile(d, P, Q, &ht)) return true;
+  // im2col tensor maps: corners are 8-bit signed, tap offsets 8-bit unsigned, strides at most 8
+  const int up_w = d.pad_w - (d.S - 1) * d.dil_w, up_h = d.pad_h - (d.R - 1) * d.dil_h;
+  if (d.pad_w > 128 || d.pad_h > 128 || up_w < -128 || up_h < -128 || up_w > 127 || up_h > 127) { *why = "padding/dilation outside the im2col corner range"; return false; }
+  if ((d.S - 1) * d.dil_w > 255 || (d.R - 1) * d.dil_h > 255) { *why = "filter extent outside the im2col offset range"; return false; }
+  if (d.stride_h > 8 || d.stride_w > 8) { *why = "stride > 8"; return false; }
+  if ((long long)d.N * d.H * d.W * d.C < 131072) { *why = "activation tensor smaller than 128 KiB"; return false; }
   return true;
 }
 
@@ -634,99 +1064,206 @@ int launch_conv_umma(const ConvArgs& a) {
   unsigned int* status = status_word_device_ptr();
   if (!status) return fail(Q8_ERR_CUDA, "conv_umma: status word not available");
 
-  const bool plain = d.R == 1 && d.S == 1 && d.stride_h == 1 && d.stride_w == 1 && d.pad_h == 0 && d.pad_w == 0;
   const bool out8 = d.y_type == Q8_U8 || d.y_type == Q8_S8;
   int res_mode = kResNone;
   if (a.residual) res_mode = (d.K % 16 == 0 && aligned16(a.residual)) ? kResTma : kResGlobal;
   const int BK = pick_bk(d.C);
-  int BN = pick_bn(d.K);
-  // the widest tile leaves too little room for A/B stages next to its epilogue tiles: narrow it
-  if (BN == 256 && stages_that_fit(BN, BK, out8, res_mode == kResTma) < 3) BN = 128;
+  const int BN = tune_env("Q8_BN", pick_bn(d.K, d.R * d.S * d.C));
   const CUtensorMapSwizzle swz = swizzle_for_bytes(BK);
-  const int PW = panel_bytes_for(BN);
 
+  UmmaParams p;
+  memset(&p, 0, sizeof(p));
+  HaloTile ht = {0, 0, 0, 0, 0.0};
+  p.a_mode = is_plain(d) ? kAPlain : ((tune_env("Q8_HALO", 1) && choose_halo_tile(d, a.P, a.Q, &ht)) ? kAHalo : kAIm2col);
+  p.bn = BN; p.bk = BK; p.ksteps = BK / 32;
+  p.P = a.P; p.Q = a.Q; p.PQ = a.P * a.Q; p.M = (int)a.M; p.K = d.K;
+  p.stride_h = d.stride_h; p.stride_w = d.stride_w; p.pad_h = d.pad_h; p.pad_w = d.pad_w; p.dil_h = d.dil_h; p.dil_w = d.dil_w;
+  p.R = d.R; p.S = d.S; p.taps = d.R * d.S;
+  p.c_blocks = (d.C + BK - 1) / BK;
+  p.C_pad = p.c_blocks * BK;
+  p.k_iters = p.taps * p.c_blocks;
+  // 8-bit tile buffers: panels as wide as the largest power of two dividing BN, at most one swizzle span
+  int pw = BN & -BN;
+  if (pw > 128) pw = 128;
+  p.pw_shift = 0;
+  while ((1 << p.pw_shift) < pw) ++p.pw_shift;
+  p.pmask = pw == 128 ? 7 : (pw == 64 ? 3 : (pw == 32 ? 1 : 0));
+  p.panels = BN / pw;
+  p.n_tiles = (d.K + BN - 1) / BN;
+  p.k_pad = p.n_tiles * BN;
+  if (p.a_mode == kAHalo) {
+    p.tw = ht.tw; p.th = ht.th; p.twb = ht.twb; p.hb = ht.hb;
+    p.q_tiles = (a.Q + ht.tw - 1) / ht.tw;
+    p.p_tiles = (a.P + ht.th - 1) / ht.th;
+    p.m_tiles = d.N * p.p_tiles * p.q_tiles;
+  } else {
+    p.m_tiles = (int)((a.M + kBM - 1) / kBM);
+  }
+  p.tile8_bytes = (unsigned)(kBM * BN);  // a multiple of 2 KiB
+  p.acc_stride = 32;
+  while (p.acc_stride < BN) p.acc_stride *= 2;
+  p.nacc = 512 / p.acc_stride < kMaxAcc ? 512 / p.acc_stride : kMaxAcc;
+  p.tmem_cols = p.nacc * p.acc_stride;  // a power of two in [32, 512]
+  p.b_tile_bytes = (unsigned)(BN * BK);
+  p.b_sub_bytes = round_up(p.b_tile_bytes, 1024u);
+
+  // ---- shared memory plan: [resident weights] [A stages] [weight ring] [8-bit tile buffers] [bias, scale]
+  const bool use_bufs = out8 || res_mode == kResTma;
+  int G = tune_env("Q8_G", BN > 128 ? 2 : 4);
+  if (G > p.nacc) G = 2;  // a group may run at most one accumulator phase ahead of the MMA warp
+  const unsigned chan_bytes = round_up((unsigned)p.k_pad * 8u, 1024u);
+  const unsigned budget = (unsigned)(kSmemLimit - kStaticSmemReserve) - 1024u /* alignment slack */ - chan_bytes;
+  // Weights stay resident when the whole layer's B operand is small: no per-tile weight traffic at all.
+  // A tile of bn*bk bytes keeps every tap tile aligned to the swizzle pattern.
+  const unsigned b_all = (unsigned)(p.n_tiles * p.c_blocks * p.taps) * p.b_tile_bytes;
+  const bool resident = tune_env("Q8_BRES", (b_all <= 80u * 1024u && p.taps <= 256 && p.b_tile_bytes % (8u * BK) == 0) ? 1 : 0) != 0;
+  p.b_mode = resident ? kBResident : (p.a_mode == kAHalo ? kBRing : kBStage);
+  const unsigned bres_bytes = resident ? round_up(b_all, 1024u) : 0u;
+  unsigned min_pipe;
+  if (p.a_mode == kAHalo) {
+    // the taps read up to (ext_h * twb + ext_w) pixels beyond accumulator row 127
+    const unsigned reach = (unsigned)(kBM + (d.R - 1) * d.dil_h * ht.twb + (d.S - 1) * d.dil_w) * BK;
+    p.a_sub_bytes = (unsigned)(BK * ht.twb * ht.hb);
+    p.a_stage_bytes = round_up(reach > p.a_sub_bytes ? reach : p.a_sub_bytes, 1024u);
+    p.kb = 1;
+    min_pipe = 2u * p.a_stage_bytes + (p.b_mode == kBRing ? 3u * p.b_sub_bytes : 0u);
+  } else {
+    p.a_sub_bytes = (unsigned)(kBM * BK);
+    const unsigned unit = p.a_sub_bytes + (p.b_mode == kBStage ? p.b_sub_bytes : 0u);
+    int kb = (int)(40u * 1024u / unit);
+    if (kb < 1) kb = 1;
+    if (kb > p.k_iters) kb = p.k_iters;
+    p.kb = tune_env("Q8_KB", kb);
+    p.a_stage_bytes = (unsigned)p.kb * unit;
+    min_pipe = 2u * p.a_stage_bytes;
+  }
+  p.nbuf = 0;
+  if (use_bufs) {
+    // two buffers per group when that still leaves a comfortable pipeline
+    p.nbuf = (budget >= bres_bytes + 2u * G * p.tile8_bytes + 2u * min_pipe && 2 * G <= kMaxSlots) ? 2 : 1;
+    p.nbuf = tune_env("Q8_NBUF", p.nbuf);
+  }
+  const unsigned buf_bytes = (unsigned)(G * p.nbuf) * p.tile8_bytes;
+  if (budget < bres_bytes + buf_bytes + min_pipe) return fail(Q8_ERR_UNSUPPORTED, "conv_umma: tile does not fit in shared memory");
+  unsigned rest = budget - bres_bytes - buf_bytes;
+  p.b_stages = 0;
+  if (p.b_mode == kBRing) {
+    int bst = (int)((rest - 2u * p.a_stage_bytes) / p.b_sub_bytes);
+    if (bst > kMaxBStages) bst = kMaxBStages;
+    p.b_stages = tune_env("Q8_BSTAGES", bst);
+    rest -= (unsigned)p.b_stages * p.b_sub_bytes;
+  }
+  int stages = (int)(rest / p.a_stage_bytes);
+  if (stages > kMaxStages) stages = kMaxStages;
+  p.stages = tune_env("Q8_STAGES", stages);
+  p.off_a = bres_bytes;
+  p.off_bring = p.off_a + (unsigned)p.stages * p.a_stage_bytes;
+  p.off_bufs = p.off_bring + (unsigned)p.b_stages * p.b_sub_bytes;
+  p.off_chan = p.off_bufs + buf_bytes;
+  size_t dyn = 1024u + p.off_chan + chan_bytes;
+  if (dyn > (size_t)(kSmemLimit - kStaticSmemReserve)) return fail(Q8_ERR_UNSUPPORTED, "conv_umma: shared memory plan exceeds the limit");
+  // at least 120 KiB so that one CTA owns an SM and with it the whole TMEM
+  if (dyn < 120 * 1024) dyn = 120 * 1024;
+
+  // ---- tensor maps
   CUtensorMap tmA, tmB, tmRes, tmY;
   memset(&tmRes, 0, sizeof(tmRes));
   memset(&tmY, 0, sizeof(tmY));
   CUresult cr;
-  if (plain) {
+  const cuuint32_t ones[4] = {1, 1, 1, 1};
+  if (p.a_mode == kAPlain) {
     cuuint64_t dims[2] = {(cuuint64_t)d.C, (cuuint64_t)a.M};
     cuuint64_t strides[1] = {(cuuint64_t)d.C};
     cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)kBM};
-    cuuint32_t estr[2] = {1, 1};
-    cr = fn.tiled(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(a.x), dims, strides, box, estr,
+    cr = fn.tiled(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(a.x), dims, strides, box, ones,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   } else {
     cuuint64_t dims[4] = {(cuuint64_t)d.C, (cuuint64_t)d.W, (cuuint64_t)d.H, (cuuint64_t)d.N};
     cuuint64_t strides[3] = {(cuuint64_t)d.C, (cuuint64_t)d.W * d.C, (cuuint64_t)d.H * d.W * d.C};
-    int lower[2] = {-d.pad_w, -d.pad_h};
-    int upper[2] = {d.pad_w - (d.S - 1) * d.dil_w, d.pad_h - (d.R - 1) * d.dil_h};
-    cuuint32_t estr[4] = {1, (cuuint32_t)d.stride_w, (cuuint32_t)d.stride_h, 1};
-    cr = fn.im2col(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(a.x), dims, strides, lower, upper,
-                   (cuuint32_t)BK, (cuuint32_t)kBM, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
-                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (p.a_mode == kAHalo) {
+      cuuint32_t box[4] = {(cuuint32_t)BK, (cuuint32_t)ht.twb, (cuuint32_t)ht.hb, 1};
+      cr = fn.tiled(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(a.x), dims, strides, box, ones,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    } else {
+      int lower[2] = {-d.pad_w, -d.pad_h};
+      int upper[2] = {d.pad_w - (d.S - 1) * d.dil_w, d.pad_h - (d.R - 1) * d.dil_h};
+      cuuint32_t estr[4] = {1, (cuuint32_t)d.stride_w, (cuuint32_t)d.stride_h, 1};
+      cr = fn.im2col(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(a.x), dims, strides, lower, upper,
+                     (cuuint32_t)BK, (cuuint32_t)kBM, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    }
   }
   if (cr != CUDA_SUCCESS) return fail(Q8_ERR_CUDA, "conv_umma: activation tensor map rejected (CUresult %d)", (int)cr);
-  {
-    cuuint64_t dims[3] = {(cuuint64_t)d.C, (cuuint64_t)d.R * d.S, (cuuint64_t)d.K};
-    cuuint64_t strides[2] = {(cuuint64_t)d.C, (cuuint64_t)d.R * d.S * d.C};
+  if (resident) {
+    // (C, K, taps) view of the KRSC weights: one box brings bn rows of every tap
+    cuuint64_t dims[3] = {(cuuint64_t)d.C, (cuuint64_t)d.K, (cuuint64_t)p.taps};
+    cuuint64_t strides[2] = {(cuuint64_t)p.taps * d.C, (cuuint64_t)d.C};
+    cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)BN, (cuuint32_t)p.taps};
+    cr = fn.tiled(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(a.w), dims, strides, box, ones,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else {
+    cuuint64_t dims[3] = {(cuuint64_t)d.C, (cuuint64_t)p.taps, (cuuint64_t)d.K};
+    cuuint64_t strides[2] = {(cuuint64_t)d.C, (cuuint64_t)p.taps * d.C};
     cuuint32_t box[3] = {(cuuint32_t)BK, 1, (cuuint32_t)BN};
-    cuuint32_t estr[3] = {1, 1, 1};
-    cr = fn.tiled(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(a.w), dims, strides, box, estr,
+    cr = fn.tiled(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(a.w), dims, strides, box, ones,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   }
   if (cr != CUDA_SUCCESS) return fail(Q8_ERR_CUDA, "conv_umma: weight tensor map rejected (CUresult %d)", (int)cr);
 
+  // Residual and output tiles: [M][channels] matrices, or for halo tiles (channels, Q, P, N) tensors whose
+  // TH x TW box lands as TH*TW dense rows.  The output map ends at the last channel this layer owns,
+  // so the store clips ragged Cout tiles and never touches a neighbouring slice of a concatenated tensor.
+  auto encode_rows = [&](CUtensorMap* tm, void* ptr, int channels, int ld, CUtensorMapL2promotion promo) -> CUresult {
+    if (p.a_mode == kAHalo) {
+      cuuint64_t dims[4] = {(cuuint64_t)channels, (cuuint64_t)a.Q, (cuuint64_t)a.P, (cuuint64_t)d.N};
+      cuuint64_t strides[3] = {(cuuint64_t)ld, (cuuint64_t)a.Q * ld, (cuuint64_t)a.P * a.Q * ld};
+      cuuint32_t box[4] = {(cuuint32_t)pw, (cuuint32_t)ht.tw, (cuuint32_t)ht.th, 1};
+      return fn.tiled(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, ptr, dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                      swizzle_for_bytes(pw), promo, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    }
+    cuuint64_t dims[2] = {(cuuint64_t)channels, (cuuint64_t)a.M};
+    cuuint64_t strides[1] = {(cuuint64_t)ld};
+    cuuint32_t box[2] = {(cuuint32_t)pw, (cuuint32_t)kBM};
+    return fn.tiled(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, ptr, dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    swizzle_for_bytes(pw), promo, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  };
   if (res_mode == kResTma) {
-    cuuint64_t dims[2] = {(cuuint64_t)d.K, (cuuint64_t)a.M};
-    cuuint64_t strides[1] = {(cuuint64_t)d.K};
-    cuuint32_t box[2] = {(cuuint32_t)PW, (cuuint32_t)kBM};
-    cuuint32_t estr[2] = {1, 1};
-    cr = fn.tiled(&tmRes, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(a.residual), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for_bytes(PW), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    cr = encode_rows(&tmRes, const_cast<void*>(a.residual), d.K, d.K, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
     if (cr != CUDA_SUCCESS) return fail(Q8_ERR_CUDA, "conv_umma: residual tensor map rejected (CUresult %d)", (int)cr);
   }
   if (out8) {
-    // the map ends at the last channel this layer owns, so the store clips ragged Cout tiles and
-    // never touches a neighbouring slice of a concatenated tensor
-    cuuint64_t dims[2] = {(cuuint64_t)(a.c_off + d.K), (cuuint64_t)a.M};
-    cuuint64_t strides[1] = {(cuuint64_t)a.ldc};
-    cuuint32_t box[2] = {(cuuint32_t)PW, (cuuint32_t)kBM};
-    cuuint32_t estr[2] = {1, 1};
-    cr = fn.tiled(&tmY, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, a.y, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                  swizzle_for_bytes(PW), CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    cr = encode_rows(&tmY, a.y, a.c_off + d.K, a.ldc, CU_TENSOR_MAP_L2_PROMOTION_NONE);
     if (cr != CUDA_SUCCESS) return fail(Q8_ERR_CUDA, "conv_umma: output tensor map rejected (CUresult %d)", (int)cr);
   }
+  p.res_tx_bytes = (unsigned)BN * (p.a_mode == kAHalo ? (unsigned)(ht.tw * ht.th) : (unsigned)kBM);
 
-  UmmaParams p;
-  p.M = (int)a.M; p.K = d.K; p.PQ = a.P * a.Q; p.Q = a.Q;
-  p.stride_h = d.stride_h; p.stride_w = d.stride_w; p.pad_h = d.pad_h; p.pad_w = d.pad_w; p.dil_h = d.dil_h; p.dil_w = d.dil_w;
-  p.S = d.S;
-  p.c_blocks = (d.C + BK - 1) / BK;
-  p.k_iters = d.R * d.S * p.c_blocks;
-  p.stages = 0; p.m_tiles = 0; p.n_tiles = 0;
-  p.a_im2col = plain ? 0 : 1;
   // instruction descriptor: D = s32 (2 << 4); A format at bit 7 (0 = u8, 1 = s8); B = s8 at bit 10;
   // both operands K-major; N/8 at bit 17; M/16 at bit 24.
   p.idesc = (2u << 4) | ((d.x_type == Q8_S8 ? 1u : 0u) << 7) | (1u << 10) | ((unsigned)(BN >> 3) << 17) | ((unsigned)(kBM >> 4) << 24);
+  // shared-memory matrix descriptor of a K-major operand tile whose rows are BK bytes (= one swizzle
+  // span): 8-row groups are 8*BK bytes apart (stride byte offset, bits 32-45), the leading byte offset
+  // (bits 16-29) is unused for swizzled K-major tiles and set to 1, descriptor version 1 (bit 46),
+  // swizzle mode from BK (bits 61-63).  Only the high word is kept here; the low word is
+  // (start address >> 4) | (1 << 16).
+  {
+    const unsigned layout = BK == 128 ? 2u : (BK == 64 ? 4u : 6u);
+    p.desc_hi = (unsigned)((8 * BK) >> 4) | (1u << 14) | (layout << 29);
+  }
   p.bias = a.bias; p.scale = a.scale; p.scale_count = d.scale_count;
   p.res = static_cast<const unsigned char*>(a.residual);
   p.res_mode = res_mode;
   p.res_signed = d.res_type == Q8_S8;
   p.res_scale = a.residual_scale;
   p.y = a.y; p.y_type = d.y_type; p.ldc = a.ldc; p.c_off = a.c_off; p.relu = d.relu;
-  p.y_tma = out8 ? 1 : 0;
+  p.out8 = out8 ? 1 : 0;
   p.y_vec = out8 ? 1 : (aligned16(a.y) && a.ldc % 4 == 0 && a.c_off % 4 == 0);
   p.status = status;
 
-  switch (BN) {
-    case 16: return launch_bk<16>(BK, tmA, tmB, tmRes, tmY, p, a.stream);
-    case 32: return launch_bk<32>(BK, tmA, tmB, tmRes, tmY, p, a.stream);
-    case 64: return launch_bk<64>(BK, tmA, tmB, tmRes, tmY, p, a.stream);
-    case 128: return launch_bk<128>(BK, tmA, tmB, tmRes, tmY, p, a.stream);
-    default: return launch_bk<256>(BK, tmA, tmB, tmRes, tmY, p, a.stream);
-  }
+  const long long tiles = (long long)p.m_tiles * p.n_tiles;
+  int grid = (int)(tiles < sm_count() ? tiles : sm_count());
+  grid = tune_env("Q8_GRID", grid);
+  if (G == 2) return launch_groups<2>(tmA, tmB, tmRes, tmY, p, dyn, grid, a.stream);
+  return launch_groups<4>(tmA, tmB, tmRes, tmY, p, dyn, grid, a.stream);
 }
 
 }  // namespace q8
