@@ -272,35 +272,33 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
   asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
 }
 
-// D[tmem] (+)= A[smem desc] * B[smem desc]^T, 8-bit integer inputs, int32 accumulate.  The 64-bit
-// shared-memory descriptors are handed over as (low, high) words: only the low word (start address)
-// changes between instructions.
-__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
-                                        uint32_t idesc, uint32_t accumulate) {
+// D[tmem] (+)= A[smem desc] * B[smem desc]^T, 8-bit integer inputs, int32 accumulate.  The issuing
+// lane retires about one instruction every six cycles, so the issue path is kept to the bare
+// instruction: descriptors live in 64-bit registers and the always-accumulate form has a constant
+// predicate.
+__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-      "setp.ne.b32 p, %6, 0;\n\t"
-      "mov.b64 da, {%1, %2};\n\t"
-      "mov.b64 db, {%3, %4};\n\t"
-      "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %5, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_i8_acc(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.eq.u32 p, 0, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc)
       : "memory");
 }
 
 // kSteps instructions over one K block of kSteps * 32 bytes: +2 in 16-byte address units per step.
 template <int kSteps>
-__device__ __forceinline__ void umma_i8_block(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
-                                              uint32_t idesc, uint32_t accumulate_first) {
-  umma_i8(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate_first);
+__device__ __forceinline__ void umma_i8_block(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate_first) {
+  umma_i8(d_tmem, a_desc, b_desc, idesc, accumulate_first);
 #pragma unroll
-  for (int k = 1; k < kSteps; ++k) umma_i8(d_tmem, a_lo + 2 * k, a_hi, b_lo + 2 * k, b_hi, idesc, 1u);
-}
-
-__device__ __forceinline__ void umma_i8_ksteps(int ksteps, uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
-                                               uint32_t b_hi, uint32_t idesc, uint32_t accumulate_first) {
-  if (ksteps == 4) umma_i8_block<4>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate_first);
-  else if (ksteps == 2) umma_i8_block<2>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate_first);
-  else umma_i8_block<1>(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate_first);
+  for (int k = 1; k < kSteps; ++k) umma_i8_acc(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc);
 }
 
 // The mbarrier gets one arrival once every tcgen05.mma issued so far by this thread has completed.
@@ -499,6 +497,101 @@ __device__ __forceinline__ void epilogue_row(const UmmaParams& p, const EpiTile&
   }
 }
 
+// ------------------------------------------------------------------------------------------ MMA role
+struct MmaRoleArgs {
+  uint32_t base, tmem_base;
+  uint32_t a_full, a_empty, b_full, b_empty, acc_full, acc_empty, bres_full;
+  const uint32_t* tap_shift16;
+  int total_tiles;
+  volatile int* abortp;
+};
+
+// The single MMA-issuing lane.  kSteps (K block bytes / 32) is a compile-time constant so that the
+// instructions of one K block are straight-line code.  Returns false if a wait gave up.
+template <int kSteps>
+__device__ __forceinline__ bool mma_role(const UmmaParams& p, const MmaRoleArgs& r) {
+  TileIter ti;
+  ti.init(p, blockIdx.x, gridDim.x);
+  const uint32_t nstages = (uint32_t)p.stages, nbst = (uint32_t)p.b_stages;
+  // descriptors: high word constant; low word = start address >> 4 (shared memory ends below 256 KiB,
+  // the 14-bit field never wraps) plus the leading-byte-offset field (bits 16-29), unused for swizzled
+  // K-major tiles and set to 1
+  const uint64_t hi = ((uint64_t)p.desc_hi << 32) | (1ull << 16);
+  const uint64_t a_d0 = hi | (((r.base + p.off_a) >> 4) & 0x3fffu), bring_d0 = hi | (((r.base + p.off_bring) >> 4) & 0x3fffu);
+  const uint64_t bres_d0 = hi | ((r.base >> 4) & 0x3fffu);
+  const uint32_t stage16 = p.a_stage_bytes >> 4, asub16 = p.a_sub_bytes >> 4, bsub16 = p.b_sub_bytes >> 4, btile16 = p.b_tile_bytes >> 4;
+  const uint32_t idesc = p.idesc;
+  const int taps = p.taps, c_blocks = p.c_blocks, k_iters = p.k_iters, kb = p.kb;
+  const bool halo = p.a_mode == kAHalo, ring = p.b_mode == kBRing, b_in_stage = p.b_mode == kBStage;
+  uint32_t stage = 0, phase = 0;
+  uint64_t a_d = a_d0;
+  uint32_t bs = 0, bphase = 0;
+  uint64_t bring_d = bring_d0;
+  uint32_t ab = 0, acc_par = 1;  // accumulator ring position and the parity to wait for on its empty barrier
+  if (p.b_mode == kBResident && !mbar_wait(r.bres_full, 0u, r.abortp)) return false;
+  for (; ti.tile < r.total_tiles; ti.next(p)) {
+    if (!mbar_wait(r.acc_empty + ab * 8u, acc_par, r.abortp)) return false;
+    tcgen05_fence_after();
+    const uint32_t d_tmem = r.tmem_base + ab * (uint32_t)p.acc_stride;
+    uint32_t accum = 0;
+    // resident weights: tile (nt, cb, tap) sits at ((nt * c_blocks + cb) * taps + tap) * b_tile_bytes
+    const uint64_t bres_nt = bres_d0 + (uint32_t)(ti.nt * c_blocks * taps) * btile16;
+    if (halo) {
+      uint64_t bres = bres_nt;  // (cb, tap) is exactly the order of the loops below
+      for (int cb = 0; cb < c_blocks; ++cb) {
+        if (!mbar_wait(r.a_full + stage * 8u, phase, r.abortp)) return false;
+        tcgen05_fence_after();
+        if (ring) {
+          for (int tap = 0; tap < taps; ++tap) {
+            if (!mbar_wait(r.b_full + bs * 8u, bphase, r.abortp)) return false;
+            tcgen05_fence_after();
+            umma_i8_block<kSteps>(d_tmem, a_d + r.tap_shift16[tap], bring_d, idesc, accum);
+            accum = 1;
+            umma_commit(r.b_empty + bs * 8u);
+            bring_d += bsub16;
+            if (++bs == nbst) { bs = 0; bphase ^= 1u; bring_d = bring_d0; }
+          }
+        } else {
+#pragma unroll 3
+          for (int tap = 0; tap < taps; ++tap) {
+            umma_i8_block<kSteps>(d_tmem, a_d + r.tap_shift16[tap], bres, idesc, accum);
+            accum = 1;
+            bres += btile16;
+          }
+        }
+        umma_commit(r.a_empty + stage * 8u);
+        a_d += stage16;
+        if (++stage == nstages) { stage = 0; phase ^= 1u; a_d = a_d0; }
+      }
+    } else {
+      uint64_t bres_tap = bres_nt, bres = bres_nt;  // iterations run over taps with the channel blocks innermost
+      int cb = 0;
+      const uint32_t b_off16 = (uint32_t)kb * asub16;
+      for (int it = 0; it < k_iters;) {
+        const int nsub = min(kb, k_iters - it);
+        if (!mbar_wait(r.a_full + stage * 8u, phase, r.abortp)) return false;
+        tcgen05_fence_after();
+        uint64_t sa = a_d, sb = a_d + b_off16;
+        for (int j = 0; j < nsub; ++j) {
+          umma_i8_block<kSteps>(d_tmem, sa, b_in_stage ? sb : bres, idesc, accum);
+          accum = 1;
+          sa += asub16;
+          sb += bsub16;
+          bres += (uint32_t)taps * btile16;
+          if (++cb == c_blocks) { cb = 0; bres_tap += btile16; bres = bres_tap; }
+        }
+        umma_commit(r.a_empty + stage * 8u);
+        it += nsub;
+        a_d += stage16;
+        if (++stage == nstages) { stage = 0; phase ^= 1u; a_d = a_d0; }
+      }
+    }
+    umma_commit(r.acc_full + ab * 8u);
+    if (++ab == (uint32_t)p.nacc) { ab = 0; acc_par ^= 1u; }
+  }
+  return true;
+}
+
 // ------------------------------------------------------------------------------------------ kernel
 // G epilogue groups; one instantiation per output type and residual source keeps a single epilogue
 // body in each kernel (several of them in one kernel made the register allocator spill).
@@ -512,7 +605,8 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
   __shared__ __align__(8) unsigned long long b_full[kMaxBStages], b_empty[kMaxBStages];
   __shared__ __align__(8) unsigned long long acc_full[kMaxAcc], acc_empty[kMaxAcc];
   __shared__ __align__(8) unsigned long long buf_full[kMaxSlots], buf_empty[kMaxSlots];
-  __shared__ __align__(8) unsigned long long store_ready[kMaxGroups];
+  __shared__ __align__(8) unsigned long long store_ready[kMaxSlots];  // per buffer: a buffer is recycled by the store
+                                                                        // lane between two uses, so no phase can be skipped
   __shared__ __align__(8) unsigned long long bres_full;
   __shared__ uint32_t tap_shift16[kMaxTaps];  // halo: descriptor start offset of a tap, in 16-byte units
   __shared__ uint32_t tmem_holder;
@@ -549,7 +643,7 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       mbar_init(smem_u32(&buf_full[i]), 1);
       mbar_init(smem_u32(&buf_empty[i]), 1);
     }
-    for (int g = 0; g < G; ++g) mbar_init(smem_u32(&store_ready[g]), kGroupThreads);
+    for (int i = 0; i < slots; ++i) mbar_init(smem_u32(&store_ready[i]), kGroupThreads);
     mbar_init(smem_u32(&bres_full), 1);
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -659,84 +753,16 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
     }
   } else if (threadIdx.x == 32) {
     // ------------------------------------------------------------------ MMA issuer
-    TileIter ti;
-    ti.init(p, blockIdx.x, gridDim.x);
-    const uint32_t nstages = (uint32_t)p.stages, nbst = (uint32_t)p.b_stages;
-    const uint32_t afull0 = smem_u32(&a_full[0]), aempty0 = smem_u32(&a_empty[0]);
-    const uint32_t bfull0 = smem_u32(&b_full[0]), bempty0 = smem_u32(&b_empty[0]);
-    const uint32_t accf0 = smem_u32(&acc_full[0]), acce0 = smem_u32(&acc_empty[0]);
-    // low descriptor words: start address >> 4 (shared memory ends below 256 KiB, the 14-bit field never
-    // wraps) plus the leading-byte-offset field (bits 16-29), unused for swizzled K-major tiles and set to 1
-    const uint32_t lbo = 1u << 16;
-    const uint32_t a_lo0 = (((base + p.off_a) >> 4) & 0x3fffu) | lbo, bring_lo0 = (((base + p.off_bring) >> 4) & 0x3fffu) | lbo;
-    const uint32_t bres_lo0 = ((base >> 4) & 0x3fffu) | lbo;
-    const uint32_t stage16 = p.a_stage_bytes >> 4, asub16 = p.a_sub_bytes >> 4, bsub16 = p.b_sub_bytes >> 4, btile16 = p.b_tile_bytes >> 4;
-    const uint32_t hi = p.desc_hi;
-    const int ksteps = p.ksteps;
-    uint32_t stage = 0, phase = 0, a_lo = a_lo0;
-    uint32_t bs = 0, bphase = 0, bring_lo = bring_lo0;
-    uint32_t ab = 0, acc_par = 1;  // accumulator ring position and the parity to wait for on its empty barrier
-    bool ok = true;
-    if (p.b_mode == kBResident) ok = mbar_wait(smem_u32(&bres_full), 0u, abortp);
-    for (; ti.tile < total_tiles && ok; ti.next(p)) {
-      if (!mbar_wait(acce0 + ab * 8u, acc_par, abortp)) { ok = false; break; }
-      tcgen05_fence_after();
-      const uint32_t d_tmem = tmem_base + ab * (uint32_t)p.acc_stride;
-      uint32_t accum = 0;
-      // resident weights: tile (nt, cb, tap) sits at ((nt * c_blocks + cb) * taps + tap) * b_tile_bytes
-      const uint32_t bres_nt = bres_lo0 + (uint32_t)(ti.nt * p.c_blocks * p.taps) * btile16;
-      if (p.a_mode == kAHalo) {
-        uint32_t bres = bres_nt;  // (cb, tap) is exactly the order of the loops below
-        for (int cb = 0; cb < p.c_blocks && ok; ++cb) {
-          if (!mbar_wait(afull0 + stage * 8u, phase, abortp)) { ok = false; break; }
-          tcgen05_fence_after();
-          for (int tap = 0; tap < p.taps; ++tap) {
-            uint32_t b_lo = bres;
-            if (p.b_mode == kBRing) {
-              if (!mbar_wait(bfull0 + bs * 8u, bphase, abortp)) { ok = false; break; }
-              tcgen05_fence_after();
-              b_lo = bring_lo;
-            }
-            umma_i8_ksteps(ksteps, d_tmem, a_lo + tap_shift16[tap], hi, b_lo, hi, p.idesc, accum);
-            accum = 1;
-            if (p.b_mode == kBRing) {
-              umma_commit(bempty0 + bs * 8u);
-              bring_lo += bsub16;
-              if (++bs == nbst) { bs = 0; bphase ^= 1u; bring_lo = bring_lo0; }
-            } else {
-              bres += btile16;
-            }
-          }
-          umma_commit(aempty0 + stage * 8u);
-          a_lo += stage16;
-          if (++stage == nstages) { stage = 0; phase ^= 1u; a_lo = a_lo0; }
-        }
-      } else {
-        uint32_t bres_tap = bres_nt, bres = bres_nt;  // iterations run over taps with the channel blocks innermost
-        int cb = 0;
-        const uint32_t b_in_stage16 = (uint32_t)p.kb * asub16;
-        for (int it = 0; it < p.k_iters;) {
-          const int nsub = min(p.kb, p.k_iters - it);
-          if (!mbar_wait(afull0 + stage * 8u, phase, abortp)) { ok = false; break; }
-          tcgen05_fence_after();
-          uint32_t sa = a_lo, sb = a_lo + b_in_stage16;
-          for (int j = 0; j < nsub; ++j) {
-            umma_i8_ksteps(ksteps, d_tmem, sa, hi, p.b_mode == kBStage ? sb : bres, hi, p.idesc, accum);
-            accum = 1;
-            sa += asub16;
-            sb += bsub16;
-            bres += (uint32_t)p.taps * btile16;
-            if (++cb == p.c_blocks) { cb = 0; bres_tap += btile16; bres = bres_tap; }
-          }
-          umma_commit(aempty0 + stage * 8u);
-          it += nsub;
-          a_lo += stage16;
-          if (++stage == nstages) { stage = 0; phase ^= 1u; a_lo = a_lo0; }
-        }
-      }
-      if (ok) umma_commit(accf0 + ab * 8u);
-      if (++ab == (uint32_t)p.nacc) { ab = 0; acc_par ^= 1u; }
-    }
+    MmaRoleArgs ra;
+    ra.base = base; ra.tmem_base = tmem_base; ra.total_tiles = total_tiles; ra.abortp = abortp;
+    ra.a_full = smem_u32(&a_full[0]); ra.a_empty = smem_u32(&a_empty[0]);
+    ra.b_full = smem_u32(&b_full[0]); ra.b_empty = smem_u32(&b_empty[0]);
+    ra.acc_full = smem_u32(&acc_full[0]); ra.acc_empty = smem_u32(&acc_empty[0]);
+    ra.bres_full = smem_u32(&bres_full); ra.tap_shift16 = tap_shift16;
+    bool ok;
+    if (p.ksteps == 4) ok = mma_role<4>(p, ra);
+    else if (p.ksteps == 2) ok = mma_role<2>(p, ra);
+    else ok = mma_role<1>(p, ra);
     if (!ok) {
       abort_flag = 1;
       atomicOr(p.status, kTimeoutMma);
@@ -780,13 +806,13 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       ti.init(p, blockIdx.x, gridDim.x);
       const uint32_t bempty0 = smem_u32(&buf_empty[0]), ready0 = smem_u32(&store_ready[0]);
       const uint32_t nslots = (uint32_t)slots;
-      uint32_t slot = 0, g = 0, gpar = 0;  // tile lt belongs to group lt % G, its j-th tile has parity j & 1
+      uint32_t slot = 0, spar = 0;  // tile lt uses buffer lt % (G*nbuf); its use number (lt / (G*nbuf)) gives the parity
       int prev_slot = -1;
       bool ok = true;
       const int pw = 1 << p.pw_shift;
       const uint32_t panel_bytes = (uint32_t)kBM << p.pw_shift;
       for (; ti.tile < total_tiles; ti.next(p)) {
-        if (!mbar_wait(ready0 + g * 8u, gpar, abortp)) { ok = false; break; }
+        if (!mbar_wait(ready0 + slot * 8u, spar, abortp)) { ok = false; break; }
         if (p.out8) {
           uint32_t src = base + p.off_bufs + slot * p.tile8_bytes;
           if (p.a_mode == kAHalo) {
@@ -802,8 +828,7 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
         } else {
           mbar_arrive(bempty0 + slot * 8u);
         }
-        if (++slot == nslots) slot = 0;
-        if (++g == (uint32_t)G) { g = 0; gpar ^= 1u; }
+        if (++slot == nslots) { slot = 0; spar ^= 1u; }
       }
       if (p.out8) {
         bulk_wait_read<0>();  // the CTA's shared memory must outlive the reads of its last stores
@@ -834,7 +859,7 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
     }
     // this group's tiles are lt = g, g + G, ... of the CTA's sequence; ring positions advance by additions
     const uint32_t accf0 = smem_u32(&acc_full[0]), acce0 = smem_u32(&acc_empty[0]);
-    const uint32_t bfull0 = smem_u32(&buf_full[0]), ready = smem_u32(&store_ready[g]);
+    const uint32_t bfull0 = smem_u32(&buf_full[0]), ready0 = smem_u32(&store_ready[0]);
     const uint32_t nslots = (uint32_t)slots, nacc = (uint32_t)p.nacc;
     uint32_t ab = (uint32_t)g % nacc, acc_par = ((uint32_t)g / nacc) & 1u;
     uint32_t slot = (uint32_t)g, slot_par = 0;
@@ -867,7 +892,7 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       if (p.nbuf > 0) {
         // this thread's reads and writes of the buffer are done; the store thread takes over
         if (p.out8) fence_proxy_async_smem();
-        mbar_arrive(ready);
+        mbar_arrive(ready0 + slot * 8u);
       }
       ab += (uint32_t)G;
       while (ab >= nacc) { ab -= nacc; acc_par ^= 1u; }
