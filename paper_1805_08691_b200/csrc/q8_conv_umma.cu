@@ -25,14 +25,15 @@
 //     stage    : (plain, im2col) one BN x BK tile next to each A block of a stage.
 //
 // Roles (one lane each unless noted):
-//   thread 0   : TMA producer of A patches / blocks and of B tiles;
-//   thread 32  : tcgen05.mma.kind::i8 issue (128 x BN x 32 per instruction, int32 accumulators in a
-//                ring of up to four TMEM buffers); tcgen05.commit releases stages and publishes
-//                accumulators.  Warp 1 also owns the TMEM allocation;
-//   thread 64  : hands 8-bit tile buffers to the epilogue groups, filled by TMA with the residual
+//   warp 0     : TMA producer of A patches / blocks and of B tiles;
+//   warps 1, 4 : tcgen05.mma.kind::i8 issue (128 x BN x 32 per instruction, int32 accumulators in a
+//                ring of up to four TMEM buffers), alternate tiles each, so that the per-tile
+//                bookkeeping of one lane overlaps the issue of the other; tcgen05.commit releases
+//                stages and publishes accumulators.  Warp 1 also owns the TMEM allocation;
+//   warp 2     : hands 8-bit tile buffers to the epilogue groups, filled by TMA with the residual
 //                tile of the fused eltwise sum when there is one;
-//   thread 96  : sends finished 8-bit tiles to global memory with TMA stores, recycles the buffers;
-//   warps 4..  : G epilogue groups of four warps; group g owns every G-th tile of the CTA.  A thread
+//   warp 3     : sends finished 8-bit tiles to global memory with TMA stores, recycles the buffers;
+//   warps 6..  : G epilogue groups of four warps; group g owns every G-th tile of the CTA.  A thread
 //                owns one accumulator row: tcgen05.ld, + bias, requantise, + residual, ReLU, round,
 //                clamp; the 16 bytes go back into the buffer the residual came from (same swizzled
 //                position), which then is the source of the TMA store.
@@ -51,7 +52,9 @@ namespace q8 {
 namespace {
 
 constexpr int kBM = 128;
-constexpr int kCtrlThreads = 128;       // warps 0-3
+constexpr int kCtrlWarps = 6;            // producer, MMA 0, buffers/residual, store, MMA 1, spare
+constexpr int kCtrlThreads = kCtrlWarps * 32;
+constexpr int kMmaWarps = 2;             // MMA-issuing lanes, tile lt belongs to lane lt % kMmaWarps
 constexpr int kGroupThreads = 128;      // one epilogue group
 constexpr int kMaxStages = 8;           // A stages
 constexpr int kMaxBStages = 8;          // weight ring
@@ -500,7 +503,7 @@ __device__ __forceinline__ void epilogue_row(const UmmaParams& p, const EpiTile&
 // ------------------------------------------------------------------------------------------ MMA role
 struct MmaRoleArgs {
   uint32_t base, tmem_base;
-  uint32_t a_full, a_empty, b_full, b_empty, acc_full, acc_empty, bres_full;
+  uint32_t a_full, a_empty, b_full, b_empty, acc_full, acc_empty, bres_full, turn;
   const uint32_t* tap_shift16;
   int total_tiles;
   volatile int* abortp;
@@ -509,9 +512,14 @@ struct MmaRoleArgs {
 // The single MMA-issuing lane.  kSteps (K block bytes / 32) is a compile-time constant so that the
 // instructions of one K block are straight-line code.  Returns false if a wait gave up.
 template <int kSteps>
-__device__ __forceinline__ bool mma_role(const UmmaParams& p, const MmaRoleArgs& r) {
+__device__ __forceinline__ bool mma_role(const UmmaParams& p, const MmaRoleArgs& r, const int who) {
+  // This lane's tiles are lt = who, who + kMmaWarps, ... of the CTA's sequence; the stage, weight-ring
+  // and accumulator positions of a tile follow from lt alone.  A parity wait is only meaningful for
+  // the use of a barrier that is in flight, so a lane starts the stage waits of tile lt only after
+  // the lane of tile lt - 1 has passed all of its own (the turn barriers); the per-tile bookkeeping
+  // and the accumulator wait run ahead of that.
   TileIter ti;
-  ti.init(p, blockIdx.x, gridDim.x);
+  ti.init(p, blockIdx.x + who * (int)gridDim.x, kMmaWarps * (int)gridDim.x);
   const uint32_t nstages = (uint32_t)p.stages, nbst = (uint32_t)p.b_stages;
   // descriptors: high word constant; low word = start address >> 4 (shared memory ends below 256 KiB,
   // the 14-bit field never wraps) plus the leading-byte-offset field (bits 16-29), unused for swizzled
@@ -523,14 +531,26 @@ __device__ __forceinline__ bool mma_role(const UmmaParams& p, const MmaRoleArgs&
   const uint32_t idesc = p.idesc;
   const int taps = p.taps, c_blocks = p.c_blocks, k_iters = p.k_iters, kb = p.kb;
   const bool halo = p.a_mode == kAHalo, ring = p.b_mode == kBRing, b_in_stage = p.b_mode == kBStage;
-  uint32_t stage = 0, phase = 0;
-  uint64_t a_d = a_d0;
+  // ring positions of tile lt = who, and how far the other lanes' tiles move them between two of ours
+  const uint32_t spt = halo ? (uint32_t)c_blocks : (uint32_t)((k_iters + kb - 1) / kb);  // A stages per tile
+  const uint32_t bpt = (uint32_t)(taps * c_blocks);                                       // ring tiles per tile
+  const uint32_t skip_a = (kMmaWarps - 1) * spt, skip_b = (kMmaWarps - 1) * bpt;
+  uint32_t stage = ((uint32_t)who * spt) % nstages, phase = (((uint32_t)who * spt) / nstages) & 1u;
   uint32_t bs = 0, bphase = 0;
-  uint64_t bring_d = bring_d0;
-  uint32_t ab = 0, acc_par = 1;  // accumulator ring position and the parity to wait for on its empty barrier
+  if (ring) { bs = ((uint32_t)who * bpt) % nbst; bphase = (((uint32_t)who * bpt) / nbst) & 1u; }
+  uint64_t a_d = a_d0 + stage * stage16;
+  uint64_t bring_d = bring_d0 + bs * bsub16;
+  const uint32_t nacc = (uint32_t)p.nacc;
+  uint32_t ab = (uint32_t)who % nacc, acc_par = 1u ^ (((uint32_t)who / nacc) & 1u);  // accumulator and the parity of its empty barrier
+  uint32_t my_k = 0;  // number of tiles this lane has issued
+  const uint32_t turn_next = r.turn + (who == 0 ? 8u : 0u);  // the other lane's turn barrier
   if (p.b_mode == kBResident && !mbar_wait(r.bres_full, 0u, r.abortp)) return false;
   for (; ti.tile < r.total_tiles; ti.next(p)) {
     if (!mbar_wait(r.acc_empty + ab * 8u, acc_par, r.abortp)) return false;
+    // turn[w] counts the tiles the other lane has finished waiting for: tile number k of lane 0 needs
+    // k of them, tile number k of lane 1 needs k + 1
+    if (who == 0) { if (my_k > 0 && !mbar_wait(r.turn, (my_k - 1) & 1u, r.abortp)) return false; }
+    else if (!mbar_wait(r.turn + 8u, my_k & 1u, r.abortp)) return false;
     tcgen05_fence_after();
     const uint32_t d_tmem = r.tmem_base + ab * (uint32_t)p.acc_stride;
     uint32_t accum = 0;
@@ -540,10 +560,13 @@ __device__ __forceinline__ bool mma_role(const UmmaParams& p, const MmaRoleArgs&
       uint64_t bres = bres_nt;  // (cb, tap) is exactly the order of the loops below
       for (int cb = 0; cb < c_blocks; ++cb) {
         if (!mbar_wait(r.a_full + stage * 8u, phase, r.abortp)) return false;
+        const bool last_cb = cb == c_blocks - 1;
+        if (last_cb && !ring) mbar_arrive(turn_next);  // this tile's last wait is behind us
         tcgen05_fence_after();
         if (ring) {
           for (int tap = 0; tap < taps; ++tap) {
             if (!mbar_wait(r.b_full + bs * 8u, bphase, r.abortp)) return false;
+            if (last_cb && tap == taps - 1) mbar_arrive(turn_next);
             tcgen05_fence_after();
             umma_i8_block<kSteps>(d_tmem, a_d + r.tap_shift16[tap], bring_d, idesc, accum);
             accum = 1;
@@ -570,6 +593,7 @@ __device__ __forceinline__ bool mma_role(const UmmaParams& p, const MmaRoleArgs&
       for (int it = 0; it < k_iters;) {
         const int nsub = min(kb, k_iters - it);
         if (!mbar_wait(r.a_full + stage * 8u, phase, r.abortp)) return false;
+        if (it + nsub >= k_iters) mbar_arrive(turn_next);  // this tile's last wait is behind us
         tcgen05_fence_after();
         uint64_t sa = a_d, sb = a_d + b_off16;
         for (int j = 0; j < nsub; ++j) {
@@ -586,8 +610,19 @@ __device__ __forceinline__ bool mma_role(const UmmaParams& p, const MmaRoleArgs&
         if (++stage == nstages) { stage = 0; phase ^= 1u; a_d = a_d0; }
       }
     }
+    ++my_k;
     umma_commit(r.acc_full + ab * 8u);
-    if (++ab == (uint32_t)p.nacc) { ab = 0; acc_par ^= 1u; }
+    ab += kMmaWarps;
+    while (ab >= nacc) { ab -= nacc; acc_par ^= 1u; }
+    // step over the stages and ring tiles of the other lanes' tiles
+    stage += skip_a;
+    while (stage >= nstages) { stage -= nstages; phase ^= 1u; }
+    a_d = a_d0 + stage * stage16;
+    if (ring) {
+      bs += skip_b;
+      while (bs >= nbst) { bs -= nbst; bphase ^= 1u; }
+      bring_d = bring_d0 + bs * bsub16;
+    }
   }
   return true;
 }
@@ -608,6 +643,7 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
   __shared__ __align__(8) unsigned long long store_ready[kMaxSlots];  // per buffer: a buffer is recycled by the store
                                                                         // lane between two uses, so no phase can be skipped
   __shared__ __align__(8) unsigned long long bres_full;
+  __shared__ __align__(8) unsigned long long mma_turn[kMmaWarps];
   __shared__ uint32_t tap_shift16[kMaxTaps];  // halo: descriptor start offset of a tap, in 16-byte units
   __shared__ uint32_t tmem_holder;
   __shared__ int abort_flag;
@@ -645,6 +681,7 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
     }
     for (int i = 0; i < slots; ++i) mbar_init(smem_u32(&store_ready[i]), kGroupThreads);
     mbar_init(smem_u32(&bres_full), 1);
+    for (int i = 0; i < kMmaWarps; ++i) mbar_init(smem_u32(&mma_turn[i]), 1);
     abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -751,18 +788,19 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       abort_flag = 1;
       atomicOr(p.status, kTimeoutProducer);
     }
-  } else if (threadIdx.x == 32) {
-    // ------------------------------------------------------------------ MMA issuer
+  } else if (threadIdx.x == 32 || threadIdx.x == 128) {
+    // ------------------------------------------------------------------ MMA issuers (lane 0 of warps 1 and 4)
+    const int who = threadIdx.x == 32 ? 0 : 1;
     MmaRoleArgs ra;
     ra.base = base; ra.tmem_base = tmem_base; ra.total_tiles = total_tiles; ra.abortp = abortp;
     ra.a_full = smem_u32(&a_full[0]); ra.a_empty = smem_u32(&a_empty[0]);
     ra.b_full = smem_u32(&b_full[0]); ra.b_empty = smem_u32(&b_empty[0]);
     ra.acc_full = smem_u32(&acc_full[0]); ra.acc_empty = smem_u32(&acc_empty[0]);
-    ra.bres_full = smem_u32(&bres_full); ra.tap_shift16 = tap_shift16;
+    ra.bres_full = smem_u32(&bres_full); ra.tap_shift16 = tap_shift16; ra.turn = smem_u32(&mma_turn[0]);
     bool ok;
-    if (p.ksteps == 4) ok = mma_role<4>(p, ra);
-    else if (p.ksteps == 2) ok = mma_role<2>(p, ra);
-    else ok = mma_role<1>(p, ra);
+    if (p.ksteps == 4) ok = mma_role<4>(p, ra, who);
+    else if (p.ksteps == 2) ok = mma_role<2>(p, ra, who);
+    else ok = mma_role<1>(p, ra, who);
     if (!ok) {
       abort_flag = 1;
       atomicOr(p.status, kTimeoutMma);
@@ -839,9 +877,9 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
         atomicOr(p.status, kTimeoutStore);
       }
     }
-  } else if (warp >= 4) {
+  } else if (warp >= kCtrlWarps) {
     // ------------------------------------------------------------------ epilogue groups
-    const int g = (warp - 4) >> 2;
+    const int g = (warp - kCtrlWarps) >> 2;
     const int quad = warp & 3;  // TMEM lane quadrant this warp may read
     const int row = quad * 32 + lane;  // accumulator row of this thread
     EpiTile t;
