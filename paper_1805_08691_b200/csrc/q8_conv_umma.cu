@@ -60,7 +60,6 @@ constexpr int kMaxStages = 8;           // A stages
 constexpr int kMaxBStages = 8;          // weight ring
 constexpr int kMaxAcc = 4;
 constexpr int kMaxSlots = 8;            // 8-bit tile buffers over all groups
-constexpr int kMaxGroups = 4;
 constexpr int kMaxTaps = 64;            // halo mode keeps a descriptor offset per tap in shared memory
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
 constexpr int kSmemLimit = 232448;                           // 227 KiB opt-in maximum per CTA
@@ -78,6 +77,16 @@ enum ResMode : int { kResNone = 0, kResTma = 1, kResGlobal = 2 };
 enum AMode : int { kAPlain = 0, kAIm2col = 1, kAHalo = 2 };
 enum BMode : int { kBStage = 0, kBResident = 1, kBRing = 2 };
 
+// Division by a launch-time constant without the ~35-instruction software divide, which costs a
+// lone control lane some 200 cycles: q = (umulhi(x, m) + x) >> l for 0 <= x < 2^31 (Granlund-Montgomery).
+struct FastDiv {
+  unsigned int m, l;
+  int d;
+#ifdef __CUDACC__
+  __device__ __forceinline__ int div(int x) const { return (int)((__umulhi((unsigned int)x, m) + (unsigned int)x) >> l); }
+#endif
+};
+
 struct UmmaParams {
   int M, K;                  // GEMM rows (pixels) and Cout
   int P, Q, PQ;              // output height, width, pixels per image
@@ -93,6 +102,7 @@ struct UmmaParams {
   int nacc, acc_stride, tmem_cols;  // TMEM accumulators, columns between them, allocation (power of two)
   int nbuf;                  // 8-bit tile buffers per epilogue group (0: none)
   int m_tiles, n_tiles;
+  FastDiv fd_ntiles, fd_perimg, fd_qtiles, fd_pq, fd_q;  // n_tiles, p_tiles*q_tiles, q_tiles, P*Q, Q
   unsigned int idesc;        // tcgen05 instruction descriptor
   unsigned int desc_hi;      // high word of the shared-memory matrix descriptors
   unsigned int a_sub_bytes;  // plain/im2col: one 128 x bk block; halo: bytes of one patch load
@@ -126,17 +136,17 @@ struct TileIter {
 
   __device__ __forceinline__ void init(const UmmaParams& p, int first, int step_) {
     tile = first; step = step_;
-    mt = first / p.n_tiles; nt = first - mt * p.n_tiles;
-    d_mt = step_ / p.n_tiles; d_nt = step_ - d_mt * p.n_tiles;
+    mt = p.fd_ntiles.div(first); nt = first - mt * p.n_tiles;
+    d_mt = p.fd_ntiles.div(step_); d_nt = step_ - d_mt * p.n_tiles;
     img = pt = qt = d_img = d_pt = d_qt = 0;
     if (p.a_mode == kAHalo) {
       const int per_img = p.p_tiles * p.q_tiles;
-      img = mt / per_img;
+      img = p.fd_perimg.div(mt);
       int r = mt - img * per_img;
-      pt = r / p.q_tiles; qt = r - pt * p.q_tiles;
-      d_img = d_mt / per_img;
+      pt = p.fd_qtiles.div(r); qt = r - pt * p.q_tiles;
+      d_img = p.fd_perimg.div(d_mt);
       r = d_mt - d_img * per_img;
-      d_pt = r / p.q_tiles; d_qt = r - d_pt * p.q_tiles;
+      d_pt = p.fd_qtiles.div(r); d_qt = r - d_pt * p.q_tiles;
     }
   }
   __device__ __forceinline__ void next(const UmmaParams& p) {
@@ -658,50 +668,54 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
   const int total_tiles = p.m_tiles * p.n_tiles;
   const int slots = G * p.nbuf;
 
-  if (threadIdx.x == 0) {
-    prefetch_tensormap(&tmA);
-    prefetch_tensormap(&tmB);
-    if (p.res_mode == kResTma) prefetch_tensormap(&tmRes);
-    if (p.out8) prefetch_tensormap(&tmY);
-    for (int s = 0; s < p.stages; ++s) {
-      mbar_init(smem_u32(&a_full[s]), 1);
-      mbar_init(smem_u32(&a_empty[s]), 1);
-    }
-    for (int s = 0; s < p.b_stages; ++s) {
-      mbar_init(smem_u32(&b_full[s]), 1);
-      mbar_init(smem_u32(&b_empty[s]), 1);
-    }
-    for (int i = 0; i < p.nacc; ++i) {
-      mbar_init(smem_u32(&acc_full[i]), 1);
-      mbar_init(smem_u32(&acc_empty[i]), 4);  // one arrival per epilogue warp of the owning group
-    }
-    for (int i = 0; i < slots; ++i) {
-      mbar_init(smem_u32(&buf_full[i]), 1);
-      mbar_init(smem_u32(&buf_empty[i]), 1);
-    }
-    for (int i = 0; i < slots; ++i) mbar_init(smem_u32(&store_ready[i]), kGroupThreads);
-    mbar_init(smem_u32(&bres_full), 1);
-    for (int i = 0; i < kMmaWarps; ++i) mbar_init(smem_u32(&mma_turn[i]), 1);
-    abort_flag = 0;
+  // Prologue.  Each control lane initialises the barriers it owns.  Warp 0 only signals the
+  // start-up barrier (bar.arrive) and goes straight to its loads, so that the first bytes are on
+  // their way while the others allocate TMEM and fetch bias and scale; everybody else waits on it.
+  const int nthreads = kCtrlThreads + G * kGroupThreads;
+  if (warp == 0) {
+    // one barrier per lane: a lone lane would spend ~50 cycles on each
+    if (lane < p.stages) { mbar_init(smem_u32(&a_full[lane]), 1); mbar_init(smem_u32(&a_empty[lane]), 1); }
+    else if (lane >= 8 && lane - 8 < p.b_stages) { mbar_init(smem_u32(&b_full[lane - 8]), 1); mbar_init(smem_u32(&b_empty[lane - 8]), 1); }
+    else if (lane == 16) { mbar_init(smem_u32(&bres_full), 1); abort_flag = 0; }
+    else if (lane == 17) prefetch_tensormap(&tmA);
+    else if (lane == 18) prefetch_tensormap(&tmB);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncwarp();
+    asm volatile("bar.arrive 1, %0;" ::"r"(nthreads) : "memory");
+  } else {
+    if (warp == 1) {
+      if (lane < p.nacc) { mbar_init(smem_u32(&acc_full[lane]), 1); mbar_init(smem_u32(&acc_empty[lane]), 4); }  // 4: one arrival per epilogue warp
+      else if (lane >= 8 && lane - 8 < kMmaWarps) mbar_init(smem_u32(&mma_turn[lane - 8]), 1);
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    } else if (warp == 2) {
+      if (lane < slots) { mbar_init(smem_u32(&buf_full[lane]), 1); mbar_init(smem_u32(&buf_empty[lane]), 1); }
+      else if (lane == 16 && p.res_mode == kResTma) prefetch_tensormap(&tmRes);
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    } else if (warp == 3) {
+      if (lane < slots) mbar_init(smem_u32(&store_ready[lane]), kGroupThreads);
+      else if (lane == 16 && p.out8) prefetch_tensormap(&tmY);
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+      __syncwarp();
+      tmem_alloc(smem_u32(&tmem_holder), (uint32_t)p.tmem_cols);
+      tmem_relinquish();
+    }
+    if (p.a_mode == kAHalo && threadIdx.x >= 32 && threadIdx.x - 32 < p.taps) {
+      const int tap = threadIdx.x - 32;
+      const int r = tap / p.S, s = tap - r * p.S;
+      tap_shift16[tap] = (uint32_t)((r * p.dil_h * p.twb + s * p.dil_w) * p.bk) >> 4;
+    }
+    // bias and scale of every channel, once per CTA (zero beyond Cout; one scale replicated if per tensor)
+    for (int i = threadIdx.x - 32; i < p.k_pad; i += nthreads - 32) {
+      s_bias[i] = (p.bias && i < p.K) ? p.bias[i] : 0;
+      s_scale[i] = p.scale ? (p.scale_count == 1 ? p.scale[0] : (i < p.K ? p.scale[i] : 0.f)) : 0.f;
+    }
+    tcgen05_fence_before();
+    asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
+    tcgen05_fence_after();
   }
-  if (warp == 1) {
-    tmem_alloc(smem_u32(&tmem_holder), (uint32_t)p.tmem_cols);
-    tmem_relinquish();
-  }
-  if (p.a_mode == kAHalo && threadIdx.x < p.taps) {
-    const int r = threadIdx.x / p.S, s = threadIdx.x - r * p.S;
-    tap_shift16[threadIdx.x] = (uint32_t)((r * p.dil_h * p.twb + s * p.dil_w) * p.bk) >> 4;
-  }
-  // bias and scale of every channel, once per CTA (zero beyond Cout; one scale replicated if per tensor)
-  for (int i = threadIdx.x; i < p.k_pad; i += blockDim.x) {
-    s_bias[i] = (p.bias && i < p.K) ? p.bias[i] : 0;
-    s_scale[i] = p.scale ? (p.scale_count == 1 ? p.scale[0] : (i < p.K ? p.scale[i] : 0.f)) : 0.f;
-  }
-  tcgen05_fence_before();
-  __syncthreads();
-  tcgen05_fence_after();
-  const uint32_t tmem_base = tmem_holder;
+  const uint32_t tmem_base = warp == 0 ? 0u : tmem_holder;  // warp 0 never touches TMEM
   volatile int* abortp = &abort_flag;
 
   if (threadIdx.x == 0) {
@@ -753,9 +767,9 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
         const int m0 = ti.mt * kBM, n0 = ti.nt * p.bn;
         int w0 = 0, h0 = 0, img = 0;
         if (p.a_mode == kAIm2col) {
-          img = m0 / p.PQ;
+          img = p.fd_pq.div(m0);
           const int rem = m0 - img * p.PQ;
-          const int pr = rem / p.Q, qc = rem - pr * p.Q;
+          const int pr = p.fd_q.div(rem), qc = rem - pr * p.Q;
           h0 = pr * p.stride_h - p.pad_h;
           w0 = qc * p.stride_w - p.pad_w;
         }
@@ -890,7 +904,7 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
     t.srow = row;
     t.smem_ok = true;
     if (p.a_mode == kAHalo) {
-      pp = row / p.twb;
+      pp = row / p.twb;  // once per thread
       qq = row - pp * p.twb;
       t.smem_ok = pp < p.th && qq < p.tw;
       t.srow = t.smem_ok ? pp * p.tw + qq : 0;
@@ -1023,6 +1037,16 @@ CUtensorMapSwizzle swizzle_for_bytes(int row_bytes) {
 }
 
 unsigned int round_up(unsigned int v, unsigned int a) { return (v + a - 1) / a * a; }
+
+FastDiv make_fastdiv(int d) {
+  FastDiv f;
+  f.d = d < 1 ? 1 : d;
+  unsigned int l = 0;
+  while ((1ull << l) < (unsigned long long)f.d) ++l;
+  f.l = l;
+  f.m = (unsigned int)(((1ull << 32) * ((1ull << l) - (unsigned long long)f.d)) / (unsigned long long)f.d + 1ull);
+  return f;
+}
 
 int tune_env(const char* name, int dflt) {
   const char* v = getenv(name);
@@ -1162,6 +1186,11 @@ int launch_conv_umma(const ConvArgs& a) {
   } else {
     p.m_tiles = (int)((a.M + kBM - 1) / kBM);
   }
+  p.fd_ntiles = make_fastdiv(p.n_tiles);
+  p.fd_perimg = make_fastdiv(p.a_mode == kAHalo ? p.p_tiles * p.q_tiles : 1);
+  p.fd_qtiles = make_fastdiv(p.a_mode == kAHalo ? p.q_tiles : 1);
+  p.fd_pq = make_fastdiv(p.PQ);
+  p.fd_q = make_fastdiv(p.Q);
   p.tile8_bytes = (unsigned)(kBM * BN);  // a multiple of 2 KiB
   p.acc_stride = 32;
   while (p.acc_stride < BN) p.acc_stride *= 2;
