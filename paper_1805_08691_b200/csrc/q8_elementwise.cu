@@ -90,19 +90,24 @@ __device__ __forceinline__ unsigned int pack4(int a, int b, int c, int d) {
          ((unsigned int)(d & 0xff) << 24);
 }
 
-// 16 floats in, 16 bytes out per thread and step.  Requires x and z 16-byte aligned.
-__global__ void __launch_bounds__(kThreads) quantize8_vec_kernel(const float4* __restrict__ x, size_t n16,
+// One float4 in, four bytes out per thread and step: a warp reads 512 contiguous bytes and writes 128.
+// Four independent steps are in flight per thread.  n4 = number of float4.  Requires x 16-byte and z
+// 4-byte aligned.
+__global__ void __launch_bounds__(kThreads) quantize8_vec_kernel(const float4* __restrict__ x, size_t n4,
                                                                  float q, int lo, int hi,
-                                                                 uint4* __restrict__ z) {
+                                                                 unsigned int* __restrict__ z) {
   const size_t nthreads = (size_t)gridDim.x * blockDim.x;
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += nthreads) {
-    float4 a = __ldcs(x + 4 * i), b = __ldcs(x + 4 * i + 1), c = __ldcs(x + 4 * i + 2), d = __ldcs(x + 4 * i + 3);
-    uint4 o;
-    o.x = pack4(quant1(a.x, q, lo, hi), quant1(a.y, q, lo, hi), quant1(a.z, q, lo, hi), quant1(a.w, q, lo, hi));
-    o.y = pack4(quant1(b.x, q, lo, hi), quant1(b.y, q, lo, hi), quant1(b.z, q, lo, hi), quant1(b.w, q, lo, hi));
-    o.z = pack4(quant1(c.x, q, lo, hi), quant1(c.y, q, lo, hi), quant1(c.z, q, lo, hi), quant1(c.w, q, lo, hi));
-    o.w = pack4(quant1(d.x, q, lo, hi), quant1(d.y, q, lo, hi), quant1(d.z, q, lo, hi), quant1(d.w, q, lo, hi));
-    __stcs(z + i, o);
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  for (; i + 3 * nthreads < n4; i += 4 * nthreads) {
+    const float4 a = __ldcs(x + i), b = __ldcs(x + i + nthreads), c = __ldcs(x + i + 2 * nthreads), d = __ldcs(x + i + 3 * nthreads);
+    __stcs(z + i, pack4(quant1(a.x, q, lo, hi), quant1(a.y, q, lo, hi), quant1(a.z, q, lo, hi), quant1(a.w, q, lo, hi)));
+    __stcs(z + i + nthreads, pack4(quant1(b.x, q, lo, hi), quant1(b.y, q, lo, hi), quant1(b.z, q, lo, hi), quant1(b.w, q, lo, hi)));
+    __stcs(z + i + 2 * nthreads, pack4(quant1(c.x, q, lo, hi), quant1(c.y, q, lo, hi), quant1(c.z, q, lo, hi), quant1(c.w, q, lo, hi)));
+    __stcs(z + i + 3 * nthreads, pack4(quant1(d.x, q, lo, hi), quant1(d.y, q, lo, hi), quant1(d.z, q, lo, hi), quant1(d.w, q, lo, hi)));
+  }
+  for (; i < n4; i += nthreads) {
+    const float4 a = __ldcs(x + i);
+    __stcs(z + i, pack4(quant1(a.x, q, lo, hi), quant1(a.y, q, lo, hi), quant1(a.z, q, lo, hi), quant1(a.w, q, lo, hi)));
   }
 }
 
@@ -163,17 +168,21 @@ __device__ __forceinline__ float4 deq4(unsigned int w, float q) {
   return r;
 }
 
+// Four bytes in, one float4 out per thread and step (a warp reads 128 contiguous bytes and writes 512),
+// four independent steps in flight.  n4 = number of 4-byte groups.
 template <bool kSigned>
-__global__ void __launch_bounds__(kThreads) dequantize8_vec_kernel(const uint4* __restrict__ z, size_t n16, float q,
+__global__ void __launch_bounds__(kThreads) dequantize8_vec_kernel(const unsigned int* __restrict__ z, size_t n4, float q,
                                                                    float4* __restrict__ r) {
   const size_t nthreads = (size_t)gridDim.x * blockDim.x;
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += nthreads) {
-    uint4 v = __ldcs(z + i);
-    __stcs(r + 4 * i, deq4<kSigned>(v.x, q));
-    __stcs(r + 4 * i + 1, deq4<kSigned>(v.y, q));
-    __stcs(r + 4 * i + 2, deq4<kSigned>(v.z, q));
-    __stcs(r + 4 * i + 3, deq4<kSigned>(v.w, q));
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  for (; i + 3 * nthreads < n4; i += 4 * nthreads) {
+    const unsigned int a = __ldcs(z + i), b = __ldcs(z + i + nthreads), c = __ldcs(z + i + 2 * nthreads), d = __ldcs(z + i + 3 * nthreads);
+    __stcs(r + i, deq4<kSigned>(a, q));
+    __stcs(r + i + nthreads, deq4<kSigned>(b, q));
+    __stcs(r + i + 2 * nthreads, deq4<kSigned>(c, q));
+    __stcs(r + i + 3 * nthreads, deq4<kSigned>(d, q));
   }
+  for (; i < n4; i += nthreads) __stcs(r + i, deq4<kSigned>(__ldcs(z + i), q));
 }
 
 template <typename InT>
@@ -307,6 +316,37 @@ __global__ void __launch_bounds__(256) pool_kernel(const unsigned char* __restri
   }
 }
 
+// Max pooling with 16 channels per thread: 16-byte loads and stores, byte-wise SIMD maximum (exact).
+template <bool kSigned>
+__global__ void __launch_bounds__(256) maxpool16_kernel(const uint4* __restrict__ x, int N, int H, int W, int cg, int kh,
+                                                        int kw, int st_h, int st_w, int pad_h, int pad_w, int P, int Q,
+                                                        uint4* __restrict__ y) {
+  const size_t total = (size_t)N * P * Q * cg;
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += nthreads) {
+    const int c = (int)(i % cg);
+    size_t t = i / cg;
+    const int q = (int)(t % Q);
+    t /= Q;
+    const int p = (int)(t % P);
+    const int n = (int)(t / P);
+    const unsigned int init = kSigned ? 0x80808080u : 0u;
+    uint4 m = make_uint4(init, init, init, init);
+    for (int r = 0; r < kh; ++r) {
+      const int h = p * st_h - pad_h + r;
+      if (h < 0 || h >= H) continue;
+      for (int s = 0; s < kw; ++s) {
+        const int w = q * st_w - pad_w + s;
+        if (w < 0 || w >= W) continue;
+        const uint4 v = __ldg(x + (((size_t)n * H + h) * W + w) * cg + c);
+        if (kSigned) { m.x = __vmaxs4(m.x, v.x); m.y = __vmaxs4(m.y, v.y); m.z = __vmaxs4(m.z, v.z); m.w = __vmaxs4(m.w, v.w); }
+        else { m.x = __vmaxu4(m.x, v.x); m.y = __vmaxu4(m.y, v.y); m.z = __vmaxu4(m.z, v.z); m.w = __vmaxu4(m.w, v.w); }
+      }
+    }
+    y[i] = m;
+  }
+}
+
 int pool_extent(int H, int k, int st, int pad, int ceil_mode) {
   int num = H + 2 * pad - k;
   int o = (ceil_mode ? (num + st - 1) / st : num / st) + 1;
@@ -326,10 +366,17 @@ int launch_pool(const void* x, int t, int N, int H, int W, int C, int kh, int kw
   int P = pool_extent(H, kh, st_h, pad_h, ceil_mode), Q = pool_extent(W, kw, st_w, pad_w, ceil_mode);
   if (P <= 0 || Q <= 0) return fail(Q8_ERR_INVALID_ARG, "pool: empty output");
   float inv = 1.0f / (float)(kh * kw);
+  cudaStream_t s = as_stream(stream);
+  if (!kAvg && C % 16 == 0 && aligned16(x) && aligned16(y)) {
+    const int cg = C / 16;
+    const int grid16 = grid_for((size_t)N * P * Q * cg, 256, 8);
+    if (t == Q8_S8) maxpool16_kernel<true><<<grid16, 256, 0, s>>>(static_cast<const uint4*>(x), N, H, W, cg, kh, kw, st_h, st_w, pad_h, pad_w, P, Q, static_cast<uint4*>(y));
+    else maxpool16_kernel<false><<<grid16, 256, 0, s>>>(static_cast<const uint4*>(x), N, H, W, cg, kh, kw, st_h, st_w, pad_h, pad_w, P, Q, static_cast<uint4*>(y));
+    return check_launch("maxpool16_kernel");
+  }
   bool vec = (C % 4 == 0) && ((reinterpret_cast<uintptr_t>(x) & 3u) == 0) && ((reinterpret_cast<uintptr_t>(y) & 3u) == 0);
   size_t total = (size_t)N * P * Q * (vec ? C / 4 : C);
   int grid = grid_for(total, 256, 8);
-  cudaStream_t s = as_stream(stream);
   const unsigned char* xp = static_cast<const unsigned char*>(x);
   unsigned char* yp = static_cast<unsigned char*>(y);
 #define Q8_POOL(SG, V) pool_kernel<SG, kAvg, V><<<grid, 256, 0, s>>>(xp, N, H, W, C, kh, kw, st_h, st_w, pad_h, pad_w, P, Q, inv, yp)
@@ -405,9 +452,9 @@ int q8_quantize(const float* x, size_t n, float q, int out_type, void* z, void* 
   }
   const int lo = out_type == Q8_U8 ? 0 : -128, hi = out_type == Q8_U8 ? 255 : 127;
   if (aligned16(x) && aligned16(z)) {
-    size_t n16 = n / 16;
-    if (n16) quantize8_vec_kernel<<<grid_for(n16, kThreads, 4), kThreads, 0, s>>>(reinterpret_cast<const float4*>(x), n16, q, lo, hi, static_cast<uint4*>(z));
-    if (n16 * 16 < n) quantize_scalar_kernel<unsigned char><<<1, kThreads, 0, s>>>(x, n16 * 16, n, q, lo, hi, static_cast<unsigned char*>(z));
+    size_t n4 = n / 4;
+    if (n4) quantize8_vec_kernel<<<grid_for(n4, kThreads * 4, 4), kThreads, 0, s>>>(reinterpret_cast<const float4*>(x), n4, q, lo, hi, static_cast<unsigned int*>(z));
+    if (n4 * 4 < n) quantize_scalar_kernel<unsigned char><<<1, kThreads, 0, s>>>(x, n4 * 4, n, q, lo, hi, static_cast<unsigned char*>(z));
   } else {
     quantize_scalar_kernel<unsigned char><<<grid_for(n, kThreads, 8), kThreads, 0, s>>>(x, 0, n, q, lo, hi, static_cast<unsigned char*>(z));
   }
@@ -440,13 +487,13 @@ int q8_dequantize(const void* z, int in_type, size_t n, float q, float* r, void*
   }
   size_t done = 0;
   if (aligned16(z) && aligned16(r)) {
-    size_t n16 = n / 16;
-    if (n16) {
-      int grid = grid_for(n16, kThreads, 4);
-      if (in_type == Q8_S8) dequantize8_vec_kernel<true><<<grid, kThreads, 0, s>>>(static_cast<const uint4*>(z), n16, q, reinterpret_cast<float4*>(r));
-      else dequantize8_vec_kernel<false><<<grid, kThreads, 0, s>>>(static_cast<const uint4*>(z), n16, q, reinterpret_cast<float4*>(r));
+    size_t n4 = n / 4;
+    if (n4) {
+      int grid = grid_for(n4, kThreads * 4, 4);
+      if (in_type == Q8_S8) dequantize8_vec_kernel<true><<<grid, kThreads, 0, s>>>(static_cast<const unsigned int*>(z), n4, q, reinterpret_cast<float4*>(r));
+      else dequantize8_vec_kernel<false><<<grid, kThreads, 0, s>>>(static_cast<const unsigned int*>(z), n4, q, reinterpret_cast<float4*>(r));
     }
-    done = n16 * 16;
+    done = n4 * 4;
   }
   if (done < n) {
     int grid = grid_for(n - done, kThreads, 8);
