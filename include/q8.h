@@ -146,8 +146,12 @@ typedef struct q8_conv_desc {
   int32_t algo;             /* q8_conv_algo */
 } q8_conv_desc;
 
-/* Bytes of device scratch q8_conv2d needs for `d` (0 for most shapes; split-K
- * partial sums otherwise).  Host only. */
+/* Bytes of device scratch with which q8_conv2d runs `d` fastest: 0 for most shapes.  Layers whose
+ * output has too few 128-row tiles to occupy the GPU (small images with long reductions, fully
+ * connected layers) split the reduction R*S*C into parts; every part writes raw int32 partial sums
+ * to the workspace (splits * N*P*Q * K * 4 bytes) and a second kernel adds them up, adds the bias and
+ * applies the epilogue.  Integer addition is exact, so the result does not depend on the split.
+ * Host only. */
 int q8_conv2d_workspace_bytes(const q8_conv_desc* d, size_t* bytes);
 
 /* Which kernel q8_conv2d would pick for `d`: writes Q8_ALGO_UMMA or
@@ -156,8 +160,9 @@ int q8_conv2d_query_algo(const q8_conv_desc* d, int* algo);
 
 /* x: device NHWC (x_type).  w: device KRSC s8.  bias: device s32[K] or NULL.
  * scale: device fp32[scale_count].  residual: device [N,P,Q,K] dense (res_type)
- * or NULL.  y: device, see above.  workspace: device, >= workspace_bytes (may be
- * NULL when 0 are needed); contents undefined afterwards.
+ * or NULL.  y: device, see above.  workspace: device, 16-byte aligned, workspace_bytes long, or NULL.
+ * It is optional: with less than q8_conv2d_workspace_bytes() the layer runs unsplit (same result,
+ * slower for the shapes that would split).  Contents undefined afterwards.
  * Alignment: the tensor-core kernel needs x, w, y, residual 16-byte aligned, C
  * a multiple of 16, and for u8/s8 output y_ldc and y_c_offset multiples of 16;
  * Q8_ALGO_AUTO falls back to the direct kernel otherwise.

@@ -105,6 +105,11 @@ int q8_conv2d_workspace_bytes(const q8_conv_desc* d, size_t* bytes) {
   if (rc != Q8_OK) return rc;
   if (!bytes) return fail(Q8_ERR_INVALID_ARG, "q8_conv2d_workspace_bytes: null pointer");
   *bytes = 0;
+  if (d->algo != Q8_ALGO_DIRECT && d->y_type != Q8_S32) {
+    const long long M = (long long)d->N * P * Q;
+    const int splits = umma_plan_splits(*d, P, Q, M);
+    if (splits > 1) *bytes = (size_t)splits * (size_t)M * (size_t)d->K * sizeof(int32_t);
+  }
   return Q8_OK;
 }
 

@@ -103,6 +103,9 @@ struct UmmaParams {
   int nbuf;                  // 8-bit tile buffers per epilogue group (0: none)
   int m_tiles, n_tiles;
   FastDiv fd_ntiles, fd_perimg, fd_qtiles, fd_pq, fd_q;  // n_tiles, p_tiles*q_tiles, q_tiles, P*Q, Q
+  int splits, kps;           // split-K: work item = (tile, split), each split runs kps of the k_iters iterations
+  FastDiv fd_splits, fd_cblocks, fd_s;  // splits, c_blocks, S
+  long long split_stride;    // elements between the partial results of two splits in the workspace
   unsigned int idesc;        // tcgen05 instruction descriptor
   unsigned int desc_hi;      // high word of the shared-memory matrix descriptors
   unsigned int a_sub_bytes;  // plain/im2col: one 128 x bk block; halo: bytes of one patch load
@@ -129,15 +132,22 @@ struct UmmaParams {
 // n tiles of one m tile adjacent (they share the A operand through L2), and for halo tiles
 // m tile -> (image, tile row, tile column).  Only additions after init().
 struct TileIter {
-  int tile, step;
+  int tile, step;    // work item index (tile * splits + split) and its stride
+  int sp, d_sp;      // split-K part of the work item
   int mt, nt;        // m tile, n tile
   int img, pt, qt;   // halo: image, tile row, tile column
   int d_mt, d_nt, d_img, d_pt, d_qt;
 
   __device__ __forceinline__ void init(const UmmaParams& p, int first, int step_) {
     tile = first; step = step_;
-    mt = p.fd_ntiles.div(first); nt = first - mt * p.n_tiles;
-    d_mt = p.fd_ntiles.div(step_); d_nt = step_ - d_mt * p.n_tiles;
+    int t0 = first, dt = step_;  // output tile and its stride
+    sp = d_sp = 0;
+    if (p.splits > 1) {
+      t0 = p.fd_splits.div(first); sp = first - t0 * p.splits;
+      dt = p.fd_splits.div(step_); d_sp = step_ - dt * p.splits;
+    }
+    mt = p.fd_ntiles.div(t0); nt = t0 - mt * p.n_tiles;
+    d_mt = p.fd_ntiles.div(dt); d_nt = dt - d_mt * p.n_tiles;
     img = pt = qt = d_img = d_pt = d_qt = 0;
     if (p.a_mode == kAHalo) {
       const int per_img = p.p_tiles * p.q_tiles;
@@ -152,7 +162,9 @@ struct TileIter {
   __device__ __forceinline__ void next(const UmmaParams& p) {
     tile += step;
     int carry = 0;
-    nt += d_nt;
+    sp += d_sp;
+    if (sp >= p.splits) { sp -= p.splits; carry = 1; }
+    nt += d_nt + carry; carry = 0;
     if (nt >= p.n_tiles) { nt -= p.n_tiles; carry = 1; }
     mt += d_mt + carry;
     if (p.a_mode == kAHalo) {
@@ -360,6 +372,7 @@ struct EpiTile {
   const float* s_scale;    // smem, k_pad entries
   unsigned char* buf;      // this tile's 8-bit buffer (residual in, output out) or nullptr
   long long m;             // output pixel (row of the [M][Cout] result) of this thread
+  long long y_off;         // element offset of this work item's output (split-K partial results), else 0
   int srow;                // row of this thread's pixel inside the 8-bit tile buffer
   int n0;                  // first channel of the tile
   bool row_ok;             // the pixel exists (inside the image and below M)
@@ -386,7 +399,7 @@ __device__ __forceinline__ void epilogue_chunk(const UmmaParams& p, const EpiTil
   if (kOut == Q8_S32) {
     if (t.row_ok && nb < p.K) {
       const int valid = min(16, p.K - nb);
-      int* yp = static_cast<int*>(p.y) + (size_t)t.m * p.ldc + p.c_off + nb;
+      int* yp = static_cast<int*>(p.y) + t.y_off + (size_t)t.m * p.ldc + p.c_off + nb;
       if (p.y_vec && valid == 16) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) reinterpret_cast<int4*>(yp)[j] = make_int4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
@@ -539,7 +552,7 @@ __device__ __forceinline__ bool mma_role(const UmmaParams& p, const MmaRoleArgs&
   const uint64_t bres_d0 = hi | ((r.base >> 4) & 0x3fffu);
   const uint32_t stage16 = p.a_stage_bytes >> 4, asub16 = p.a_sub_bytes >> 4, bsub16 = p.b_sub_bytes >> 4, btile16 = p.b_tile_bytes >> 4;
   const uint32_t idesc = p.idesc;
-  const int taps = p.taps, c_blocks = p.c_blocks, k_iters = p.k_iters, kb = p.kb;
+  const int taps = p.taps, c_blocks = p.c_blocks, k_iters = p.kps, kb = p.kb;  // k iterations of one work item
   const bool halo = p.a_mode == kAHalo, ring = p.b_mode == kBRing, b_in_stage = p.b_mode == kBStage;
   // ring positions of tile lt = who, and how far the other lanes' tiles move them between two of ours
   const uint32_t spt = halo ? (uint32_t)c_blocks : (uint32_t)((k_iters + kb - 1) / kb);  // A stages per tile
@@ -599,6 +612,12 @@ __device__ __forceinline__ bool mma_role(const UmmaParams& p, const MmaRoleArgs&
     } else {
       uint64_t bres_tap = bres_nt, bres = bres_nt;  // iterations run over taps with the channel blocks innermost
       int cb = 0;
+      if (p.splits > 1) {
+        const int it0 = ti.sp * k_iters, tap0 = p.fd_cblocks.div(it0);
+        cb = it0 - tap0 * c_blocks;
+        bres_tap += (uint32_t)tap0 * btile16;
+        bres = bres_tap + (uint32_t)(cb * taps) * btile16;
+      }
       const uint32_t b_off16 = (uint32_t)kb * asub16;
       for (int it = 0; it < k_iters;) {
         const int nsub = min(kb, k_iters - it);
@@ -665,7 +684,7 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
   int* const s_bias = reinterpret_cast<int*>(base_ptr + p.off_chan);
   float* const s_scale = reinterpret_cast<float*>(base_ptr + p.off_chan) + p.k_pad;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int total_tiles = p.m_tiles * p.n_tiles;
+  const int total_tiles = p.m_tiles * p.n_tiles * p.splits;  // work items
   const int slots = G * p.nbuf;
 
   // Prologue.  Each control lane initialises the barriers it owns.  Warp 0 only signals the
@@ -774,8 +793,16 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
           w0 = qc * p.stride_w - p.pad_w;
         }
         int c = 0, tap = 0, s = 0, off_w = 0, off_h = 0;
-        for (int it = 0; it < p.k_iters;) {
-          const int nsub = min(p.kb, p.k_iters - it);
+        if (p.splits > 1) {  // this split starts at iteration sp * kps = (tap, channel block)
+          const int it0 = ti.sp * p.kps;
+          tap = p.fd_cblocks.div(it0);
+          c = (it0 - tap * p.c_blocks) * p.bk;
+          const int r0 = p.fd_s.div(tap);
+          s = tap - r0 * p.S;
+          off_w = s * p.dil_w; off_h = r0 * p.dil_h;
+        }
+        for (int it = 0; it < p.kps;) {
+          const int nsub = min(p.kb, p.kps - it);
           if (!mbar_wait(aempty0 + stage * 8u, phase ^ 1u, abortp)) { ok = false; break; }
           const uint32_t bar = afull0 + stage * 8u;
           mbar_arrive_expect_tx(bar, (uint32_t)nsub * sub_tx);
@@ -930,6 +957,7 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       }
       tcgen05_fence_after();
       t.n0 = ti.nt * p.bn;
+      t.y_off = (long long)ti.sp * p.split_stride;
       if (p.a_mode == kAHalo) {
         const int pr = ti.pt * p.th + pp, qc = ti.qt * p.tw + qq;
         t.row_ok = t.smem_ok && pr < p.P && qc < p.Q;
@@ -1144,7 +1172,52 @@ bool umma_shape_eligible(const q8_conv_desc& d, const char** why) {
   return true;
 }
 
+// Split-K plan: layers whose output tiles cannot occupy half of the SMs split the reduction over
+// (tap, channel block) iterations into `splits` equal parts; every part writes raw int32 partial sums
+// (integer addition is associative, so the result stays bit exact).  Only the plain and im2col operand
+// paths split.  Returns 1 when the layer runs unsplit.
+int umma_plan_splits(const q8_conv_desc& d, int P, int Q, long long M) {
+  if (!umma_shape_eligible(d, nullptr)) return 1;
+  HaloTile ht;
+  if (!is_plain(d) && choose_halo_tile(d, P, Q, &ht)) return 1;
+  const int BK = pick_bk(d.C), BN = pick_bn(d.K, d.R * d.S * d.C);
+  const long long tiles = ((M + kBM - 1) / kBM) * ((d.K + BN - 1) / BN);
+  const int k_iters = d.R * d.S * ((d.C + BK - 1) / BK);
+  const int sms = sm_count();
+  if (tiles * 2 > sms) return 1;
+  int best = 1;
+  for (int sp = 2; sp <= 16 && tiles * sp <= sms; ++sp)
+    if (k_iters % sp == 0 && k_iters / sp >= 4) best = sp;
+  return best;
+}
+
+namespace {
+int launch_conv_umma_impl(const ConvArgs& a, int splits);
+}
+
 int launch_conv_umma(const ConvArgs& a) {
+  const q8_conv_desc& d = a.d;
+  const int splits = umma_plan_splits(d, a.P, a.Q, a.M);
+  const size_t need = splits > 1 ? (size_t)splits * (size_t)a.M * d.K * sizeof(int) : 0;
+  if (splits > 1 && d.y_type != Q8_S32 && a.workspace && a.workspace_bytes >= need && aligned16(a.workspace)) {
+    // pass 1: raw partial accumulators of every split into the workspace; pass 2: sum, bias, epilogue
+    ConvArgs part = a;
+    part.d.y_type = Q8_S32;
+    part.d.relu = 0;
+    part.y = a.workspace;
+    part.ldc = d.K;
+    part.c_off = 0;
+    part.bias = nullptr;
+    part.residual = nullptr;
+    int rc = launch_conv_umma_impl(part, splits);
+    if (rc != Q8_OK) return rc;
+    return launch_splitk_reduce(a, splits);
+  }
+  return launch_conv_umma_impl(a, 1);
+}
+
+namespace {
+int launch_conv_umma_impl(const ConvArgs& a, int splits) {
   const q8_conv_desc& d = a.d;
   DriverFns& fn = driver_fns();
   if (!fn.tiled || !fn.im2col) return fail(Q8_ERR_CUDA, "conv_umma: cuTensorMapEncode* entry points not available");
@@ -1169,6 +1242,12 @@ int launch_conv_umma(const ConvArgs& a) {
   p.c_blocks = (d.C + BK - 1) / BK;
   p.C_pad = p.c_blocks * BK;
   p.k_iters = p.taps * p.c_blocks;
+  p.splits = splits;
+  p.kps = p.k_iters / splits;  // the plan only splits evenly
+  p.fd_splits = make_fastdiv(splits);
+  p.fd_cblocks = make_fastdiv(p.c_blocks);
+  p.fd_s = make_fastdiv(d.S);
+  p.split_stride = (long long)a.M * a.ldc;
   // 8-bit tile buffers: panels as wide as the largest power of two dividing BN, at most one swizzle span
   int pw = BN & -BN;
   if (pw > 128) pw = 128;
@@ -1224,7 +1303,7 @@ int launch_conv_umma(const ConvArgs& a) {
     const unsigned unit = p.a_sub_bytes + (p.b_mode == kBStage ? p.b_sub_bytes : 0u);
     int kb = (int)(40u * 1024u / unit);
     if (kb < 1) kb = 1;
-    if (kb > p.k_iters) kb = p.k_iters;
+    if (kb > p.kps) kb = p.kps;
     p.kb = tune_env("Q8_KB", kb);
     p.a_stage_bytes = (unsigned)p.kb * unit;
     min_pipe = 2u * p.a_stage_bytes;
@@ -1351,11 +1430,12 @@ int launch_conv_umma(const ConvArgs& a) {
   p.y_vec = out8 ? 1 : (aligned16(a.y) && a.ldc % 4 == 0 && a.c_off % 4 == 0);
   p.status = status;
 
-  const long long tiles = (long long)p.m_tiles * p.n_tiles;
+  const long long tiles = (long long)p.m_tiles * p.n_tiles * splits;  // work items
   int grid = (int)(tiles < sm_count() ? tiles : sm_count());
   grid = tune_env("Q8_GRID", grid);
   if (G == 2) return launch_groups<2>(tmA, tmB, tmRes, tmY, p, dyn, grid, a.stream);
   return launch_groups<4>(tmA, tmB, tmRes, tmY, p, dyn, grid, a.stream);
 }
+}  // namespace
 
 }  // namespace q8

@@ -49,6 +49,11 @@ struct ConvArgs {
 // Eligibility of the tensor-core kernel for a descriptor (pointer alignment checked at launch).
 bool umma_shape_eligible(const q8_conv_desc& d, const char** why);
 int launch_conv_umma(const ConvArgs& a);
+// Number of split-K parts the tensor-core kernel uses for this layer when it is given a workspace of
+// splits * M * K int32 (1: none).  Host only.
+int umma_plan_splits(const q8_conv_desc& d, int P, int Q, long long M);
+// Sums the split-K partial accumulators in a.workspace, adds the bias and applies the epilogue of `a`.
+int launch_splitk_reduce(const ConvArgs& a, int splits);
 int launch_conv_direct(const ConvArgs& a);
 
 }  // namespace q8

@@ -137,3 +137,39 @@ def test_forced_umma_rejects_ineligible_shapes(q8):
     with pytest.raises(q8.Q8Error) as e:
         q8.q8_conv2d(d, x, w, None, torch.ones(1, device="cuda"))
     assert e.value.code == 2
+
+
+SPLITK_CASES = [
+    # name, N,H,W,C,K,R,S,stride,pad, y type, residual, relu
+    ("fc_c2048_k1000_f32", 64, 1, 1, 2048, 1000, 1, 1, 1, 0, F32, None, False),
+    ("3x3_7x7_c512_k512_res", 8, 7, 7, 512, 512, 3, 3, 1, 1, U8, "u8", True),
+    ("1x1_c2048_k512", 8, 7, 7, 2048, 512, 1, 1, 1, 0, U8, None, True),
+    ("3x3s2_c256_k256_s8", 4, 15, 15, 256, 256, 3, 3, 2, 1, S8, None, False),
+    ("1x1_c1024_k24_slice", 2, 10, 10, 1024, 24, 1, 1, 1, 0, F32, None, True),
+]
+
+
+@pytest.mark.parametrize("case", SPLITK_CASES, ids=[c[0] for c in SPLITK_CASES])
+def test_split_k_matches_oracle_and_unsplit(q8, case):
+    """Layers with few output tiles split the reduction when given a workspace; the result must not change."""
+    name, N, H, W, C, K, R, S, st, pad, ytype, res, relu = case
+    g = np.random.default_rng(sum(map(ord, name)))
+    x = g.integers(0, 256, (N, H, W, C), dtype=np.uint8)
+    w = g.integers(-128, 128, (K, R, S, C)).astype(np.int8)
+    bias = g.integers(-5000, 5000, K).astype(np.int32)
+    acc = o.conv_acc(x, w, bias, (st, st), (pad, pad), (1, 1), threads=8)
+    P, Q = acc.shape[1:3]
+    resid = g.integers(0, 256, (N, P, Q, K), dtype=np.uint8) if res else None
+    scale = np.float32(100.0 / max(1, np.abs(acc).max()))
+    rs = 0.37 if resid is not None else 0.0
+    want = o.epilogue(acc, scale, resid, rs, relu, OT[ytype])
+    d = q8.make_conv_desc(N, H, W, C, K, R, S, (st, st), (pad, pad), (1, 1), U8, U8, ytype, relu)
+    nbytes = q8.q8_conv2d_workspace_bytes(d)
+    assert nbytes > 0, "this shape is expected to split"
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    args = (_cuda(x), _cuda(w), _cuda(bias), torch.tensor([scale], device="cuda"), _cuda(resid) if res else None, rs)
+    y_split = q8.q8_conv2d(d, *args, workspace=ws)
+    y_plain = q8.q8_conv2d(d, *args)
+    q8.q8_read_status()
+    assert np.array_equal(_bits(y_split.cpu().numpy()), _bits(want))
+    assert np.array_equal(_bits(y_plain.cpu().numpy()), _bits(want))
