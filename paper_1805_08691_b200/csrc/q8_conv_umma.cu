@@ -1109,7 +1109,11 @@ bool choose_halo_tile(const q8_conv_desc& d, int P, int Q, HaloTile* out) {
     const double score = eff / (1.0 + 0.04 * halo);
     if (score > best_score) { best_score = score; best = {tw, th, twb, hb, eff}; }
   }
-  if (best.eff < 0.5) return false;
+  // Tiny images waste accumulator rows (a 7x7 image fills 49 of 128 rows).  Where the im2col path is
+  // open it is the better choice for them (it can split the reduction); tensors below its size limit
+  // still take halo tiles rather than leave the tensor cores.
+  const bool im2col_closed = (long long)d.N * d.H * d.W * d.C < 131072;
+  if (best.eff < (im2col_closed ? 0.2 : 0.5)) return false;
   *out = best;
   return true;
 }
@@ -1172,7 +1176,7 @@ bool umma_shape_eligible(const q8_conv_desc& d, const char** why) {
   return true;
 }
 
-// Split-K plan: layers whose output tiles cannot occupy half of the SMs split the reduction over
+// Split-K plan: layers whose output tiles cannot occupy a quarter of the SMs split the reduction over
 // (tap, channel block) iterations into `splits` equal parts; every part writes raw int32 partial sums
 // (integer addition is associative, so the result stays bit exact).  Only the plain and im2col operand
 // paths split.  Returns 1 when the layer runs unsplit.
@@ -1184,7 +1188,8 @@ int umma_plan_splits(const q8_conv_desc& d, int P, int Q, long long M) {
   const long long tiles = ((M + kBM - 1) / kBM) * ((d.K + BN - 1) / BN);
   const int k_iters = d.R * d.S * ((d.C + BK - 1) / BK);
   const int sms = sm_count();
-  if (tiles * 2 > sms) return 1;
+  // a split costs a second (small) kernel and the partial-sum traffic: it pays once most SMs would idle
+  if (tiles * 4 > sms) return 1;
   int best = 1;
   for (int sp = 2; sp <= 16 && tiles * sp <= sms; ++sp)
     if (k_iters % sp == 0 && k_iters / sp >= 4) best = sp;
