@@ -173,6 +173,26 @@ int q8_conv2d(const q8_conv_desc* d, const void* x, const int8_t* w, const int32
               const float* scale, const void* residual, float residual_scale, void* y,
               void* workspace, size_t workspace_bytes, void* stream);
 
+/* q8_conv2d for callers that cannot allocate device memory (the paper has no counterpart; this is a
+ * property of the library, not of the method).  Meant for hosts where every byte of device memory was
+ * handed out before this library is called, or where cudaMalloc is off limits because it stalls the
+ * device: the scratch of the split reduction (see q8_conv2d_workspace_bytes) is a fixed array of
+ * q8_static_workspace_bytes() = 16 MiB inside the library image instead of a caller buffer.
+ *  - Every GPU on which the library is loaded holds that array until the process exits.
+ *  - A layer that would need more scratch is refused with Q8_ERR_WORKSPACE (nothing is launched);
+ *    q8_conv2d with workspace = NULL still runs it, unsplit.  Layers that need none just run.
+ *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that
+ *    device current).  Make that first call outside any stream capture.
+ *  - All calls share the one array and it keeps the previous call's contents.  Nothing needs clearing
+ *    (each call writes every partial sum before reading it), but two calls whose kernels overlap on the
+ *    GPU (different streams, or threads) race on it: serialise them.
+ *  - No cudaMalloc, cudaFree or other allocating call is made.
+ * Arguments, result and errors otherwise as q8_conv2d. */
+size_t q8_static_workspace_bytes(void);
+int q8_conv2d_static_workspace(const q8_conv_desc* d, const void* x, const int8_t* w, const int32_t* bias,
+                               const float* scale, const void* residual, float residual_scale, void* y,
+                               void* stream);
+
 /* ------------------------------------------------------------------------
  * Channel concatenation of quantized branches under one factor (the paper
  * gives no rule; the caller passes the shared factor, normally the largest

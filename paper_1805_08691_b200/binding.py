@@ -20,7 +20,8 @@ STATUS_NAMES = {0: "Q8_OK", 1: "Q8_ERR_INVALID_ARG", 2: "Q8_ERR_UNSUPPORTED", 3:
 TORCH_DTYPES = {Q8_U8: torch.uint8, Q8_S8: torch.int8, Q8_S32: torch.int32, Q8_F32: torch.float32}
 EXPORTS = ["q8_version", "q8_last_error", "q8_read_status", "q8_calibrate_maxabs", "q8_factor", "q8_requant_scale",
            "q8_bias_factor", "q8_quantize", "q8_quantize_pad_channels", "q8_dequantize", "q8_fold_bn",
-           "q8_conv2d_workspace_bytes", "q8_conv2d_query_algo", "q8_conv2d", "q8_concat", "q8_pool_out_extent",
+           "q8_conv2d_workspace_bytes", "q8_conv2d_query_algo", "q8_conv2d", "q8_static_workspace_bytes",
+           "q8_conv2d_static_workspace", "q8_concat", "q8_pool_out_extent",
            "q8_maxpool2d", "q8_avgpool2d"]
 
 
@@ -64,12 +65,15 @@ lib.q8_fold_bn.argtypes = [_vp] * 6 + [C.c_double, _i, _sz, _vp, _vp, _vp]
 lib.q8_conv2d_workspace_bytes.argtypes = [C.POINTER(q8_conv_desc), C.POINTER(_sz)]
 lib.q8_conv2d_query_algo.argtypes = [C.POINTER(q8_conv_desc), _ip]
 lib.q8_conv2d.argtypes = [C.POINTER(q8_conv_desc), _vp, _vp, _vp, _vp, _vp, _f, _vp, _vp, _sz, _vp]
+lib.q8_static_workspace_bytes.argtypes = []
+lib.q8_conv2d_static_workspace.argtypes = [C.POINTER(q8_conv_desc), _vp, _vp, _vp, _vp, _vp, _f, _vp, _vp]
 lib.q8_concat.argtypes = [_i, C.POINTER(_vp), _ip, _fp, _f, _i, _sz, _vp, _vp]
 lib.q8_pool_out_extent.argtypes = [_i] * 5 + [_ip]
 lib.q8_maxpool2d.argtypes = [_vp, _i] + [_i] * 11 + [_vp, _vp]
 lib.q8_avgpool2d.argtypes = [_vp, _i] + [_i] * 11 + [_vp, _vp]
 for _n in EXPORTS[2:]:
     getattr(lib, _n).restype = C.c_int
+lib.q8_static_workspace_bytes.restype = C.c_size_t
 
 
 def _check(rc):
@@ -193,6 +197,21 @@ def q8_conv2d(d, x, w, bias, scale, residual=None, residual_scale=0.0, y=None, w
     _check(lib.q8_conv2d(C.byref(d), _dev(x, "x"), _dev(w, "w"), _dev(bias, "bias"), _dev(scale, "scale"),
                          _dev(residual, "residual"), residual_scale, _dev(y, "y"), _dev(workspace, "workspace"),
                          ws_bytes, _stream()))
+    return y
+
+
+def q8_static_workspace_bytes():
+    return int(lib.q8_static_workspace_bytes())
+
+
+def q8_conv2d_static_workspace(d, x, w, bias, scale, residual=None, residual_scale=0.0, y=None):
+    """q8_conv2d with the library's built-in scratch array instead of a caller workspace; allocates nothing
+    (pass `y`; it is only created here, by torch, when omitted)."""
+    if y is None:
+        P, Q = conv_out_shape(d)
+        y = torch.empty((d.N, P, Q, d.y_ldc or d.K), dtype=TORCH_DTYPES[d.y_type], device=x.device)
+    _check(lib.q8_conv2d_static_workspace(C.byref(d), _dev(x, "x"), _dev(w, "w"), _dev(bias, "bias"), _dev(scale, "scale"),
+                                          _dev(residual, "residual"), residual_scale, _dev(y, "y"), _stream()))
     return y
 
 
