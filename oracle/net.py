@@ -44,3 +44,79 @@ def calib_maxima(samples_per_batch):
         for k, v in batch.items():
             m[k] = o.maxabs(v, init=m.get(k, 0.0))
     return m
+
+
+# --------------------------------------------------------------------------------------------------
+# Whole networks (layer lists from workloads.nets), oracle calls only.
+#
+# Factor rules (calibration paragraph of Sec. "8-bit Low Precision Inference", Eq. arithmetics):
+#   network input (signed)            : s8, q = max|x| / 127
+#   conv + ReLU                       : u8, q = max / 255
+#   conv without ReLU                 : s8, q = max|y| / 127
+#   conv + residual sum + ReLU        : u8, q = max(max|conv|, max|residual|) / 255   ("+" rule on a common footing)
+#   dequantized output (logits, heads): fp32, the accumulator is only multiplied by q_x * q_w
+#   pooling                           : type and factor of its input
+#   concat                            : largest branch factor, branches re-expressed at it
+# A 3-channel input is zero padded to 16 channels (weights too): zeros are exact under a symmetric quantizer.
+# --------------------------------------------------------------------------------------------------
+def _pad_c(a, c_pad):
+    if a.shape[-1] == c_pad:
+        return a
+    out = np.zeros(a.shape[:-1] + (c_pad,), dtype=a.dtype)
+    out[..., :a.shape[-1]] = a
+    return out
+
+
+def network_prepare(layers, folded, maxima):
+    """Returns {layer name: dict} with the quantized parameters and the (type, factor) of every tensor."""
+    info = {"input": (o.S8, o.factor(maxima["input"], 7))}
+    prep = {}
+    for L in layers:
+        t_in, q_in = info[L.src[0]]
+        if L.op == "conv":
+            w, b = folded[L.name]
+            c_pad = -(-w.shape[-1] // 16) * 16
+            q_w = o.factor(o.maxabs(w), 7)
+            w_q = _pad_c(o.quantize(w, q_w, o.S8), c_pad)
+            b_q = o.quantize(b, o.bias_factor(q_in, q_w), o.S32)
+            d = dict(w_q=w_q, b_q=b_q, q_w=q_w, res_scale=0.0, c_pad=c_pad)
+            if L.f32_out:
+                d.update(y_type=o.F32, q_y=1.0)
+            elif L.residual is not None:
+                q_y = o.factor(max(maxima[L.name + ":pre"], maxima[L.residual]), 8)
+                d.update(y_type=o.U8, q_y=q_y, res_scale=o.requant_scale(info[L.residual][1], 1.0, q_y))
+            elif L.conv.relu:
+                d.update(y_type=o.U8, q_y=o.factor(maxima[L.name], 8))
+            else:
+                d.update(y_type=o.S8, q_y=o.factor(maxima[L.name], 7))
+            d["scale"] = o.requant_scale(q_in, q_w, d["q_y"])
+            prep[L.name] = d
+            info[L.name] = (d["y_type"], d["q_y"])
+        elif L.op in ("maxpool", "avgpool"):
+            info[L.name] = (t_in, q_in)
+        elif L.op == "concat":
+            info[L.name] = (t_in, max(info[s][1] for s in L.src))
+        else:
+            raise ValueError(L.op)
+    return prep, info
+
+
+def network_forward(layers, prep, info, x_f32, threads=1):
+    """Quantized run; returns every tensor (quantized payloads, fp32 for dequantized outputs)."""
+    first = next(L for L in layers if L.op == "conv")
+    xq = o.quantize(x_f32, info["input"][1], o.S8)
+    out = {"input": _pad_c(xq, prep[first.name]["c_pad"])}
+    for L in layers:
+        x = out[L.src[0]]
+        if L.op == "conv":
+            d, sp = prep[L.name], L.conv
+            res = out[L.residual] if L.residual is not None else None
+            out[L.name] = o.conv2d(x, d["w_q"], d["b_q"], d["scale"], sp.stride, sp.pad, sp.dil, res, d["res_scale"],
+                                   sp.relu, d["y_type"], threads=threads)
+        elif L.op == "maxpool":
+            out[L.name] = o.pool(x, "max", L.k, L.stride, L.pad, L.ceil_mode)
+        elif L.op == "avgpool":
+            out[L.name] = o.pool(x, "avg", L.k, L.stride, L.pad, L.ceil_mode)
+        elif L.op == "concat":
+            out[L.name] = o.concat([out[s] for s in L.src], [info[s][1] for s in L.src], info[L.name][1])
+    return out

@@ -1,0 +1,85 @@
+"""Whole networks: the library's quantized run must equal the oracle's bit for bit, layer by layer.
+
+Both sides start from the same seeded FP32 parameters and the same FP32 calibration samples (one FP32 run
+on the GPU shared by both), then fold BN, derive factors, quantize and run on their own.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle as o
+import workloads as wl
+from oracle import net as oracle_net
+from workloads import nets
+
+pytestmark = pytest.mark.gpu
+
+
+def _cuda(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def _run_both(q8, layers, hw, batch, calib_batches, seed, check_layers=None):
+    from paper_1805_08691_b200 import network, pipeline
+    # fold BN on both sides, must agree bit for bit
+    folded_o, folded_g = {}, {}
+    for L in layers:
+        if L.op != "conv":
+            continue
+        sp = L.conv
+        if sp.bn:
+            wo, bo = o.fold_bn(sp.w, sp.b, sp.gamma, sp.beta, sp.mean, sp.var, 1e-5)
+            wg, bg = q8.q8_fold_bn(_cuda(sp.w), _cuda(sp.b) if sp.b is not None else None, _cuda(sp.gamma), _cuda(sp.beta),
+                                   _cuda(sp.mean), _cuda(sp.var), 1e-5)
+            assert np.array_equal(wg.cpu().numpy(), wo) and np.array_equal(bg.cpu().numpy(), bo)
+        else:
+            wo, bo = sp.w, (sp.b if sp.b is not None else np.zeros(sp.K, np.float32))
+            wg, bg = _cuda(wo), _cuda(bo)
+        folded_o[L.name], folded_g[L.name] = (wo, bo), (wg, bg)
+    # calibration: FP32 run on seeded batches, running max-abs on both sides
+    names = None
+    cal = None
+    max_o = {}
+    for i in range(calib_batches):
+        acts = nets.fp32_forward(layers, nets.images(seed + 10 + i, batch, hw), folded_o, device="cuda")
+        if cal is None:
+            names = sorted(acts)
+            cal = pipeline.Calibrator(names)
+        for k in names:
+            cal.observe(k, _cuda(acts[k]))
+            max_o[k] = o.maxabs(acts[k], init=max_o.get(k, 0.0))
+    max_g = cal.maxima()
+    assert max_g == max_o
+    # prepare and run
+    x = nets.images(seed + 1, batch, hw)
+    prep, info = oracle_net.network_prepare(layers, folded_o, max_o)
+    want = oracle_net.network_forward(layers, prep, info, x, threads=batch)
+    net = network.QuantNetwork(layers, folded_g, max_g, x.shape)
+    got = net.forward(_cuda(x))
+    q8.q8_read_status()
+    for L in layers:
+        if check_layers is not None and L.name not in check_layers:
+            continue
+        a, e = got[L.name].cpu().numpy(), want[L.name]
+        if a.dtype == np.float32:
+            a, e = a.view(np.uint32), e.view(np.uint32)
+        assert a.shape == e.shape and np.array_equal(a, e), L.name
+        assert net.info[L.name][1] == info[L.name][1], L.name
+    ref = nets.fp32_forward(layers, x, folded_o, device="cuda")
+    return got, want, ref, net
+
+
+def test_bottleneck_stack_every_layer(q8):
+    layers = nets.bottleneck_stack(C=64, blocks=2)
+    _run_both(q8, layers, hw=32, batch=3, calib_batches=2, seed=3100)
+
+
+def test_resnet50_logits_bit_exact_and_close_to_fp32(q8):
+    """Config 3 at a batch the oracle finishes in seconds: all 54 affine layers, pools, dequantized logits."""
+    layers = nets.resnet50()
+    assert nets.macs(layers, 224) == 3857973248  # 3.858 GMAC per image
+    got, want, ref, net = _run_both(q8, layers, hw=224, batch=2, calib_batches=2, seed=3000)
+    logits, fp32 = got["fc1000"].cpu().numpy().reshape(2, -1), ref["fc1000"].reshape(2, -1)
+    rel = float(np.linalg.norm(logits - fp32) / np.linalg.norm(fp32))
+    print(f"ResNet-50 int8 vs FP32 logits: relative L2 error {rel:.4f}")
+    assert rel < 0.5
