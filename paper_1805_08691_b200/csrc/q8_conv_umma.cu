@@ -96,7 +96,9 @@ struct UmmaParams {
   int bn, bk, ksteps;        // tile width (multiple of 16), K bytes per block (32/64/128), bk / 32
   int a_mode, b_mode;
   int k_iters, kb;           // plain/im2col: taps * c_blocks (tap, block) iterations, kb of them per A stage
-  int tw, th, twb, hb;       // halo: tile and patch extents in pixels
+  int tw, th, twb, hb;       // halo: tile and patch extents in pixels (pixel pairs along W when halo_sw == 2)
+  int halo_sw, halo_e, c_true;  // halo: stride along W (1 or 2), parity of pad_w, channels per input pixel
+  unsigned int tap_shift16[kMaxTaps];  // halo: descriptor start offset of every tap, in 16-byte units
   int p_tiles, q_tiles;      // halo: tiles per image column / row
   int stages, b_stages;      // A stages, weight-ring stages
   int nacc, acc_stride, tmem_cols;  // TMEM accumulators, columns between them, allocation (power of two)
@@ -720,11 +722,7 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       tmem_alloc(smem_u32(&tmem_holder), (uint32_t)p.tmem_cols);
       tmem_relinquish();
     }
-    if (p.a_mode == kAHalo && threadIdx.x >= 32 && threadIdx.x - 32 < p.taps) {
-      const int tap = threadIdx.x - 32;
-      const int r = tap / p.S, s = tap - r * p.S;
-      tap_shift16[tap] = (uint32_t)((r * p.dil_h * p.twb + s * p.dil_w) * p.bk) >> 4;
-    }
+    if (p.a_mode == kAHalo && threadIdx.x >= 32 && threadIdx.x - 32 < p.taps) tap_shift16[threadIdx.x - 32] = p.tap_shift16[threadIdx.x - 32];
     // bias and scale of every channel, once per CTA (zero beyond Cout; one scale replicated if per tensor)
     for (int i = threadIdx.x - 32; i < p.k_pad; i += nthreads - 32) {
       s_bias[i] = (p.bias && i < p.K) ? p.bias[i] : 0;
@@ -754,12 +752,20 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       const uint32_t bar = smem_u32(&bres_full);
       mbar_arrive_expect_tx(bar, (uint32_t)(p.n_tiles * p.c_blocks * p.taps) * p.b_tile_bytes);
       uint32_t dst = base;
-      for (int nt = 0; nt < p.n_tiles; ++nt)
-        for (int c = 0; c < p.C_pad; c += p.bk, dst += (uint32_t)p.taps * p.b_tile_bytes) tma_load_3d(dst, &tmB, bar, c, nt * p.bn, 0);
+      if (p.a_mode == kAHalo && p.halo_sw == 2) {
+        // pixel-pair taps: tap t' of a filter row covers s = 2t' - e and 2t' - e + 1, whose weights are 2C
+        // contiguous bytes of the (s, c) axis; a start left of s = 0 is zero filled.  One load per t' brings
+        // all R filter rows: tile order (t', r).
+        for (int nt = 0; nt < p.n_tiles; ++nt)
+          for (int t = 0; t < p.S; ++t, dst += (uint32_t)p.R * p.b_tile_bytes) tma_load_3d(dst, &tmB, bar, (2 * t - p.halo_e) * p.c_true, nt * p.bn, 0);
+      } else {
+        for (int nt = 0; nt < p.n_tiles; ++nt)
+          for (int c = 0; c < p.C_pad; c += p.bk, dst += (uint32_t)p.taps * p.b_tile_bytes) tma_load_3d(dst, &tmB, bar, c, nt * p.bn, 0);
+      }
     }
     if (p.a_mode == kAHalo) {
       for (; ti.tile < total_tiles && ok; ti.next(p)) {
-        const int n0 = ti.nt * p.bn, q0 = ti.qt * p.tw - p.pad_w, p0 = ti.pt * p.th - p.pad_h;
+        const int n0 = ti.nt * p.bn, q0 = ti.qt * p.tw - p.pad_w, p0 = ti.pt * p.th * p.stride_h - p.pad_h;
         for (int c = 0; c < p.C_pad && ok; c += p.bk) {
           if (!mbar_wait(aempty0 + stage * 8u, phase ^ 1u, abortp)) { ok = false; break; }
           const uint32_t bar = afull0 + stage * 8u;
@@ -1087,27 +1093,45 @@ int tune_env(const char* name, int dflt) {
 struct HaloTile {
   int tw, th, twb, hb;
   double eff;  // useful output pixels per computed accumulator row
+  int sw;      // stride along W: 1, or 2 = the input is read as pixel pairs [N, H, W/2, 2C]
+  int s_eff;   // filter taps along W in that view
+  int pad_w_eff, e;  // left padding in that view; parity of pad_w
 };
 
+// Stride 2 along W needs no data movement: with W even, NHWC memory is also a tensor of pixel pairs with 2C
+// channels, and output column q reads pairs q + t' - pad', t' = 0 .. S'-1, i.e. a stride-1 filter of
+// S' = ceil((S + e) / 2) taps (e = pad_w & 1).  Stride along H is served by tiles of one output row.
 bool choose_halo_tile(const q8_conv_desc& d, int P, int Q, HaloTile* out) {
-  if (d.stride_h != 1 || d.stride_w != 1) return false;
-  const int taps = d.R * d.S;
+  const int sw = d.stride_w;
+  if (sw != 1 && sw != 2) return false;
+  int s_eff = d.S, pad_eff = d.pad_w, e = 0, dil_w = d.dil_w;
+  if (sw == 2) {
+    if (d.W % 2 || d.dil_w != 1 || (d.C != 16 && d.C != 32 && d.C != 64)) return false;
+    e = d.pad_w & 1;
+    s_eff = (d.S + e + 1) / 2;
+    pad_eff = (d.pad_w + e) / 2;
+    dil_w = 1;
+    // this view keeps the weights resident in shared memory
+    const int BN = pick_bn(d.K, d.R * d.S * d.C);
+    if ((long long)((d.K + BN - 1) / BN) * BN * d.R * s_eff * 2 * d.C > 80 * 1024) return false;
+  }
+  const int taps = d.R * s_eff;
   if (taps < 2 || taps > kMaxTaps) return false;
-  const int ext_w = (d.S - 1) * d.dil_w, ext_h = (d.R - 1) * d.dil_h;
-  HaloTile best = {0, 0, 0, 0, 0.0};
+  const int ext_w = (s_eff - 1) * dil_w, ext_h = (d.R - 1) * d.dil_h;
+  HaloTile best = {0, 0, 0, 0, 0.0, sw, s_eff, pad_eff, e};
   double best_score = 0.0;
   for (int tw = 1; tw <= Q && tw + ext_w <= kBM; ++tw) {
     const int twb = tw + ext_w;
-    int th = kBM / twb;
+    int th = d.stride_h == 1 ? kBM / twb : 1;
     if (th > P) th = P;
     if (th < 1) continue;
-    const int hb = th + ext_h;
+    const int hb = (th - 1) * d.stride_h + ext_h + 1;
     if (hb > 256 || twb > 256) continue;
     const long long tiles = (long long)((Q + tw - 1) / tw) * ((P + th - 1) / th);
     const double eff = (double)P * Q / ((double)tiles * kBM);
     const double halo = (double)hb * twb / ((double)th * tw);
     const double score = eff / (1.0 + 0.04 * halo);
-    if (score > best_score) { best_score = score; best = {tw, th, twb, hb, eff}; }
+    if (score > best_score) { best_score = score; best.tw = tw; best.th = th; best.twb = twb; best.hb = hb; best.eff = eff; }
   }
   // Tiny images waste accumulator rows (a 7x7 image fills 49 of 128 rows).  Where the im2col path is
   // open it is the better choice for them (it can split the reduction); tensors below its size limit
@@ -1232,19 +1256,32 @@ int launch_conv_umma_impl(const ConvArgs& a, int splits) {
   const bool out8 = d.y_type == Q8_U8 || d.y_type == Q8_S8;
   int res_mode = kResNone;
   if (a.residual) res_mode = (d.K % 16 == 0 && aligned16(a.residual)) ? kResTma : kResGlobal;
-  const int BK = pick_bk(d.C);
-  const int BN = tune_env("Q8_BN", pick_bn(d.K, d.R * d.S * d.C));
-  const CUtensorMapSwizzle swz = swizzle_for_bytes(BK);
-
   UmmaParams p;
   memset(&p, 0, sizeof(p));
-  HaloTile ht = {0, 0, 0, 0, 0.0};
+  HaloTile ht = {0, 0, 0, 0, 0.0, 1, d.S, d.pad_w, 0};
   p.a_mode = is_plain(d) ? kAPlain : ((tune_env("Q8_HALO", 1) && choose_halo_tile(d, a.P, a.Q, &ht)) ? kAHalo : kAIm2col);
+  const bool paired = p.a_mode == kAHalo && ht.sw == 2;  // input read as pixel pairs with 2C channels
+  const int c_eff = paired ? 2 * d.C : d.C;
+  const int BK = pick_bk(c_eff);
+  const int BN = tune_env("Q8_BN", pick_bn(d.K, d.R * d.S * d.C));
+  const CUtensorMapSwizzle swz = swizzle_for_bytes(BK);
   p.bn = BN; p.bk = BK; p.ksteps = BK / 32;
   p.P = a.P; p.Q = a.Q; p.PQ = a.P * a.Q; p.M = (int)a.M; p.K = d.K;
   p.stride_h = d.stride_h; p.stride_w = d.stride_w; p.pad_h = d.pad_h; p.pad_w = d.pad_w; p.dil_h = d.dil_h; p.dil_w = d.dil_w;
   p.R = d.R; p.S = d.S; p.taps = d.R * d.S;
-  p.c_blocks = (d.C + BK - 1) / BK;
+  p.halo_sw = 1; p.halo_e = 0; p.c_true = d.C;
+  if (p.a_mode == kAHalo) {
+    p.S = ht.s_eff; p.taps = d.R * ht.s_eff; p.pad_w = ht.pad_w_eff;
+    p.halo_sw = ht.sw; p.halo_e = ht.e;
+    const int dil_w = paired ? 1 : d.dil_w;
+    for (int r = 0; r < d.R; ++r)
+      for (int t = 0; t < ht.s_eff; ++t) {
+        // tap order = order of the weight tiles in shared memory: (r, s) normally, (t', r) for pixel pairs
+        const int tap = paired ? t * d.R + r : r * ht.s_eff + t;
+        p.tap_shift16[tap] = (unsigned)((r * d.dil_h * ht.twb + t * dil_w) * BK) >> 4;
+      }
+  }
+  p.c_blocks = (c_eff + BK - 1) / BK;
   p.C_pad = p.c_blocks * BK;
   p.k_iters = p.taps * p.c_blocks;
   p.splits = splits;
@@ -1298,7 +1335,7 @@ int launch_conv_umma_impl(const ConvArgs& a, int splits) {
   unsigned min_pipe;
   if (p.a_mode == kAHalo) {
     // the taps read up to (ext_h * twb + ext_w) pixels beyond accumulator row 127
-    const unsigned reach = (unsigned)(kBM + (d.R - 1) * d.dil_h * ht.twb + (d.S - 1) * d.dil_w) * BK;
+    const unsigned reach = (unsigned)(kBM + (d.R - 1) * d.dil_h * ht.twb + (ht.s_eff - 1) * (paired ? 1 : d.dil_w)) * BK;
     p.a_sub_bytes = (unsigned)(BK * ht.twb * ht.hb);
     p.a_stage_bytes = round_up(reach > p.a_sub_bytes ? reach : p.a_sub_bytes, 1024u);
     p.kb = 1;
@@ -1357,6 +1394,7 @@ int launch_conv_umma_impl(const ConvArgs& a, int splits) {
     cuuint64_t dims[4] = {(cuuint64_t)d.C, (cuuint64_t)d.W, (cuuint64_t)d.H, (cuuint64_t)d.N};
     cuuint64_t strides[3] = {(cuuint64_t)d.C, (cuuint64_t)d.W * d.C, (cuuint64_t)d.H * d.W * d.C};
     if (p.a_mode == kAHalo) {
+      if (paired) { dims[0] = (cuuint64_t)c_eff; dims[1] = (cuuint64_t)(d.W / 2); strides[0] = (cuuint64_t)c_eff; }
       cuuint32_t box[4] = {(cuuint32_t)BK, (cuuint32_t)ht.twb, (cuuint32_t)ht.hb, 1};
       cr = fn.tiled(&tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(a.x), dims, strides, box, ones,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -1370,7 +1408,14 @@ int launch_conv_umma_impl(const ConvArgs& a, int splits) {
     }
   }
   if (cr != CUDA_SUCCESS) return fail(Q8_ERR_CUDA, "conv_umma: activation tensor map rejected (CUresult %d)", (int)cr);
-  if (resident) {
+  if (resident && paired) {
+    // (S*C, K, R) view of the KRSC weights: a box of 2C bytes along the (s, c) axis is one pixel-pair tap
+    cuuint64_t dims[3] = {(cuuint64_t)d.S * d.C, (cuuint64_t)d.K, (cuuint64_t)d.R};
+    cuuint64_t strides[2] = {(cuuint64_t)d.R * d.S * d.C, (cuuint64_t)d.S * d.C};
+    cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)BN, (cuuint32_t)d.R};
+    cr = fn.tiled(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(a.w), dims, strides, box, ones,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else if (resident) {
     // (C, K, taps) view of the KRSC weights: one box brings bn rows of every tap
     cuuint64_t dims[3] = {(cuuint64_t)d.C, (cuuint64_t)d.K, (cuuint64_t)p.taps};
     cuuint64_t strides[2] = {(cuuint64_t)p.taps * d.C, (cuuint64_t)d.C};

@@ -49,6 +49,12 @@ CASES = [
     ("3x3_c512_k512", 1, 16, 16, 512, 512, 3, 3, 1, 1, 1, False, U8, "u8", True),
     ("3x3_c3_k8_direct", 2, 17, 19, 3, 8, 3, 3, 2, 1, 1, True, U8, None, True),
     ("config1_shape", 1, 14, 14, 64, 64, 3, 3, 1, 1, 1, False, U8, None, True),
+    # stride 2 read as pixel pairs (even W, C in 16/32/64): odd and even padding, odd and even S
+    ("7x7s2_c16_k64_conv1", 2, 112, 112, 16, 64, 7, 7, 2, 3, 1, True, U8, None, True),
+    ("3x3s2_c64_k96_pad1", 2, 30, 36, 64, 96, 3, 3, 2, 1, 1, False, U8, None, True),
+    ("3x3s2_c32_k32_pad0", 3, 31, 34, 32, 32, 3, 3, 2, 0, 1, False, S8, None, False),
+    ("2x2s2_c64_k64", 2, 20, 24, 64, 64, 2, 2, 2, 0, 1, False, U8, None, True),
+    ("5x4s2_c16_k48_pad2", 2, 25, 26, 16, 48, 5, 4, 2, 2, 1, True, F32, None, False),
 ]
 
 
