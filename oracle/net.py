@@ -56,7 +56,11 @@ def calib_maxima(samples_per_batch):
 #   conv + residual sum + ReLU        : u8, q = max(max|conv|, max|residual|) / 255   ("+" rule on a common footing)
 #   dequantized output (logits, heads): fp32, the accumulator is only multiplied by q_x * q_w
 #   pooling                           : type and factor of its input
-#   concat                            : largest branch factor, branches re-expressed at it
+#   concat                            : ONE factor for the whole output: the largest branch factor.  A conv + ReLU
+#                                       whose only reader is a concat (or a concat nested in one) is quantized
+#                                       straight at that shared factor (one rounding); any other branch (a pooled
+#                                       tensor) is re-expressed at it by the concat.  A nested concat shares the
+#                                       factor of the outermost one.
 # A 3-channel input is zero padded to 16 channels (weights too): zeros are exact under a symmetric quantizer.
 # --------------------------------------------------------------------------------------------------
 def _pad_c(a, c_pad):
@@ -67,9 +71,67 @@ def _pad_c(a, c_pad):
     return out
 
 
+def _concat_groups(layers):
+    """For every tensor that ends in a concat: the outermost concat it belongs to.  Returns (root of each
+    concat, shared-factor convs -> root, leaves of each root)."""
+    readers = {}
+    for L in layers:
+        for s in L.src + ([L.residual] if L.residual else []):
+            readers.setdefault(s, []).append(L)
+    by_name = {L.name: L for L in layers}
+
+    def root_of(name):
+        r = readers.get(name, [])
+        while len(r) == 1 and r[0].op == "concat":
+            name = r[0].name
+            r = readers.get(name, [])
+        return name
+
+    root, shared, leaves = {}, {}, {}
+    for L in layers:
+        if L.op != "concat":
+            continue
+        root[L.name] = root_of(L.name)
+        for s in L.src:
+            if by_name[s].op == "concat":
+                continue
+            leaves.setdefault(root[L.name], []).append(s)
+            Ls = by_name[s]
+            if (Ls.op == "conv" and Ls.conv.relu and not Ls.f32_out and Ls.residual is None
+                    and len(readers[s]) == 1):
+                shared[s] = root[L.name]
+    return root, shared, leaves
+
+
 def network_prepare(layers, folded, maxima):
     """Returns {layer name: dict} with the quantized parameters and the (type, factor) of every tensor."""
-    info = {"input": (o.S8, o.factor(maxima["input"], 7))}
+    root, shared, leaves = _concat_groups(layers)
+    by_name = {L.name: L for L in layers}
+    own = {}
+
+    def own_factor(name):
+        """Factor a tensor has before any sharing: its calibrated maximum, or its input's factor for a pool."""
+        if name not in own:
+            L = by_name.get(name)
+            if name == "input":
+                own[name] = o.factor(maxima["input"], 7)
+            elif L.op in ("maxpool", "avgpool"):
+                own[name] = final_factor(L.src[0])
+            elif L.op == "concat":
+                own[name] = group_factor(root[name])
+            elif L.residual is not None:
+                own[name] = o.factor(max(maxima[name + ":pre"], maxima[L.residual]), 8)
+            else:
+                own[name] = o.factor(maxima[name], 8 if L.conv.relu else 7)
+        return own[name]
+
+    def group_factor(r):
+        return max(own_factor(s) for s in leaves[r])
+
+    def final_factor(name):
+        return group_factor(shared[name]) if name in shared else own_factor(name)
+
+    info = {"input": (o.S8, own_factor("input"))}
     prep = {}
     for L in layers:
         t_in, q_in = info[L.src[0]]
@@ -83,19 +145,19 @@ def network_prepare(layers, folded, maxima):
             if L.f32_out:
                 d.update(y_type=o.F32, q_y=1.0)
             elif L.residual is not None:
-                q_y = o.factor(max(maxima[L.name + ":pre"], maxima[L.residual]), 8)
+                q_y = final_factor(L.name)
                 d.update(y_type=o.U8, q_y=q_y, res_scale=o.requant_scale(info[L.residual][1], 1.0, q_y))
             elif L.conv.relu:
-                d.update(y_type=o.U8, q_y=o.factor(maxima[L.name], 8))
+                d.update(y_type=o.U8, q_y=final_factor(L.name))
             else:
-                d.update(y_type=o.S8, q_y=o.factor(maxima[L.name], 7))
+                d.update(y_type=o.S8, q_y=final_factor(L.name))
             d["scale"] = o.requant_scale(q_in, q_w, d["q_y"])
             prep[L.name] = d
             info[L.name] = (d["y_type"], d["q_y"])
         elif L.op in ("maxpool", "avgpool"):
             info[L.name] = (t_in, q_in)
         elif L.op == "concat":
-            info[L.name] = (t_in, max(info[s][1] for s in L.src))
+            info[L.name] = (t_in, group_factor(root[L.name]))
         else:
             raise ValueError(L.op)
     return prep, info

@@ -1,0 +1,123 @@
+"""CPU pins of the oracle's whole-network assembly (factor rules, residual sum, concat under one factor) and of
+the layer lists: the quantized run must track the FP32 run of the same seeded network, and the structural
+rules must hold on the tensors it returns."""
+import numpy as np
+
+import oracle as o
+from oracle import net as oracle_net
+from workloads import nets
+from workloads.nets import Layer, _conv
+from workloads.synth import rng
+
+
+def _fold(layers):
+    folded = {}
+    for L in layers:
+        if L.op != "conv":
+            continue
+        sp = L.conv
+        if sp.bn:
+            folded[L.name] = o.fold_bn(sp.w, sp.b, sp.gamma, sp.beta, sp.mean, sp.var, 1e-5)
+        else:
+            folded[L.name] = (sp.w, sp.b if sp.b is not None else np.zeros(sp.K, np.float32))
+    return folded
+
+
+def _calibrate(layers, folded, seed, batch, hw, batches=2):
+    maxima = {}
+    for i in range(batches):
+        acts = nets.fp32_forward(layers, nets.images(seed + 10 + i, batch, hw), folded)
+        for k, v in acts.items():
+            maxima[k] = o.maxabs(v, init=maxima.get(k, 0.0))
+    return maxima
+
+
+def _mini_inception(seed=77):
+    """Stem, one module with conv / avg-pool branches and a nested concat, one reduction module with a max-pool
+    branch, classifier."""
+    g = rng(seed)
+    L = []
+    x = _conv(g, L, "stem", "input", 3, 32, 3, pad=1)
+    b1 = _conv(g, L, "m0_1x1", x, 32, 16, 1)
+    r = _conv(g, L, "m0_reduce", x, 32, 16, 1)
+    L.append(Layer("m0_pair", "concat", [_conv(g, L, "m0_1x3", r, 16, 16, 1, 3, pad=(0, 1)),
+                                         _conv(g, L, "m0_3x1", r, 16, 16, 3, 1, pad=(1, 0))]))
+    L.append(Layer("m0_pool", "avgpool", [x], k=(3, 3), stride=(1, 1), pad=(1, 1)))
+    b4 = _conv(g, L, "m0_proj", "m0_pool", 32, 16, 1)
+    L.append(Layer("m0", "concat", [b1, "m0_pair", b4]))
+    c1 = _conv(g, L, "m1_3x3_s2", "m0", 64, 32, 3, stride=2)
+    L.append(Layer("m1_pool", "maxpool", ["m0"], k=(3, 3), stride=(2, 2)))
+    L.append(Layer("m1", "concat", [c1, "m1_pool"]))
+    L.append(Layer("gap", "avgpool", ["m1"], k=(5, 5), stride=(1, 1)))
+    _conv(g, L, "fc", "gap", 96, 10, 1, relu=False, bn=False, bias=True, f32_out=True)
+    return L
+
+
+def _rel(a, b):
+    return float(np.linalg.norm(a.astype(np.float64) - b) / np.linalg.norm(b))
+
+
+def test_concat_groups_share_one_factor_and_copy_their_conv_branches():
+    layers = _mini_inception()
+    folded = _fold(layers)
+    maxima = _calibrate(layers, folded, 77, 2, 12)
+    prep, info = oracle_net.network_prepare(layers, folded, maxima)
+    # module 0: every leaf is a conv + ReLU read only by the concat tree -> all five tensors carry one factor,
+    # the largest of the leaves' own max/255
+    leaves0 = ["m0_1x1", "m0_1x3", "m0_3x1", "m0_proj"]
+    q0 = max(o.factor(maxima[n], 8) for n in leaves0)
+    for n in leaves0 + ["m0_pair", "m0"]:
+        assert info[n] == (o.U8, q0), n
+    # module 1: the pooled branch keeps the factor of its input (q0) and is re-expressed by the concat
+    q1 = max(o.factor(maxima["m1_3x3_s2"], 8), q0)
+    assert info["m1_pool"] == (o.U8, q0) and info["m1"][1] == q1 and info["m1_3x3_s2"][1] == q1
+    # a tensor with a second reader keeps its own factor
+    assert info["stem"][1] == o.factor(maxima["stem"], 8) and info["m0_reduce"][1] == o.factor(maxima["m0_reduce"], 8)
+
+    x = nets.images(78, 2, 12)
+    out = oracle_net.network_forward(layers, prep, info, x)
+    assert np.array_equal(out["m0"], np.concatenate([out["m0_1x1"], out["m0_1x3"], out["m0_3x1"], out["m0_proj"]], -1))
+    assert np.array_equal(out["m1"][..., :32], out["m1_3x3_s2"])
+    assert np.array_equal(out["m1"][..., 32:], o.concat([out["m1_pool"]], [q0], q1))
+    # the quantized tensors follow the FP32 run
+    ref = nets.fp32_forward(layers, x, folded)
+    for n in ("stem", "m0", "m1"):
+        assert _rel(o.dequantize(out[n], info[n][1]), ref[n]) < 0.06, n
+    assert _rel(out["fc"], ref["fc"]) < 0.1
+
+
+def test_residual_stack_follows_fp32_and_uses_the_plus_rule():
+    layers = nets.bottleneck_stack(C=16, blocks=2)
+    folded = _fold(layers)
+    maxima = _calibrate(layers, folded, 31, 2, 16)
+    prep, info = oracle_net.network_prepare(layers, folded, maxima)
+    assert info["input"] == (o.S8, o.factor(maxima["input"], 7))
+    assert info["blk0_branch1"] == (o.S8, o.factor(maxima["blk0_branch1"], 7))        # no ReLU: signed, p = 7
+    assert info["blk0_branch2c"][1] == o.factor(max(maxima["blk0_branch2c:pre"], maxima["blk0_branch1"]), 8)
+    assert info["blk1_branch2c"][1] == o.factor(max(maxima["blk1_branch2c:pre"], maxima["blk0_branch2c"]), 8)
+    assert info["pool1"] == info["conv1"]
+    x = nets.images(32, 2, 16)
+    out = oracle_net.network_forward(layers, prep, info, x)
+    ref = nets.fp32_forward(layers, x, folded)
+    for L in layers:
+        assert _rel(o.dequantize(out[L.name], info[L.name][1]), ref[L.name]) < 0.12, L.name
+    # the fused sum equals the literal "+" of the two quantized summands up to one output code
+    pre = oracle_net.network_forward([L for L in layers if L.name != "blk1_branch2c"], prep, info, x)
+    d = prep["blk1_branch2c"]
+    sp = layers[-1].conv
+    unfused = o.conv2d(pre["blk1_branch2b"], d["w_q"], d["b_q"], d["scale"], sp.stride, sp.pad, sp.dil, None, 0.0, False, o.F32)
+    want = np.clip(np.rint(np.maximum(unfused + out["blk0_branch2c"].astype(np.float32) * np.float32(d["res_scale"]), 0)), 0, 255)
+    assert np.array_equal(out["blk1_branch2c"], want.astype(np.uint8))
+
+
+def test_layer_lists_match_the_published_architectures():
+    r50, inc, ssd = nets.resnet50(), nets.inception_v3(), nets.ssd300()
+    assert sum(L.op == "conv" for L in r50) == 54 and nets.macs(r50, 224) == 3857973248
+    assert sum(L.op == "conv" for L in inc) == 95 and nets.macs(inc, 299) == 5713216096
+    assert sum(L.op == "conv" for L in ssd) == 35 and nets.macs(ssd, 300) == 31373537792
+    assert sum(L.op == "concat" for L in inc) == 15
+    heads = [L for L in ssd if L.f32_out]
+    assert len(heads) == 12 and sorted({L.conv.K for L in heads}) == [16, 24, 84, 126]
+    fc6 = next(L for L in ssd if L.name == "fc6").conv
+    assert (fc6.R, fc6.dil, fc6.pad) == (3, (6, 6), (6, 6))
+    assert next(L for L in ssd if L.name == "pool3").ceil_mode

@@ -31,12 +31,15 @@ class Layer:
     ceil_mode: bool = False
 
 
+def _pair(v):
+    return tuple(v) if isinstance(v, (tuple, list)) else (v, v)
+
+
 def _conv(g, layers, name, src, C, K, R=1, S=None, stride=1, pad=0, dil=1, relu=True, bn=True, bias=False,
           residual=None, f32_out=False):
     S = R if S is None else S
-    sp = make_conv(g, name, C, K, R, S, stride, pad, dil, relu, bn, bias)
-    if isinstance(pad, tuple):
-        sp.pad = pad
+    sp = make_conv(g, name, C, K, R, S, 1, 0, 1, relu, bn, bias)
+    sp.stride, sp.pad, sp.dil = _pair(stride), _pair(pad), _pair(dil)
     layers.append(Layer(name, "conv", [src], conv=sp, residual=residual, f32_out=f32_out))
     return name
 
@@ -83,6 +86,133 @@ def bottleneck_stack(seed: int = 3100, C: int = 64, blocks: int = 2) -> List[Lay
         bb = _conv(g, L, tag + "_branch2b", a, C, C, 3, pad=1)
         x = _conv(g, L, tag + "_branch2c", bb, C, C * 4, 1, relu=True, residual=short)
         c_in = C * 4
+    return L
+
+
+def inception_v3(seed: int = 4000, classes: int = 1000) -> List[Layer]:
+    """Inception-v3 for 299x299 inputs: stem, 3 modules at 35x35, grid reduction, 4 modules with factorized
+    7x7 filters at 17x17, grid reduction, 2 expanded modules at 8x8, global pool, classifier.  Every convolution
+    is conv + BN + ReLU; branches meet in channel concatenations; 95 affine layers, 5.71 GMAC per image."""
+    g = rng(seed)
+    L: List[Layer] = []
+
+    def cat(name, srcs):
+        L.append(Layer(name, "concat", list(srcs)))
+        return name
+
+    def pool(name, src, kind, k, stride, pad=0):
+        L.append(Layer(name, kind, [src], k=(k, k), stride=(stride, stride), pad=(pad, pad)))
+        return name
+
+    x = _conv(g, L, "conv1_3x3_s2", "input", 3, 32, 3, stride=2)
+    x = _conv(g, L, "conv2_3x3", x, 32, 32, 3)
+    x = _conv(g, L, "conv3_3x3", x, 32, 64, 3, pad=1)
+    x = pool("pool1", x, "maxpool", 3, 2)
+    x = _conv(g, L, "conv4_1x1", x, 64, 80, 1)
+    x = _conv(g, L, "conv5_3x3", x, 80, 192, 3)
+    x = pool("pool2", x, "maxpool", 3, 2)
+    c = 192
+    for i, pf in enumerate((32, 64, 64)):                      # 35x35 modules
+        t = f"mixed{i}"
+        b1 = _conv(g, L, t + "_1x1", x, c, 64, 1)
+        b2 = _conv(g, L, t + "_5x5_reduce", x, c, 48, 1)
+        b2 = _conv(g, L, t + "_5x5", b2, 48, 64, 5, pad=2)
+        b3 = _conv(g, L, t + "_3x3_reduce", x, c, 64, 1)
+        b3 = _conv(g, L, t + "_3x3_1", b3, 64, 96, 3, pad=1)
+        b3 = _conv(g, L, t + "_3x3_2", b3, 96, 96, 3, pad=1)
+        b4 = pool(t + "_pool", x, "avgpool", 3, 1, 1)
+        b4 = _conv(g, L, t + "_pool_proj", b4, c, pf, 1)
+        x, c = cat(t, (b1, b2, b3, b4)), 64 + 64 + 96 + pf
+    t = "mixed3"                                                # 35 -> 17
+    b1 = _conv(g, L, t + "_3x3_s2", x, c, 384, 3, stride=2)
+    b2 = _conv(g, L, t + "_dbl_reduce", x, c, 64, 1)
+    b2 = _conv(g, L, t + "_dbl_1", b2, 64, 96, 3, pad=1)
+    b2 = _conv(g, L, t + "_dbl_2_s2", b2, 96, 96, 3, stride=2)
+    b3 = pool(t + "_pool", x, "maxpool", 3, 2)
+    x, c = cat(t, (b1, b2, b3)), 384 + 96 + c
+    for i, c7 in enumerate((128, 160, 160, 192), start=4):     # 17x17 modules
+        t = f"mixed{i}"
+        b1 = _conv(g, L, t + "_1x1", x, c, 192, 1)
+        b2 = _conv(g, L, t + "_7x7_reduce", x, c, c7, 1)
+        b2 = _conv(g, L, t + "_1x7", b2, c7, c7, 1, 7, pad=(0, 3))
+        b2 = _conv(g, L, t + "_7x1", b2, c7, 192, 7, 1, pad=(3, 0))
+        b3 = _conv(g, L, t + "_dbl_reduce", x, c, c7, 1)
+        b3 = _conv(g, L, t + "_dbl_7x1_1", b3, c7, c7, 7, 1, pad=(3, 0))
+        b3 = _conv(g, L, t + "_dbl_1x7_1", b3, c7, c7, 1, 7, pad=(0, 3))
+        b3 = _conv(g, L, t + "_dbl_7x1_2", b3, c7, c7, 7, 1, pad=(3, 0))
+        b3 = _conv(g, L, t + "_dbl_1x7_2", b3, c7, 192, 1, 7, pad=(0, 3))
+        b4 = pool(t + "_pool", x, "avgpool", 3, 1, 1)
+        b4 = _conv(g, L, t + "_pool_proj", b4, c, 192, 1)
+        x, c = cat(t, (b1, b2, b3, b4)), 768
+    t = "mixed8"                                                # 17 -> 8
+    b1 = _conv(g, L, t + "_3x3_reduce", x, c, 192, 1)
+    b1 = _conv(g, L, t + "_3x3_s2", b1, 192, 320, 3, stride=2)
+    b2 = _conv(g, L, t + "_7x7x3_reduce", x, c, 192, 1)
+    b2 = _conv(g, L, t + "_7x7x3_1x7", b2, 192, 192, 1, 7, pad=(0, 3))
+    b2 = _conv(g, L, t + "_7x7x3_7x1", b2, 192, 192, 7, 1, pad=(3, 0))
+    b2 = _conv(g, L, t + "_7x7x3_3x3_s2", b2, 192, 192, 3, stride=2)
+    b3 = pool(t + "_pool", x, "maxpool", 3, 2)
+    x, c = cat(t, (b1, b2, b3)), 320 + 192 + c
+    for i in (9, 10):                                           # 8x8 modules
+        t = f"mixed{i}"
+        b1 = _conv(g, L, t + "_1x1", x, c, 320, 1)
+        r = _conv(g, L, t + "_3x3_reduce", x, c, 384, 1)
+        b2 = cat(t + "_3x3", (_conv(g, L, t + "_3x3_1x3", r, 384, 384, 1, 3, pad=(0, 1)),
+                              _conv(g, L, t + "_3x3_3x1", r, 384, 384, 3, 1, pad=(1, 0))))
+        r = _conv(g, L, t + "_dbl_reduce", x, c, 448, 1)
+        r = _conv(g, L, t + "_dbl_3x3", r, 448, 384, 3, pad=1)
+        b3 = cat(t + "_dbl", (_conv(g, L, t + "_dbl_1x3", r, 384, 384, 1, 3, pad=(0, 1)),
+                              _conv(g, L, t + "_dbl_3x1", r, 384, 384, 3, 1, pad=(1, 0))))
+        b4 = pool(t + "_pool", x, "avgpool", 3, 1, 1)
+        b4 = _conv(g, L, t + "_pool_proj", b4, c, 192, 1)
+        x, c = cat(t, (b1, b2, b3, b4)), 2048
+    L.append(Layer("pool3", "avgpool", [x], k=(8, 8), stride=(1, 1)))
+    _conv(g, L, "fc", "pool3", 2048, classes, 1, relu=False, bn=False, bias=True, f32_out=True)
+    return L
+
+
+def ssd300(seed: int = 5000, classes: int = 21) -> List[Layer]:
+    """SSD-300 on VGG-16: the base network through conv5_3 (pool3 in ceil mode, pool5 3x3 stride 1), fc6 as
+    a dilated 3x3 (dilation 6), fc7 as 1x1, four extra stages, and a 3x3 localisation and confidence head on
+    each of the six source maps (38, 19, 10, 5, 3, 1; 4/6/6/6/4/4 boxes per cell, 8732 boxes).  Convolutions
+    carry a bias and no BN; head outputs are dequantized FP32.  No normalisation layer on conv4_3."""
+    g = rng(seed)
+    L: List[Layer] = []
+
+    def conv(name, src, C, K, R=3, **kw):
+        kw.setdefault("pad", 1 if R == 3 else 0)
+        return _conv(g, L, name, src, C, K, R, bn=False, bias=True, **kw)
+
+    def pool(name, src, k, stride, pad=0, ceil_mode=False):
+        L.append(Layer(name, "maxpool", [src], k=(k, k), stride=(stride, stride), pad=(pad, pad), ceil_mode=ceil_mode))
+        return name
+
+    x, c = "input", 3
+    for stage, (n, k) in enumerate(((2, 64), (2, 128), (3, 256), (3, 512), (3, 512)), start=1):
+        for i in range(1, n + 1):
+            x, c = conv(f"conv{stage}_{i}", x, c, k), k
+        if stage < 5:
+            x = pool(f"pool{stage}", x, 2, 2, ceil_mode=(stage == 3))
+    sources = [("conv4_3", 512, 4)]
+    x = pool("pool5", x, 3, 1, 1)
+    x = conv("fc6", x, 512, 1024, 3, pad=6, dil=6)
+    x = conv("fc7", x, 1024, 1024, 1)
+    sources.append((x, 1024, 6))
+    x = conv("conv6_1", x, 1024, 256, 1)
+    x = conv("conv6_2", x, 256, 512, 3, stride=2)
+    sources.append((x, 512, 6))
+    x = conv("conv7_1", x, 512, 128, 1)
+    x = conv("conv7_2", x, 128, 256, 3, stride=2)
+    sources.append((x, 256, 6))
+    x = conv("conv8_1", x, 256, 128, 1)
+    x = conv("conv8_2", x, 128, 256, 3, pad=0)
+    sources.append((x, 256, 4))
+    x = conv("conv9_1", x, 256, 128, 1)
+    x = conv("conv9_2", x, 128, 256, 3, pad=0)
+    sources.append((x, 256, 4))
+    for src, c, boxes in sources:
+        conv(src + "_mbox_loc", src, c, boxes * 4, relu=False, f32_out=True)
+        conv(src + "_mbox_conf", src, c, boxes * classes, relu=False, f32_out=True)
     return L
 
 
