@@ -206,6 +206,16 @@ int q8_conv2d_static_workspace(const q8_conv_desc* d, const void* x, const int8_
 int q8_concat(int n_in, const void* const* xs, const int* channels, const float* in_factors,
               float out_factor, int t, size_t pixels, void* y, void* stream);
 
+/* One branch of such a concatenation, written into a channel slice of a wider tensor: for branches that
+ * cannot be produced in place (a pooled tensor whose factor differs from the shared one) while the
+ * convolution branches write their slices themselves (q8_conv_desc y_ldc / y_c_offset).
+ * x: device [pixels][channels].  y: device [pixels][y_ldc]; channels y_c_offset .. y_c_offset+channels-1
+ * are written, the rest of y is untouched.  Same arithmetic as q8_concat.
+ * Errors: Q8_ERR_INVALID_ARG (null pointer, channels <= 0, slice outside y_ldc, type not U8/S8),
+ * Q8_ERR_NONFINITE (factor not finite positive). */
+int q8_concat_branch(const void* x, int channels, float in_factor, float out_factor, int t, size_t pixels,
+                     void* y, int y_ldc, int y_c_offset, void* stream);
+
 /* ------------------------------------------------------------------------
  * Pooling between quantized layers (not described in the paper; needed to
  * run whole networks in int8).  The factor is unchanged.

@@ -21,7 +21,7 @@ TORCH_DTYPES = {Q8_U8: torch.uint8, Q8_S8: torch.int8, Q8_S32: torch.int32, Q8_F
 EXPORTS = ["q8_version", "q8_last_error", "q8_read_status", "q8_calibrate_maxabs", "q8_factor", "q8_requant_scale",
            "q8_bias_factor", "q8_quantize", "q8_quantize_pad_channels", "q8_dequantize", "q8_fold_bn",
            "q8_conv2d_workspace_bytes", "q8_conv2d_query_algo", "q8_conv2d", "q8_static_workspace_bytes",
-           "q8_conv2d_static_workspace", "q8_concat", "q8_pool_out_extent",
+           "q8_conv2d_static_workspace", "q8_concat", "q8_concat_branch", "q8_pool_out_extent",
            "q8_maxpool2d", "q8_avgpool2d"]
 
 
@@ -68,6 +68,7 @@ lib.q8_conv2d.argtypes = [C.POINTER(q8_conv_desc), _vp, _vp, _vp, _vp, _vp, _f, 
 lib.q8_static_workspace_bytes.argtypes = []
 lib.q8_conv2d_static_workspace.argtypes = [C.POINTER(q8_conv_desc), _vp, _vp, _vp, _vp, _vp, _f, _vp, _vp]
 lib.q8_concat.argtypes = [_i, C.POINTER(_vp), _ip, _fp, _f, _i, _sz, _vp, _vp]
+lib.q8_concat_branch.argtypes = [_vp, _i, _f, _f, _i, _sz, _vp, _i, _i, _vp]
 lib.q8_pool_out_extent.argtypes = [_i] * 5 + [_ip]
 lib.q8_maxpool2d.argtypes = [_vp, _i] + [_i] * 11 + [_vp, _vp]
 lib.q8_avgpool2d.argtypes = [_vp, _i] + [_i] * 11 + [_vp, _vp]
@@ -226,6 +227,15 @@ def q8_concat(xs, in_factors, out_factor, out=None):
         _dev(a, "branch")
     _check(lib.q8_concat(len(xs), ptrs, (C.c_int * len(xs))(*chans), (C.c_float * len(xs))(*in_factors), out_factor, t,
                          pixels, _dev(out, "out"), _stream()))
+    return out
+
+
+def q8_concat_branch(x, in_factor, out_factor, out, c_offset):
+    """Writes x (re-expressed at out_factor) into channels c_offset.. of the wider tensor `out`."""
+    t = {torch.uint8: Q8_U8, torch.int8: Q8_S8}[x.dtype]
+    ch = int(x.shape[-1])
+    _check(lib.q8_concat_branch(_dev(x, "x"), ch, in_factor, out_factor, t, x.numel() // ch, _dev(out, "out"),
+                                int(out.shape[-1]), c_offset, _stream()))
     return out
 
 

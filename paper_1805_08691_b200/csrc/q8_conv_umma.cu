@@ -1038,27 +1038,27 @@ int sm_count() {
 }
 
 int pick_bk(int C) {
-  int best = 32, best_pad = ((C + 31) / 32) * 32;
-  for (int bk : {64, 128}) {
-    int padded = ((C + bk - 1) / bk) * bk;
-    if (padded <= best_pad) { best = bk; best_pad = padded; }
-  }
-  return best;
+  // A pipeline iteration costs one TMA operation per operand (several hundred cycles whatever its size), so the
+  // widest channel block that C reaches wins even when it pads C: out-of-range channels are zero filled by TMA
+  // and cost tensor-core time only, which a short reduction has to spare.
+  return C <= 32 ? 32 : (C <= 64 ? 64 : 128);
 }
 
 // Tile width: the multiple of 16 (power-of-two panels keep the 8-bit tile layout simple) that pads
 // Cout least; short reductions are bandwidth bound and take narrower tiles, which leaves room for
 // four TMEM accumulators and more tile buffers.
 int pick_bn(int K, int kgemm) {
-  static const int widths[] = {16, 32, 48, 64, 96, 128, 192, 256};
   const int cap = kgemm <= 640 ? 128 : 256;
+  const double k_steps = (kgemm + 31) / 32, k_iters = (kgemm + 127) / 128;
   int best = 16;
-  long long best_cost = -1;
-  for (int w : widths) {
-    if (w > cap) break;
-    const long long padded = (long long)((K + w - 1) / w) * w;
-    // padded columns are wasted MMA and epilogue work; every extra tile re-reads A once more
-    const long long cost = padded * 8 + (padded / w) * 24;
+  double best_cost = -1.0;
+  for (int w = 16; w <= cap; w += 16) {
+    const int n_tiles = (K + w - 1) / w;
+    // cycles per 128-row block of the output: every tile of columns runs the whole reduction again (one
+    // 128 x w x 32 MMA takes max(59, 0.53 w) cycles, a pipeline iteration about 550), the epilogue pays for
+    // every padded column
+    const double mma = k_steps * (0.53 * w > 59.0 ? 0.53 * w : 59.0), feed = k_iters * 550.0;
+    const double cost = n_tiles * ((mma > feed ? mma : feed) + 200.0) + (double)n_tiles * w * 8.0;
     if (best_cost < 0 || cost <= best_cost) { best = w; best_cost = cost; }
   }
   return best;
@@ -1137,7 +1137,8 @@ bool choose_halo_tile(const q8_conv_desc& d, int P, int Q, HaloTile* out) {
   // open it is the better choice for them (it can split the reduction); tensors below its size limit
   // still take halo tiles rather than leave the tensor cores.
   const bool im2col_closed = (long long)d.N * d.H * d.W * d.C < 131072;
-  if (best.eff < (im2col_closed ? 0.2 : 0.5)) return false;
+  if (!im2col_closed && best.eff < 0.5) return false;
+  if (best.tw == 0) return false;
   *out = best;
   return true;
 }
@@ -1221,8 +1222,20 @@ int umma_plan_splits(const q8_conv_desc& d, int P, int Q, long long M) {
 }
 
 namespace {
-int launch_conv_umma_impl(const ConvArgs& a, int splits);
+constexpr int kPlanNoFit = -1000;  // internal: this tile shape needs more shared memory than an SM has
+int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_halo);
+
+// Tries tile shapes from the preferred one down: halo patches of dilated filters on wide channel blocks can
+// exceed shared memory, narrower channel blocks shrink them; im2col loads need the least.
+int launch_conv_umma_impl(const ConvArgs& a, int splits) {
+  static const struct { int bk_cap; bool halo; } kTries[] = {{128, true}, {64, true}, {32, true}, {128, false}, {64, false}};
+  for (const auto& t : kTries) {
+    const int rc = launch_conv_umma_plan(a, splits, t.bk_cap, t.halo);
+    if (rc != kPlanNoFit) return rc;
+  }
+  return fail(Q8_ERR_UNSUPPORTED, "conv_umma: no tile shape of this layer fits in shared memory");
 }
+}  // namespace
 
 int launch_conv_umma(const ConvArgs& a) {
   const q8_conv_desc& d = a.d;
@@ -1246,7 +1259,7 @@ int launch_conv_umma(const ConvArgs& a) {
 }
 
 namespace {
-int launch_conv_umma_impl(const ConvArgs& a, int splits) {
+int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_halo) {
   const q8_conv_desc& d = a.d;
   DriverFns& fn = driver_fns();
   if (!fn.tiled || !fn.im2col) return fail(Q8_ERR_CUDA, "conv_umma: cuTensorMapEncode* entry points not available");
@@ -1259,10 +1272,10 @@ int launch_conv_umma_impl(const ConvArgs& a, int splits) {
   UmmaParams p;
   memset(&p, 0, sizeof(p));
   HaloTile ht = {0, 0, 0, 0, 0.0, 1, d.S, d.pad_w, 0};
-  p.a_mode = is_plain(d) ? kAPlain : ((tune_env("Q8_HALO", 1) && choose_halo_tile(d, a.P, a.Q, &ht)) ? kAHalo : kAIm2col);
+  p.a_mode = is_plain(d) ? kAPlain : ((allow_halo && tune_env("Q8_HALO", 1) && choose_halo_tile(d, a.P, a.Q, &ht)) ? kAHalo : kAIm2col);
   const bool paired = p.a_mode == kAHalo && ht.sw == 2;  // input read as pixel pairs with 2C channels
   const int c_eff = paired ? 2 * d.C : d.C;
-  const int BK = pick_bk(c_eff);
+  const int BK = pick_bk(c_eff) < bk_cap ? pick_bk(c_eff) : bk_cap;
   const int BN = tune_env("Q8_BN", pick_bn(d.K, d.R * d.S * d.C));
   const CUtensorMapSwizzle swz = swizzle_for_bytes(BK);
   p.bn = BN; p.bk = BK; p.ksteps = BK / 32;
@@ -1357,7 +1370,7 @@ int launch_conv_umma_impl(const ConvArgs& a, int splits) {
     p.nbuf = tune_env("Q8_NBUF", p.nbuf);
   }
   const unsigned buf_bytes = (unsigned)(G * p.nbuf) * p.tile8_bytes;
-  if (budget < bres_bytes + buf_bytes + min_pipe) return fail(Q8_ERR_UNSUPPORTED, "conv_umma: tile does not fit in shared memory");
+  if (budget < bres_bytes + buf_bytes + min_pipe) return kPlanNoFit;
   unsigned rest = budget - bres_bytes - buf_bytes;
   p.b_stages = 0;
   if (p.b_mode == kBRing) {
@@ -1374,7 +1387,7 @@ int launch_conv_umma_impl(const ConvArgs& a, int splits) {
   p.off_bufs = p.off_bring + (unsigned)p.b_stages * p.b_sub_bytes;
   p.off_chan = p.off_bufs + buf_bytes;
   size_t dyn = 1024u + p.off_chan + chan_bytes;
-  if (dyn > (size_t)(kSmemLimit - kStaticSmemReserve)) return fail(Q8_ERR_UNSUPPORTED, "conv_umma: shared memory plan exceeds the limit");
+  if (dyn > (size_t)(kSmemLimit - kStaticSmemReserve)) return kPlanNoFit;
   // at least 120 KiB so that one CTA owns an SM and with it the whole TMEM
   if (dyn < 120 * 1024) dyn = 120 * 1024;
 

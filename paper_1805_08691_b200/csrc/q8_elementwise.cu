@@ -347,6 +347,59 @@ __global__ void __launch_bounds__(256) maxpool16_kernel(const uint4* __restrict_
   }
 }
 
+// Average pooling with 16 channels per thread.  Bytes are summed as pairs of 16-bit lanes (window of at most
+// 256 cells: 256 * 255 < 2^16); signed bytes are biased by +128 first and the bias of the cells that were
+// inside the image is taken off the sum.  Then float(sum) * fp32(1/(kh kw)), round half even, clamp.
+template <bool kSigned>
+__global__ void __launch_bounds__(256) avgpool16_kernel(const uint4* __restrict__ x, int N, int H, int W, int cg, int kh,
+                                                        int kw, int st_h, int st_w, int pad_h, int pad_w, int P, int Q,
+                                                        float inv, uint4* __restrict__ y) {
+  const size_t total = (size_t)N * P * Q * cg;
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += nthreads) {
+    const int c = (int)(i % cg);
+    size_t t = i / cg;
+    const int q = (int)(t % Q);
+    t /= Q;
+    const int p = (int)(t % P);
+    const int n = (int)(t / P);
+    unsigned int even[4] = {0, 0, 0, 0}, odd[4] = {0, 0, 0, 0};  // bytes 0,2 and bytes 1,3 of each word
+    int cells = 0;
+    for (int r = 0; r < kh; ++r) {
+      const int h = p * st_h - pad_h + r;
+      if (h < 0 || h >= H) continue;
+      for (int s = 0; s < kw; ++s) {
+        const int w = q * st_w - pad_w + s;
+        if (w < 0 || w >= W) continue;
+        uint4 v = __ldg(x + (((size_t)n * H + h) * W + w) * cg + c);
+        if (kSigned) { v.x ^= 0x80808080u; v.y ^= 0x80808080u; v.z ^= 0x80808080u; v.w ^= 0x80808080u; }
+        const unsigned int word[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          even[j] += word[j] & 0x00ff00ffu;
+          odd[j] += (word[j] >> 8) & 0x00ff00ffu;
+        }
+        ++cells;
+      }
+    }
+    const int bias = kSigned ? 128 * cells : 0;
+    unsigned int out[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int sum[4] = {(int)(even[j] & 0xffffu) - bias, (int)(odd[j] & 0xffffu) - bias, (int)(even[j] >> 16) - bias,
+                          (int)(odd[j] >> 16) - bias};
+      int o[4];
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const int z = __float2int_rn(__fmul_rn((float)sum[b], inv));
+        o[b] = kSigned ? min(max(z, -128), 127) : min(max(z, 0), 255);
+      }
+      out[j] = pack4(o[0], o[1], o[2], o[3]);
+    }
+    y[i] = make_uint4(out[0], out[1], out[2], out[3]);
+  }
+}
+
 int pool_extent(int H, int k, int st, int pad, int ceil_mode) {
   int num = H + 2 * pad - k;
   int o = (ceil_mode ? (num + st - 1) / st : num / st) + 1;
@@ -373,6 +426,13 @@ int launch_pool(const void* x, int t, int N, int H, int W, int C, int kh, int kw
     if (t == Q8_S8) maxpool16_kernel<true><<<grid16, 256, 0, s>>>(static_cast<const uint4*>(x), N, H, W, cg, kh, kw, st_h, st_w, pad_h, pad_w, P, Q, static_cast<uint4*>(y));
     else maxpool16_kernel<false><<<grid16, 256, 0, s>>>(static_cast<const uint4*>(x), N, H, W, cg, kh, kw, st_h, st_w, pad_h, pad_w, P, Q, static_cast<uint4*>(y));
     return check_launch("maxpool16_kernel");
+  }
+  if (kAvg && C % 16 == 0 && kh * kw <= 256 && aligned16(x) && aligned16(y)) {
+    const int cg = C / 16;
+    const int grid16 = grid_for((size_t)N * P * Q * cg, 256, 8);
+    if (t == Q8_S8) avgpool16_kernel<true><<<grid16, 256, 0, s>>>(static_cast<const uint4*>(x), N, H, W, cg, kh, kw, st_h, st_w, pad_h, pad_w, P, Q, inv, static_cast<uint4*>(y));
+    else avgpool16_kernel<false><<<grid16, 256, 0, s>>>(static_cast<const uint4*>(x), N, H, W, cg, kh, kw, st_h, st_w, pad_h, pad_w, P, Q, inv, static_cast<uint4*>(y));
+    return check_launch("avgpool16_kernel");
   }
   bool vec = (C % 4 == 0) && ((reinterpret_cast<uintptr_t>(x) & 3u) == 0) && ((reinterpret_cast<uintptr_t>(y) & 3u) == 0);
   size_t total = (size_t)N * P * Q * (vec ? C / 4 : C);
@@ -515,6 +575,33 @@ int q8_fold_bn(const float* w, const float* b, const float* gamma, const float* 
   return check_launch("fold_bn_kernel");
 }
 
+int q8_concat_branch(const void* x, int channels, float in_factor, float out_factor, int t, size_t pixels, void* y,
+                     int y_ldc, int y_c_offset, void* stream) {
+  clear_error();
+  if (!x || !y || channels <= 0 || y_c_offset < 0 || (long long)y_c_offset + channels > (long long)y_ldc)
+    return fail(Q8_ERR_INVALID_ARG, "q8_concat_branch: bad argument");
+  if (t != Q8_U8 && t != Q8_S8) return fail(Q8_ERR_INVALID_ARG, "q8_concat_branch: type must be Q8_U8 or Q8_S8");
+  if (!(out_factor > 0.f) || std::isinf(out_factor) || !(in_factor > 0.f) || std::isinf(in_factor))
+    return fail(Q8_ERR_NONFINITE, "q8_concat_branch: factors must be finite and positive");
+  if (pixels == 0) return Q8_OK;
+  cudaStream_t s = as_stream(stream);
+  volatile double ratio = (double)in_factor / (double)out_factor;
+  float sc = (float)ratio;
+  int copy_only = sc == 1.0f;
+  const int ch = channels, ctot = y_ldc, off = y_c_offset;
+  bool vec = (ch % 16 == 0) && (ctot % 16 == 0) && (off % 16 == 0) && aligned16(x) && aligned16(y);
+  if (vec) {
+    int grid = grid_for(pixels * (ch / 16), kThreads, 4);
+    if (t == Q8_S8) concat_vec_kernel<true><<<grid, kThreads, 0, s>>>(static_cast<const uint4*>(x), pixels, ch / 16, ctot / 16, off / 16, sc, copy_only, static_cast<uint4*>(y));
+    else concat_vec_kernel<false><<<grid, kThreads, 0, s>>>(static_cast<const uint4*>(x), pixels, ch / 16, ctot / 16, off / 16, sc, copy_only, static_cast<uint4*>(y));
+  } else {
+    int grid = grid_for(pixels * ch, kThreads, 8);
+    if (t == Q8_S8) concat_scalar_kernel<true><<<grid, kThreads, 0, s>>>(static_cast<const unsigned char*>(x), pixels, ch, ctot, off, sc, copy_only, static_cast<unsigned char*>(y));
+    else concat_scalar_kernel<false><<<grid, kThreads, 0, s>>>(static_cast<const unsigned char*>(x), pixels, ch, ctot, off, sc, copy_only, static_cast<unsigned char*>(y));
+  }
+  return check_launch("concat_kernel");
+}
+
 int q8_concat(int n_in, const void* const* xs, const int* channels, const float* in_factors, float out_factor,
               int t, size_t pixels, void* y, void* stream) {
   clear_error();
@@ -527,27 +614,12 @@ int q8_concat(int n_in, const void* const* xs, const int* channels, const float*
     if (!(in_factors[i] > 0.f) || std::isinf(in_factors[i])) return fail(Q8_ERR_NONFINITE, "q8_concat: factor %d not finite positive", i);
     ctot += channels[i];
   }
-  if (pixels == 0) return Q8_OK;
-  cudaStream_t s = as_stream(stream);
+  if (ctot > 0x7fffffffLL) return fail(Q8_ERR_INVALID_ARG, "q8_concat: too many channels");
   int off = 0;
   for (int i = 0; i < n_in; ++i) {
-    volatile double ratio = (double)in_factors[i] / (double)out_factor;
-    float sc = (float)ratio;
-    int copy_only = sc == 1.0f;
-    int ch = channels[i];
-    bool vec = (ch % 16 == 0) && (ctot % 16 == 0) && (off % 16 == 0) && aligned16(xs[i]) && aligned16(y);
-    if (vec) {
-      int grid = grid_for(pixels * (ch / 16), kThreads, 4);
-      if (t == Q8_S8) concat_vec_kernel<true><<<grid, kThreads, 0, s>>>(static_cast<const uint4*>(xs[i]), pixels, ch / 16, (int)(ctot / 16), off / 16, sc, copy_only, static_cast<uint4*>(y));
-      else concat_vec_kernel<false><<<grid, kThreads, 0, s>>>(static_cast<const uint4*>(xs[i]), pixels, ch / 16, (int)(ctot / 16), off / 16, sc, copy_only, static_cast<uint4*>(y));
-    } else {
-      int grid = grid_for(pixels * ch, kThreads, 8);
-      if (t == Q8_S8) concat_scalar_kernel<true><<<grid, kThreads, 0, s>>>(static_cast<const unsigned char*>(xs[i]), pixels, ch, (int)ctot, off, sc, copy_only, static_cast<unsigned char*>(y));
-      else concat_scalar_kernel<false><<<grid, kThreads, 0, s>>>(static_cast<const unsigned char*>(xs[i]), pixels, ch, (int)ctot, off, sc, copy_only, static_cast<unsigned char*>(y));
-    }
-    int rc = check_launch("concat_kernel");
+    int rc = q8_concat_branch(xs[i], channels[i], in_factors[i], out_factor, t, pixels, y, (int)ctot, off, stream);
     if (rc != Q8_OK) return rc;
-    off += ch;
+    off += channels[i];
   }
   return Q8_OK;
 }

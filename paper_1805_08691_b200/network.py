@@ -9,7 +9,12 @@ for the fused residual sum; all tensor arithmetic runs in the library's kernels.
   conv without ReLU                 : s8, q = max|y| / 127
   conv + residual sum + ReLU        : u8, q = max(max|conv|, max|residual|) / 255
   dequantized output (logits, heads): fp32
-  pooling                           : type and factor of its input;  concat: largest branch factor
+  pooling                           : type and factor of its input
+  concat                            : one factor for the whole output, the largest factor among its branches.  A
+                                      conv + ReLU read by nothing but the concat writes its channel slice of the
+                                      concat buffer itself, quantized at that factor; other branches (pooled
+                                      tensors) are re-expressed and copied in by q8_concat_branch; a concat nested
+                                      in another is a slice of the outer buffer and shares its factor
 """
 from typing import Dict, List
 
@@ -25,14 +30,17 @@ class QuantNetwork:
         """folded[name] = (w KRSC, b K) FP32 device tensors; maxima: calibrated max-abs of "input", every layer
         output and "<name>:pre" of residual convolutions; in_shape = (N, H, W, 3)."""
         self.layers = layers
-        self.info = {"input": (q8.Q8_S8, q8.q8_factor(maxima["input"], 7))}
-        self.shape = {}
+        self.maxima = maxima
+        self.by_name = {L.name: L for L in layers}
         self.convs: Dict[str, pipeline.QuantConv] = {}
         self.bufs: Dict[str, torch.Tensor] = {}
         N, H, W, _ = in_shape
         first = next(L for L in layers if L.op == "conv")
         self.c_pad_in = -(-first.conv.C // 16) * 16
-        self.shape["input"] = (N, H, W, self.c_pad_in)
+        self._shapes((N, H, W, self.c_pad_in))
+        self._place_concats()
+        self._factors = {}
+        self.info = {"input": (q8.Q8_S8, self._factor("input"))}
         self.bufs["input"] = torch.empty(self.shape["input"], dtype=torch.int8, device=device)
         ws_bytes = 0
         for L in layers:
@@ -45,38 +53,110 @@ class QuantNetwork:
                     wf = F.pad(wf, (0, c - wf.shape[-1]))
                 if L.f32_out:
                     y_type, q_y = q8.Q8_F32, 1.0
-                elif L.residual is not None:
-                    y_type = q8.Q8_U8
-                    q_y = q8.q8_factor(max(maxima[L.name + ":pre"], maxima[L.residual]), 8)
-                elif sp.relu:
-                    y_type, q_y = q8.Q8_U8, q8.q8_factor(maxima[L.name], 8)
                 else:
-                    y_type, q_y = q8.Q8_S8, q8.q8_factor(maxima[L.name], 7)
+                    y_type, q_y = (q8.Q8_U8 if (sp.relu or L.residual is not None) else q8.Q8_S8), self._factor(L.name)
                 q_res, res_type = None, q8.Q8_U8
                 if L.residual is not None:
                     res_type, q_res = self.info[L.residual]
+                ldc, off = 0, 0
+                if L.name in self.in_place:
+                    root, off = self.slot[L.name]
+                    ldc = self.shape[root][3]
                 qc = pipeline.prepare_conv(wf.contiguous(), bf, (n, h, w_, c), q_in, q_y, t_in, y_type, sp.relu, sp.stride,
-                                           sp.pad, sp.dil, q_res, res_type)
+                                           sp.pad, sp.dil, q_res, res_type, ldc, off)
                 self.convs[L.name] = qc
-                P, Q = q8.conv_out_shape(qc.desc)
-                self.shape[L.name] = (n, P, Q, sp.K)
                 self.info[L.name] = (y_type, qc.q_y)
                 ws_bytes = max(ws_bytes, q8.q8_conv2d_workspace_bytes(qc.desc))
+            elif L.op in ("maxpool", "avgpool"):
+                self.info[L.name] = (t_in, q_in)
+            elif L.op == "concat":
+                self.info[L.name] = (t_in, self._factor(L.name))
+            else:
+                raise ValueError(L.op)
+            dt = q8.TORCH_DTYPES[self.info[L.name][0]]
+            if L.name in self.in_place or (L.op == "concat" and self.slot[L.name][0] != L.name):
+                continue  # a slice of the outermost concat's buffer, bound below
+            self.bufs[L.name] = torch.empty(self.shape[L.name], dtype=dt, device=device)
+        for name, (root, off) in self.slot.items():
+            if name in self.in_place or (self.by_name[name].op == "concat" and root != name):
+                self.bufs[name] = self.bufs[root][..., off:off + self.shape[name][3]]
+        self.workspace = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device=device) if ws_bytes else None
+
+    # ---- host bookkeeping ---------------------------------------------------------------------------
+    def _shapes(self, in_shape):
+        self.shape = {"input": in_shape}
+        for L in self.layers:
+            n, h, w_, c = self.shape[L.src[0]]
+            if L.op == "conv":
+                sp = L.conv
+                P = (h + 2 * sp.pad[0] - sp.dil[0] * (sp.R - 1) - 1) // sp.stride[0] + 1
+                Q = (w_ + 2 * sp.pad[1] - sp.dil[1] * (sp.S - 1) - 1) // sp.stride[1] + 1
+                self.shape[L.name] = (n, P, Q, sp.K)
             elif L.op in ("maxpool", "avgpool"):
                 P = q8.q8_pool_out_extent(h, L.k[0], L.stride[0], L.pad[0], L.ceil_mode)
                 Q = q8.q8_pool_out_extent(w_, L.k[1], L.stride[1], L.pad[1], L.ceil_mode)
                 self.shape[L.name] = (n, P, Q, c)
-                self.info[L.name] = (t_in, q_in)
             elif L.op == "concat":
                 self.shape[L.name] = (n, h, w_, sum(self.shape[s][3] for s in L.src))
-                self.info[L.name] = (t_in, max(self.info[s][1] for s in L.src))
             else:
                 raise ValueError(L.op)
-            self.bufs[L.name] = torch.empty(self.shape[L.name], dtype=q8.TORCH_DTYPES[self.info[L.name][0]], device=device)
-        self.workspace = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device=device) if ws_bytes else None
 
+    def _place_concats(self):
+        """slot[name] = (outermost concat, channel offset) for every tensor that is part of a concat;
+        in_place = the convolutions that write their slice themselves; members[root] = all non-concat parts."""
+        uses: Dict[str, List] = {}
+        for L in self.layers:
+            for s in L.src + ([L.residual] if L.residual else []):
+                uses.setdefault(s, []).append(L)
+        self.slot, self.in_place, self.members = {}, set(), {}
+
+        def place(cat, root, base):
+            self.slot[cat.name] = (root, base)
+            for s in cat.src:
+                Ls = self.by_name[s]
+                self.slot[s] = (root, base)
+                if Ls.op == "concat":
+                    place(Ls, root, base)
+                else:
+                    self.members.setdefault(root, []).append(s)
+                    if (Ls.op == "conv" and Ls.conv.relu and Ls.residual is None and not Ls.f32_out
+                            and len(uses[s]) == 1):
+                        self.in_place.add(s)
+                base += self.shape[s][3]
+
+        for L in self.layers:
+            u = uses.get(L.name, [])
+            if L.op == "concat" and not (len(u) == 1 and u[0].op == "concat"):
+                place(L, L.name, 0)
+
+    def _factor(self, name):
+        """Output factor of a tensor under the rules in the module docstring."""
+        if name in self._factors:
+            return self._factors[name]
+        if name in self.in_place or (name in self.slot and self.by_name[name].op == "concat"):
+            q = max(self._own_factor(m) for m in self.members[self.slot[name][0]])
+        else:
+            q = self._own_factor(name)
+        self._factors[name] = q
+        return q
+
+    def _own_factor(self, name):
+        m = self.maxima
+        if name == "input":
+            return q8.q8_factor(m["input"], 7)
+        L = self.by_name[name]
+        if L.op in ("maxpool", "avgpool"):
+            return self._factor(L.src[0])
+        if L.op == "concat":
+            return self._factor(name)
+        if L.residual is not None:
+            return q8.q8_factor(max(m[name + ":pre"], m[L.residual]), 8)
+        return q8.q8_factor(m[name], 8 if L.conv.relu else 7)
+
+    # ---- device work --------------------------------------------------------------------------------
     def forward(self, x_f32: torch.Tensor) -> Dict[str, torch.Tensor]:
-        """Enqueues the whole network on the current stream; returns the tensors (views of preallocated buffers)."""
+        """Enqueues the whole network on the current stream; returns the tensors (preallocated buffers, or
+        channel slices of a concat buffer)."""
         q8.q8_quantize_pad_channels(x_f32, self.c_pad_in, self.info["input"][1], q8.Q8_S8, out=self.bufs["input"])
         self.run_quantized()
         return self.bufs
@@ -89,10 +169,15 @@ class QuantNetwork:
             if L.op == "conv":
                 qc = self.convs[L.name]
                 res = b[L.residual] if L.residual is not None else None
-                q8.q8_conv2d(qc.desc, x, qc.w_q, qc.b_q, qc.scale, res, qc.res_scale, b[L.name], self.workspace)
+                y = b[self.slot[L.name][0]] if L.name in self.in_place else b[L.name]
+                q8.q8_conv2d(qc.desc, x, qc.w_q, qc.b_q, qc.scale, res, qc.res_scale, y, self.workspace)
             elif L.op == "maxpool":
                 q8.q8_maxpool2d(x, L.k, L.stride, L.pad, L.ceil_mode, out=b[L.name])
             elif L.op == "avgpool":
                 q8.q8_avgpool2d(x, L.k, L.stride, L.pad, L.ceil_mode, out=b[L.name])
             elif L.op == "concat":
-                q8.q8_concat([b[s] for s in L.src], [self.info[s][1] for s in L.src], self.info[L.name][1], out=b[L.name])
+                for s in L.src:
+                    if s in self.in_place or self.by_name[s].op == "concat":
+                        continue
+                    root, off = self.slot[s]
+                    q8.q8_concat_branch(b[s], self.info[s][1], self.info[L.name][1], b[root], off)

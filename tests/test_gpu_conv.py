@@ -55,6 +55,25 @@ CASES = [
     ("3x3s2_c32_k32_pad0", 3, 31, 34, 32, 32, 3, 3, 2, 0, 1, False, S8, None, False),
     ("2x2s2_c64_k64", 2, 20, 24, 64, 64, 2, 2, 2, 0, 1, False, U8, None, True),
     ("5x4s2_c16_k48_pad2", 2, 25, 26, 16, 48, 5, 4, 2, 2, 1, True, F32, None, False),
+    # tile widths that are not a power of two times 16/32/64, channel counts padded to a 128-wide block
+    ("1x1_c64_k80", 2, 37, 37, 64, 80, 1, 1, 1, 0, 1, False, U8, None, True),
+    ("1x7_c160_k160", 2, 17, 17, 160, 160, 1, 7, 1, (0, 3), 1, False, U8, None, True),
+    ("7x1_c160_k192_res", 2, 17, 17, 160, 192, 7, 1, 1, (3, 0), 1, False, U8, "u8", True),
+    ("1x1_c768_k320_s8", 2, 17, 17, 768, 320, 1, 1, 1, 0, 1, False, S8, "s8", False),
+    ("1x1_c1280_k448", 4, 8, 8, 1280, 448, 1, 1, 1, 0, 1, False, U8, None, True),
+    ("3x3_c448_k384", 4, 8, 8, 448, 384, 3, 3, 1, 1, 1, False, U8, None, True),
+    ("3x3_c80_k192_pad0", 2, 25, 25, 80, 192, 3, 3, 1, 0, 1, False, U8, None, True),
+    ("1x1_c96_k112_f32", 2, 20, 20, 96, 112, 1, 1, 1, 0, 1, False, F32, None, False),
+    ("1x1_c320_k144_raw", 2, 20, 20, 320, 144, 1, 1, 1, 0, 1, False, S32, None, False),
+    ("3x3_c192_k176", 2, 20, 20, 192, 176, 3, 3, 1, 1, 1, False, U8, "u8", True),
+    ("3x3_c128_k208", 2, 20, 20, 128, 208, 3, 3, 1, 1, 1, True, S8, None, False),
+    ("3x3_c128_k240", 2, 20, 20, 128, 240, 3, 3, 1, 1, 1, False, U8, None, True),
+    # images smaller than an accumulator tile: halo tiles with mostly empty rows instead of the fallback
+    ("3x3_5x5_pad0_c128_k256", 8, 5, 5, 128, 256, 3, 3, 1, 0, 1, False, U8, None, True),
+    ("3x3_3x3_pad0_c128_k256", 8, 3, 3, 128, 256, 3, 3, 1, 0, 1, False, U8, None, True),
+    ("3x3_3x3_pad1_c256_k84_f32", 8, 3, 3, 256, 84, 3, 3, 1, 1, 1, False, F32, None, False),
+    ("3x3_1x1_pad1_c256_k16_f32", 8, 1, 1, 256, 16, 3, 3, 1, 1, 1, False, F32, None, False),
+    ("3x3_1x1_pad1_c256_k126_f32", 32, 1, 1, 256, 126, 3, 3, 1, 1, 1, False, F32, None, False),
 ]
 
 

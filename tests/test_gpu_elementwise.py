@@ -100,7 +100,7 @@ def test_concat_bit_exact(q8, chans, signed):
 
 
 @pytest.mark.parametrize("k,st,pad,ceil", [(3, 2, 1, False), (2, 2, 0, True), (3, 1, 1, False), (3, 2, 0, False), (7, 1, 0, False)])
-@pytest.mark.parametrize("C", [64, 5])
+@pytest.mark.parametrize("C", [64, 48, 12, 5])
 def test_pools_bit_exact(q8, k, st, pad, ceil, C):
     g = np.random.default_rng(k * 10 + C)
     x = g.integers(0, 256, (2, 15, 13, C), dtype=np.uint8)
@@ -111,3 +111,29 @@ def test_pools_bit_exact(q8, k, st, pad, ceil, C):
     xs = x.view(np.int8)
     got = q8.q8_maxpool2d(_cuda(xs), (k, k), (st, st), (pad, pad), ceil).cpu().numpy()
     assert np.array_equal(got, o.pool(xs, "max", (k, k), (st, st), (pad, pad), ceil))
+    got = q8.q8_avgpool2d(_cuda(xs), (k, k), (st, st), (pad, pad), ceil).cpu().numpy()
+    assert np.array_equal(got, o.pool(xs, "avg", (k, k), (st, st), (pad, pad), ceil))
+
+
+@pytest.mark.parametrize("value,dt", [(255, np.uint8), (-128, np.int8), (127, np.int8)])
+def test_avgpool_extreme_codes_largest_window(q8, value, dt):
+    """A 16 x 16 window of one extreme code: the packed 16-bit lane sums may not carry into their neighbours."""
+    x = np.full((1, 17, 18, 32), value, dtype=dt)
+    x[0, 3, 4, 5] = 0
+    got = q8.q8_avgpool2d(_cuda(x), (16, 16), (1, 1), (0, 0), False).cpu().numpy()
+    assert np.array_equal(got, o.pool(x, "avg", (16, 16), (1, 1), (0, 0), False))
+
+
+@pytest.mark.parametrize("signed", [False, True])
+@pytest.mark.parametrize("ch,ldc,off", [(32, 96, 48), (20, 50, 7)])
+def test_concat_branch_writes_only_its_slice(q8, signed, ch, ldc, off):
+    g = np.random.default_rng(ch + ldc)
+    dt, lo, hi = (np.int8, -128, 128) if signed else (np.uint8, 0, 256)
+    x = g.integers(lo, hi, (3, 7, 5, ch)).astype(dt)
+    y0 = g.integers(lo, hi, (3, 7, 5, ldc)).astype(dt)
+    for q_in, q_out in ((0.02, 0.05), (0.05, 0.05)):
+        y = _cuda(y0.copy())
+        q8.q8_concat_branch(_cuda(x), q_in, q_out, y, off)
+        want = y0.copy()
+        want[..., off:off + ch] = o.concat([x], [q_in], q_out)
+        assert np.array_equal(y.cpu().numpy(), want)

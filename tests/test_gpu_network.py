@@ -83,3 +83,43 @@ def test_resnet50_logits_bit_exact_and_close_to_fp32(q8):
     rel = float(np.linalg.norm(logits - fp32) / np.linalg.norm(fp32))
     print(f"ResNet-50 int8 vs FP32 logits: relative L2 error {rel:.4f}")
     assert rel < 0.5
+
+
+def test_concat_modules_write_in_place_and_match_the_oracle(q8):
+    """Conv / pooled / nested-concat branches under one factor: every tensor of a small Inception-like net."""
+    from tests.test_oracle_network import _mini_inception
+    layers = _mini_inception()
+    got, want, ref, net = _run_both(q8, layers, hw=12, batch=3, calib_batches=2, seed=77)
+    assert {"m0_1x1", "m0_1x3", "m0_3x1", "m0_proj", "m1_3x3_s2"} == net.in_place
+    assert got["m0_1x3"].data_ptr() == got["m0"].data_ptr() + 16      # a slice of the concat buffer, not a copy
+
+
+def test_inception_v3_bit_exact_and_close_to_fp32(q8):
+    """Config 4 at batch 2: 95 affine layers, 15 concatenations (11 modules, 4 nested), 1x7 / 7x1 / 5x5 filters,
+    stride-2 reductions with a pooled branch, 3x3 average pools, dequantized logits."""
+    layers = nets.inception_v3()
+    got, want, ref, net = _run_both(q8, layers, hw=299, batch=2, calib_batches=2, seed=4000)
+    logits, fp32 = got["fc"].cpu().numpy().reshape(2, -1), ref["fc"].reshape(2, -1)
+    rel = float(np.linalg.norm(logits - fp32) / np.linalg.norm(fp32))
+    print(f"Inception-v3 int8 vs FP32 logits: relative L2 error {rel:.4f}")
+    assert rel < 0.5
+
+
+def test_ssd300_heads_bit_exact_and_close_to_fp32(q8):
+    """Config 5 at batch 1: VGG-16 base with ceil-mode pool3, dilation-6 fc6, extra stages, and the twelve
+    dequantized 3x3 heads (16/24 and 84/126 output channels) over 8732 boxes."""
+    layers = nets.ssd300()
+    got, want, ref, net = _run_both(q8, layers, hw=300, batch=1, calib_batches=1, seed=5000)
+    boxes = 0
+    num = den = 0.0
+    for L in layers:
+        if not L.f32_out:
+            continue
+        a, f = got[L.name].cpu().numpy().astype(np.float64), ref[L.name]
+        num, den = num + float(((a - f) ** 2).sum()), den + float((f.astype(np.float64) ** 2).sum())
+        if L.name.endswith("_loc"):
+            boxes += a.size // 4
+    assert boxes == 8732
+    rel = (num / den) ** 0.5
+    print(f"SSD-300 int8 vs FP32 head outputs: relative L2 error {rel:.4f}")
+    assert rel < 0.5
