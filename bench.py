@@ -158,10 +158,19 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------------------ GPU arm
-def resnet50_numbers(dev, batches=(64, 1), reps=20):
-    """Whole ResNet-50 (configs[2]) through the library: int8 forward of seeded synthetic images as one CUDA
-    graph replay per batch (input quantization included), He-init weights, BN folded, factors from a short
-    seeded calibration run (timing does not depend on the factors)."""
+# The paper's own whole-network int8 figures (Tables 1 and 2: one 18-core Xeon socket; throughput at this
+# batch, latency at batch 1).  Another machine: context beside the numbers below, not a target.
+NETWORKS = {
+    "resnet50": dict(fn="resnet50", hw=224, batch=64, seed=3000, paper_xeon={"images_per_s": 462, "latency_ms": 3.5}),
+    "inception_v3": dict(fn="inception_v3", hw=299, batch=64, seed=4000, paper_xeon={"images_per_s": 282, "latency_ms": 5.9}),
+    "ssd300": dict(fn="ssd300", hw=300, batch=32, seed=5000, paper_xeon={"images_per_s": 43, "latency_ms": 24.8}),
+}
+
+
+def network_numbers(dev, name, reps=20):
+    """One whole network (configs[2..4]) through the library: int8 forward of seeded synthetic images as one
+    CUDA graph replay per batch (input quantization included), He-init weights, BN folded, factors from a
+    short seeded calibration run (timing does not depend on the factors)."""
     import torch
     import paper_1805_08691_b200 as q8
     from paper_1805_08691_b200 import network, pipeline
@@ -170,7 +179,9 @@ def resnet50_numbers(dev, batches=(64, 1), reps=20):
     def cuda(a):
         return torch.from_numpy(np.ascontiguousarray(a)).to(dev)
 
-    layers = nets.resnet50()
+    cfg = NETWORKS[name]
+    hw = cfg["hw"]
+    layers = getattr(nets, cfg["fn"])()
     folded = {}
     for L in layers:
         if L.op != "conv":
@@ -179,15 +190,16 @@ def resnet50_numbers(dev, batches=(64, 1), reps=20):
         folded[L.name] = (q8.q8_fold_bn(cuda(sp.w), None, cuda(sp.gamma), cuda(sp.beta), cuda(sp.mean), cuda(sp.var), 1e-5)
                           if sp.bn else (cuda(sp.w), cuda(sp.b)))
     folded_np = {k: (w.cpu().numpy(), b.cpu().numpy()) for k, (w, b) in folded.items()}
-    acts = nets.fp32_forward(layers, nets.images(3010, 4, 224), folded_np, device=dev)
+    acts = nets.fp32_forward(layers, nets.images(cfg["seed"] + 10, 2, hw), folded_np, device=dev)
     cal = pipeline.Calibrator(sorted(acts), device=dev)
     for k, v in acts.items():
         cal.observe(k, cuda(v))
     maxima = cal.maxima()
-    out = {"macs_per_image": nets.macs(layers, 224), "launches_per_forward": 1 + sum(1 for _ in layers)}
-    for batch in batches:
-        net = network.QuantNetwork(layers, folded, maxima, (batch, 224, 224, 3), device=dev)
-        x = cuda(nets.images(3001, batch, 224))
+    del acts
+    out = {"macs_per_image": nets.macs(layers, hw), "paper_xeon": cfg["paper_xeon"]}
+    for batch in (cfg["batch"], 1):
+        net = network.QuantNetwork(layers, folded, maxima, (batch, hw, hw, 3), device=dev)
+        x = cuda(nets.images(cfg["seed"] + 1, batch, hw))
         net.forward(x)
         torch.cuda.synchronize()
         q8.q8_read_status()
@@ -206,7 +218,8 @@ def resnet50_numbers(dev, batches=(64, 1), reps=20):
         ms = e0.elapsed_time(e1) / reps
         out[f"batch{batch}"] = {"ms_per_forward": ms, "images_per_s": batch / ms * 1e3,
                                 "TOPS": 2.0 * out["macs_per_image"] * batch / ms / 1e9}
-        del net, g
+        del net, g, x
+    torch.cuda.empty_cache()
     return out
 
 
@@ -385,8 +398,8 @@ def run_ours(args):
             "gpu_launches": 3 * args.steps,
             "roofline": roofline, "kernels": kernels,
             "images_per_s": BATCH * world / ms_step * 1e3}
-    if world == 1 and not args.skip_resnet50:
-        line["resnet50"] = resnet50_numbers(dev)
+    if world == 1 and not args.skip_networks:
+        line["networks"] = {name: network_numbers(dev, name) for name in NETWORKS}
     if world == 1 and not args.skip_cpu_baseline:
         r = oracle_time_steps(steps=2, warmup=1)
         line["cpu_baseline"] = {"value": r["value"], "unit": UNIT, "cores": r["threads"], "kind": "oracle",
@@ -404,7 +417,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sets", type=int, default=6, help="rotating buffer sets (working set must exceed L2)")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
-    ap.add_argument("--skip-resnet50", action="store_true", help="leave out the whole-network ResNet-50 numbers")
+    ap.add_argument("--skip-networks", "--skip-resnet50", dest="skip_networks", action="store_true",
+                    help="leave out the whole-network numbers (ResNet-50, Inception-v3, SSD-300)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -689,6 +689,12 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
   const int total_tiles = p.m_tiles * p.n_tiles * p.splits;  // work items
   const int slots = G * p.nbuf;
 
+  // Programmatic dependent launch: the next kernel of the stream may be scheduled onto SMs as they fall idle
+  // (it waits below, like this one, before it touches global memory), and this kernel's own set-up (barriers,
+  // TMEM allocation, descriptor prefetch) runs while the previous kernel drains.  Both are no-ops for a
+  // launch without the attribute.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
   // Prologue.  Each control lane initialises the barriers it owns.  Warp 0 only signals the
   // start-up barrier (bar.arrive) and goes straight to its loads, so that the first bytes are on
   // their way while the others allocate TMEM and fetch bias and scale; everybody else waits on it.
@@ -702,6 +708,7 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
     else if (lane == 18) prefetch_tensormap(&tmB);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncwarp();
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // everything the previous kernel wrote is visible from here
     asm volatile("bar.arrive 1, %0;" ::"r"(nthreads) : "memory");
   } else {
     if (warp == 1) {
@@ -723,6 +730,7 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       tmem_relinquish();
     }
     if (p.a_mode == kAHalo && threadIdx.x >= 32 && threadIdx.x - 32 < p.taps) tap_shift16[threadIdx.x - 32] = p.tap_shift16[threadIdx.x - 32];
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     // bias and scale of every channel, once per CTA (zero beyond Cout; one scale replicated if per tensor)
     for (int i = threadIdx.x - 32; i < p.k_pad; i += nthreads - 32) {
       s_bias[i] = (p.bias && i < p.K) ? p.bias[i] : 0;
@@ -1154,7 +1162,20 @@ int launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtenso
     if (rc != Q8_OK) return rc;
     configured = true;
   }
-  kernel<<<grid, kCtrlThreads + G * kGroupThreads, dyn, stream>>>(tmA, tmB, tmRes, tmY, p);
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3((unsigned)(kCtrlThreads + G * kGroupThreads));
+  cfg.dynamicSmemBytes = dyn;
+  cfg.stream = stream;
+  // let this kernel's set-up overlap the tail of the kernel before it in the stream
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = tune_env("Q8_PDL", 1) ? 1 : 0;
+  int rc = check_cuda(cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, tmRes, tmY, p), "conv_umma: launch");
+  if (rc != Q8_OK) return rc;
   return check_launch("conv_umma_kernel");
 }
 

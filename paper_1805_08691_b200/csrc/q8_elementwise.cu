@@ -148,6 +148,25 @@ __global__ void __launch_bounds__(kThreads) quantize_pad_kernel(const float* __r
   }
 }
 
+// The same with one 16-byte store per thread: thread = (pixel, group of 16 output channels).  A warp reads
+// 32 consecutive pixels (contiguous floats when C <= 16) and writes 512 contiguous bytes.
+__global__ void __launch_bounds__(kThreads) quantize_pad16_kernel(const float* __restrict__ x, size_t pixels, int C,
+                                                                  int groups, float q, int lo, int hi,
+                                                                  uint4* __restrict__ z) {
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  const size_t total = pixels * (size_t)groups;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += nthreads) {
+    const size_t px = i / groups;
+    const int c0 = (int)(i - px * groups) * 16;
+    const float* src = x + px * C + c0;
+    int v[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v[j] = (c0 + j < C) ? quant1(__ldcs(src + j), q, lo, hi) : 0;
+    z[i] = make_uint4(pack4(v[0], v[1], v[2], v[3]), pack4(v[4], v[5], v[6], v[7]), pack4(v[8], v[9], v[10], v[11]),
+                      pack4(v[12], v[13], v[14], v[15]));
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Eq. (D): r = q * float(z), one fp32 multiply.
 // ---------------------------------------------------------------------------------------------
@@ -529,6 +548,12 @@ int q8_quantize_pad_channels(const float* x, size_t pixels, int C, int C_pad, fl
   if (out_type != Q8_U8 && out_type != Q8_S8) return fail(Q8_ERR_INVALID_ARG, "q8_quantize_pad_channels: bad out_type");
   if (pixels == 0) return Q8_OK;
   const int lo = out_type == Q8_U8 ? 0 : -128, hi = out_type == Q8_U8 ? 255 : 127;
+  if (C_pad % 16 == 0 && aligned16(z)) {
+    const int groups = C_pad / 16;
+    quantize_pad16_kernel<<<grid_for(pixels * groups, kThreads, 8), kThreads, 0, as_stream(stream)>>>(
+        x, pixels, C, groups, q, lo, hi, static_cast<uint4*>(z));
+    return check_launch("quantize_pad16_kernel");
+  }
   quantize_pad_kernel<unsigned char><<<grid_for(pixels * C_pad, kThreads, 8), kThreads, 0, as_stream(stream)>>>(
       x, pixels, C, C_pad, q, lo, hi, static_cast<unsigned char*>(z));
   return check_launch("quantize_pad_kernel");

@@ -52,12 +52,13 @@ def test_quantize_calibrated_extremes(q8):
     assert int(z.max()) == 255 and np.array_equal(z.cpu().numpy(), o.quantize(r, qf, o.U8))
 
 
-def test_quantize_pad_channels(q8):
-    g = np.random.default_rng(4)
-    x = g.standard_normal((2, 9, 7, 3)).astype(np.float32)
-    got = q8.q8_quantize_pad_channels(_cuda(x), 16, 0.02, 1).cpu().numpy()
-    assert got.shape == (2, 9, 7, 16)
-    assert np.array_equal(got[..., :3], o.quantize(x, 0.02, o.S8)) and np.all(got[..., 3:] == 0)
+@pytest.mark.parametrize("C,C_pad,out", [(3, 16, 1), (3, 16, 0), (20, 32, 1), (5, 8, 1), (16, 16, 0)])
+def test_quantize_pad_channels(q8, C, C_pad, out):
+    g = np.random.default_rng(4 + C)
+    x = (g.standard_normal((2, 37, 41, C)) * 2).astype(np.float32)
+    got = q8.q8_quantize_pad_channels(_cuda(x), C_pad, 0.02, out).cpu().numpy()
+    assert got.shape == (2, 37, 41, C_pad)
+    assert np.array_equal(got[..., :C], o.quantize(x, 0.02, o.S8 if out else o.U8)) and np.all(got[..., C:] == 0)
 
 
 @pytest.mark.parametrize("dt", [np.uint8, np.int8, np.int32])
