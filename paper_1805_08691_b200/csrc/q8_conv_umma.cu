@@ -368,6 +368,27 @@ __device__ __forceinline__ unsigned int pack4_sat(int z0, int z1, int z2, int z3
   return kSigned ? pack_sat_s8(z1, z0, pack_sat_s8(z3, z2, 0u)) : pack_sat_u8(z1, z0, pack_sat_u8(z3, z2, 0u));
 }
 
+// Packed fp32 arithmetic: two independent IEEE operations (round to nearest even, no contraction) in one
+// instruction slot.  The epilogue of a layer with a short reduction is bound by instruction issue.
+__device__ __forceinline__ unsigned long long pack_f2(float a, float b) {
+  unsigned long long d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(a), "f"(b));
+  return d;
+}
+__device__ __forceinline__ void unpack_f2(unsigned long long d, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(d));
+}
+__device__ __forceinline__ unsigned long long fmul2(unsigned long long a, unsigned long long b) {
+  unsigned long long d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ unsigned long long fsub2(unsigned long long a, unsigned long long b) {
+  unsigned long long d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
 // ------------------------------------------------------------------------------------------ epilogue
 struct EpiTile {
   const int* s_bias;       // smem, k_pad entries
@@ -421,16 +442,15 @@ __device__ __forceinline__ void epilogue_chunk(const UmmaParams& p, const EpiTil
     off ^= ((off >> 7) & (uint32_t)p.pmask) << 4;
     off += (uint32_t)pn * ((uint32_t)kBM << p.pw_shift);
   }
+  unsigned long long v2[8];  // v[2i], v[2i + 1]
   float v[16];
   {
     const float4* sp = reinterpret_cast<const float4*>(t.s_scale + nb);
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const float4 s = sp[j];
-      v[4 * j] = __fmul_rn(__int2float_rn(acc[4 * j]), s.x);
-      v[4 * j + 1] = __fmul_rn(__int2float_rn(acc[4 * j + 1]), s.y);
-      v[4 * j + 2] = __fmul_rn(__int2float_rn(acc[4 * j + 2]), s.z);
-      v[4 * j + 3] = __fmul_rn(__int2float_rn(acc[4 * j + 3]), s.w);
+      v2[2 * j] = fmul2(pack_f2(__int2float_rn(acc[4 * j]), __int2float_rn(acc[4 * j + 1])), pack_f2(s.x, s.y));
+      v2[2 * j + 1] = fmul2(pack_f2(__int2float_rn(acc[4 * j + 2]), __int2float_rn(acc[4 * j + 3])), pack_f2(s.z, s.w));
     }
   }
   if (kRes != kResNone) {
@@ -449,12 +469,23 @@ __device__ __forceinline__ void epilogue_chunk(const UmmaParams& p, const EpiTil
     // byte is first biased by 128
     const unsigned int sign_mask = p.res_signed ? 0x80808080u : 0u;
     const float magic = p.res_signed ? 8388736.0f : 8388608.0f;
+    const unsigned long long magic2 = pack_f2(magic, magic), rs2 = pack_f2(p.res_scale, p.res_scale);
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      const unsigned int w = rw[j >> 2] ^ sign_mask;
-      const float r = __fsub_rn(__uint_as_float(__byte_perm(w, 0x4B000000u, 0x7540u | (unsigned)(j & 3))), magic);
-      v[j] = __fadd_rn(v[j], __fmul_rn(r, p.res_scale));
+    for (int j = 0; j < 8; ++j) {
+      const unsigned int w = rw[j >> 1] ^ sign_mask;
+      const float r0 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7540u | (unsigned)((2 * j) & 3)));
+      const float r1 = __uint_as_float(__byte_perm(w, 0x4B000000u, 0x7540u | (unsigned)((2 * j + 1) & 3)));
+      // the sum stays scalar: the assembler contracts a packed multiply followed by a packed add into one
+      // fused operation (one rounding instead of two), which would break the two-rounding definition
+      float t0, t1;
+      unpack_f2(fmul2(fsub2(pack_f2(r0, r1), magic2), rs2), t0, t1);
+      unpack_f2(v2[j], v[2 * j], v[2 * j + 1]);
+      v[2 * j] = __fadd_rn(v[2 * j], t0);
+      v[2 * j + 1] = __fadd_rn(v[2 * j + 1], t1);
     }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) unpack_f2(v2[j], v[2 * j], v[2 * j + 1]);
   }
   if (kOut == Q8_F32) {
     if (p.relu) {

@@ -110,6 +110,36 @@ def test_conv_matches_oracle(q8, case, algo):
     assert np.array_equal(_bits(y.cpu().numpy()), _bits(want))
 
 
+@pytest.mark.parametrize("xs8", [False, True])
+@pytest.mark.parametrize("extra", [0, 1, 1 << 29])
+def test_short_reduction_extreme_accumulators(q8, xs8, extra):
+    """1x1, C = 64: accumulators at their bound (all-extreme inputs and weights) with biases that bring
+    |acc + bias| to 2^22 - 1, to 2^22 and to ~2^29: int -> float conversion and scaling of extreme values."""
+    N, H, W, C, K = 2, 12, 12, 64, 128
+    g = np.random.default_rng(5 + extra % 7)
+    x = g.integers(-128, 128, (N, H, W, C)).astype(np.int8) if xs8 else g.integers(0, 256, (N, H, W, C), dtype=np.uint8)
+    w = g.integers(-128, 128, (K, 1, 1, C)).astype(np.int8)
+    xmax = 128 if xs8 else 255
+    x[0, 0, 0, :] = -128 if xs8 else 255          # pixel 0 with filters 0 / 1 reaches -bound / +bound (s8: +bound - 64*128)
+    w[0], w[1] = -128, (-128 if xs8 else 127)
+    bound = C * xmax * 128
+    margin = (1 << 22) - 1 - bound + extra
+    bias = g.integers(-margin, margin + 1, K).astype(np.int64)
+    bias[0], bias[1], bias[2], bias[3] = (-margin if not xs8 else margin), margin, -margin, margin
+    bias = bias.astype(np.int32)
+    acc = o.conv_acc(x, w, bias, (1, 1), (0, 0), (1, 1), threads=4)
+    assert extra or np.abs(acc.astype(np.int64)).max() == (1 << 22) - 1
+    scale = np.float32(127.0 / (1 << 22)) if extra < 2 else np.float32(127.0 / (1 << 30))
+    resid = g.integers(0, 256, (N, H, W, K), dtype=np.uint8)
+    for ytype, res, relu in ((S8, None, False), (U8, resid, True), (F32, None, False)):
+        want = o.epilogue(acc, scale, res, 0.21 if res is not None else 0.0, relu, OT[ytype])
+        d = q8.make_conv_desc(N, H, W, C, K, 1, 1, (1, 1), (0, 0), (1, 1), S8 if xs8 else U8, U8, ytype, relu)
+        y = q8.q8_conv2d(d, _cuda(x), _cuda(w), _cuda(bias), torch.tensor([scale], device="cuda"),
+                         _cuda(res) if res is not None else None, 0.21 if res is not None else 0.0)
+        q8.q8_read_status()
+        assert np.array_equal(_bits(y.cpu().numpy()), _bits(want))
+
+
 def test_tensor_core_kernel_is_selected(q8):
     """The shapes of the paper's networks must run on tcgen05, not on the fallback."""
     for (N, H, W, C, K, R, S, st, pad) in [(32, 56, 56, 256, 64, 1, 1, 1, 0), (32, 56, 56, 64, 64, 3, 3, 1, 1),
