@@ -197,8 +197,21 @@ def network_numbers(dev, name, reps=20):
     maxima = cal.maxima()
     del acts
     out = {"macs_per_image": nets.macs(layers, hw), "paper_xeon": cfg["paper_xeon"]}
-    for batch in (cfg["batch"], 1):
-        net = network.QuantNetwork(layers, folded, maxima, (batch, hw, hw, 3), device=dev)
+    variants = [("batch%d" % cfg["batch"], cfg["batch"], layers), ("batch1", 1, layers)]
+    if name == "resnet50":
+        # the paper's "remove sparsity" graph rewrite: same FP32 function, 3 % fewer MACs (throughput is still
+        # quoted on the MACs of the original network)
+        from paper_1805_08691_b200 import graph
+        variants.append(("batch%d_sparsity_removed" % cfg["batch"], cfg["batch"], graph.remove_sparsity(layers)))
+    for key, batch, net_layers in variants:
+        if net_layers is not layers:
+            acts = nets.fp32_forward(net_layers, nets.images(cfg["seed"] + 10, 2, hw), folded_np, device=dev)
+            cal = pipeline.Calibrator(sorted(acts), device=dev)
+            for k, v in acts.items():
+                cal.observe(k, cuda(v))
+            maxima = cal.maxima()
+            del acts
+        net = network.QuantNetwork(net_layers, folded, maxima, (batch, hw, hw, 3), device=dev)
         x = cuda(nets.images(cfg["seed"] + 1, batch, hw))
         net.forward(x)
         torch.cuda.synchronize()
@@ -216,7 +229,7 @@ def network_numbers(dev, name, reps=20):
         e1.record()
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / reps
-        out[f"batch{batch}"] = {"ms_per_forward": ms, "images_per_s": batch / ms * 1e3,
+        out[key] = {"ms_per_forward": ms, "images_per_s": batch / ms * 1e3,
                                 "TOPS": 2.0 * out["macs_per_image"] * batch / ms / 1e9}
         del net, g, x
     torch.cuda.empty_cache()

@@ -68,6 +68,12 @@ int q8_read_status(void* stream);
  * NaN/Inf (largest bit pattern wins); q8_factor then reports it. */
 int q8_calibrate_maxabs(const float* x, size_t n, float* d_running_max, void* stream);
 
+/* The same for every row of a row-major [rows][cols] matrix: d_running_max[r] = max(d_running_max[r],
+ * max_c |x[r][c]|).  For one factor per output channel of a weight tensor [K][R*S*C] (the paper takes one
+ * factor per tensor; per-channel factors are an extension the convolution supports through scale_count = K).
+ * x: device.  d_running_max: device, rows fp32 values the caller zeroes first. */
+int q8_calibrate_maxabs_rows(const float* x, size_t rows, size_t cols, float* d_running_max, void* stream);
+
 /* Host helper: *q = maxabs / (2^p - 1) as one fp32 division; *q = 1 when
  * maxabs == 0.  p in [1,31].  Q8_ERR_NONFINITE if maxabs is NaN/Inf/negative. */
 int q8_factor(float maxabs, int p, float* q);
@@ -89,6 +95,12 @@ int q8_bias_factor(float q_x, float q_w, float* q_b);
  * (-128,127) for Q8_S8, (-2^31, 2^31-1) for Q8_S32.  fp32 IEEE division.  NaN
  * maps to 0.  x, z: device, n elements, same layout.  q must be finite, > 0. */
 int q8_quantize(const float* x, size_t n, float q, int out_type, void* z, void* stream);
+
+/* Eq. (Q) with one factor per row of a row-major [rows][cols] matrix: z[r][c] = clamp(Round(x[r][c] / q[r])).
+ * d_q: DEVICE array of rows factors, each finite and > 0 (not checked: a bad factor yields saturated or
+ * zero codes for its row).  out_type: Q8_U8, Q8_S8 or Q8_S32.  x, z: device, same layout. */
+int q8_quantize_rows(const float* x, size_t rows, size_t cols, const float* d_q, int out_type, void* z,
+                     void* stream);
 
 /* As q8_quantize for an NHWC tensor of `pixels` x C values, but the output has
  * C_pad >= C channels per pixel and channels C..C_pad-1 are written as 0 (the

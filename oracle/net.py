@@ -103,8 +103,10 @@ def _concat_groups(layers):
     return root, shared, leaves
 
 
-def network_prepare(layers, folded, maxima):
-    """Returns {layer name: dict} with the quantized parameters and the (type, factor) of every tensor."""
+def network_prepare(layers, folded, maxima, per_channel=False):
+    """Returns {layer name: dict} with the quantized parameters and the (type, factor) of every tensor.
+    per_channel: one weight factor per output channel, max|w[k]| / 127 (the paper takes one per tensor); bias
+    and requantisation multiplier of channel k then use q_w[k]."""
     root, shared, leaves = _concat_groups(layers)
     by_name = {L.name: L for L in layers}
     own = {}
@@ -138,9 +140,14 @@ def network_prepare(layers, folded, maxima):
         if L.op == "conv":
             w, b = folded[L.name]
             c_pad = -(-w.shape[-1] // 16) * 16
-            q_w = o.factor(o.maxabs(w), 7)
-            w_q = _pad_c(o.quantize(w, q_w, o.S8), c_pad)
-            b_q = o.quantize(b, o.bias_factor(q_in, q_w), o.S32)
+            if per_channel:
+                q_w = [o.factor(o.maxabs(w[k]), 7) for k in range(w.shape[0])]
+                w_q = _pad_c(np.stack([o.quantize(w[k], q_w[k], o.S8) for k in range(w.shape[0])]), c_pad)
+                b_q = np.concatenate([o.quantize(b[k:k + 1], o.bias_factor(q_in, q_w[k]), o.S32) for k in range(w.shape[0])])
+            else:
+                q_w = o.factor(o.maxabs(w), 7)
+                w_q = _pad_c(o.quantize(w, q_w, o.S8), c_pad)
+                b_q = o.quantize(b, o.bias_factor(q_in, q_w), o.S32)
             d = dict(w_q=w_q, b_q=b_q, q_w=q_w, res_scale=0.0, c_pad=c_pad)
             if L.f32_out:
                 d.update(y_type=o.F32, q_y=1.0)
@@ -151,7 +158,10 @@ def network_prepare(layers, folded, maxima):
                 d.update(y_type=o.U8, q_y=final_factor(L.name))
             else:
                 d.update(y_type=o.S8, q_y=final_factor(L.name))
-            d["scale"] = o.requant_scale(q_in, q_w, d["q_y"])
+            if per_channel:
+                d["scale"] = np.array([o.requant_scale(q_in, qk, d["q_y"]) for qk in q_w], dtype=np.float32)
+            else:
+                d["scale"] = o.requant_scale(q_in, q_w, d["q_y"])
             prep[L.name] = d
             info[L.name] = (d["y_type"], d["q_y"])
         elif L.op in ("maxpool", "avgpool"):

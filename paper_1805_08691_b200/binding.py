@@ -21,7 +21,7 @@ TORCH_DTYPES = {Q8_U8: torch.uint8, Q8_S8: torch.int8, Q8_S32: torch.int32, Q8_F
 EXPORTS = ["q8_version", "q8_last_error", "q8_read_status", "q8_calibrate_maxabs", "q8_factor", "q8_requant_scale",
            "q8_bias_factor", "q8_quantize", "q8_quantize_pad_channels", "q8_dequantize", "q8_fold_bn",
            "q8_conv2d_workspace_bytes", "q8_conv2d_query_algo", "q8_conv2d", "q8_static_workspace_bytes",
-           "q8_conv2d_static_workspace", "q8_concat", "q8_concat_branch", "q8_pool_out_extent",
+           "q8_conv2d_static_workspace", "q8_concat", "q8_concat_branch", "q8_calibrate_maxabs_rows", "q8_quantize_rows", "q8_pool_out_extent",
            "q8_maxpool2d", "q8_avgpool2d"]
 
 
@@ -68,6 +68,8 @@ lib.q8_conv2d.argtypes = [C.POINTER(q8_conv_desc), _vp, _vp, _vp, _vp, _vp, _f, 
 lib.q8_static_workspace_bytes.argtypes = []
 lib.q8_conv2d_static_workspace.argtypes = [C.POINTER(q8_conv_desc), _vp, _vp, _vp, _vp, _vp, _f, _vp, _vp]
 lib.q8_concat.argtypes = [_i, C.POINTER(_vp), _ip, _fp, _f, _i, _sz, _vp, _vp]
+lib.q8_calibrate_maxabs_rows.argtypes = [_vp, _sz, _sz, _vp, _vp]
+lib.q8_quantize_rows.argtypes = [_vp, _sz, _sz, _vp, _i, _vp, _vp]
 lib.q8_concat_branch.argtypes = [_vp, _i, _f, _f, _i, _sz, _vp, _i, _i, _vp]
 lib.q8_pool_out_extent.argtypes = [_i] * 5 + [_ip]
 lib.q8_maxpool2d.argtypes = [_vp, _i] + [_i] * 11 + [_vp, _vp]
@@ -228,6 +230,22 @@ def q8_concat(xs, in_factors, out_factor, out=None):
     _check(lib.q8_concat(len(xs), ptrs, (C.c_int * len(xs))(*chans), (C.c_float * len(xs))(*in_factors), out_factor, t,
                          pixels, _dev(out, "out"), _stream()))
     return out
+
+
+def q8_calibrate_maxabs_rows(x, running):
+    """running[r] = max(running[r], max|x[r, ...]|) for a tensor whose first dimension indexes the rows."""
+    rows = int(x.shape[0])
+    _check(lib.q8_calibrate_maxabs_rows(_dev(x, "x"), rows, x.numel() // max(rows, 1), _dev(running, "running"), _stream()))
+    return running
+
+
+def q8_quantize_rows(x, q_rows, out_type):
+    """Eq. (Q) with the device vector q_rows holding one factor per row (first dimension) of x."""
+    rows = int(x.shape[0])
+    z = torch.empty(x.shape, dtype=TORCH_DTYPES[out_type], device=x.device)
+    _check(lib.q8_quantize_rows(_dev(x, "x"), rows, x.numel() // max(rows, 1), _dev(q_rows, "q_rows"), out_type, _dev(z, "z"),
+                                _stream()))
+    return z
 
 
 def q8_concat_branch(x, in_factor, out_factor, out, c_offset):

@@ -134,6 +134,39 @@ __global__ void __launch_bounds__(kThreads) quantize32_vec_kernel(const float4* 
   }
 }
 
+// One factor per row: a block walks rows (grid stride), its threads the columns.
+__global__ void __launch_bounds__(256) maxabs_rows_kernel(const float* __restrict__ x, size_t rows, size_t cols,
+                                                          unsigned int* __restrict__ running) {
+  __shared__ unsigned int warp_max[8];
+  for (size_t r = blockIdx.x; r < rows; r += gridDim.x) {
+    const float* row = x + r * cols;
+    unsigned int m = 0;
+    for (size_t c = threadIdx.x; c < cols; c += blockDim.x) m = max(m, abs_bits(row[c]));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+#pragma unroll
+      for (int w = 1; w < 8; ++w) m = max(m, warp_max[w]);
+      atomicMax(running + r, m);
+    }
+    __syncthreads();
+  }
+}
+
+template <typename OutT>
+__global__ void __launch_bounds__(256) quantize_rows_kernel(const float* __restrict__ x, size_t rows, size_t cols,
+                                                            const float* __restrict__ q, int lo, int hi,
+                                                            OutT* __restrict__ z) {
+  for (size_t r = blockIdx.x; r < rows; r += gridDim.x) {
+    const float qr = q[r];
+    const float* row = x + r * cols;
+    OutT* out = z + r * cols;
+    for (size_t c = threadIdx.x; c < cols; c += blockDim.x) out[c] = (OutT)quant1(row[c], qr, lo, hi);
+  }
+}
+
 // NHWC pixels with C real channels -> C_pad channels, zeros appended.  One thread per pixel group.
 template <typename OutT>
 __global__ void __launch_bounds__(kThreads) quantize_pad_kernel(const float* __restrict__ x, size_t pixels, int C,
@@ -480,6 +513,29 @@ int q8_calibrate_maxabs(const float* x, size_t n, float* d_running_max, void* st
   int grid = grid_for((n + 3) / 4, kThreads * 4, 4);
   maxabs_kernel<<<grid, kThreads, 0, as_stream(stream)>>>(x, n, reinterpret_cast<unsigned int*>(d_running_max));
   return check_launch("maxabs_kernel");
+}
+
+int q8_calibrate_maxabs_rows(const float* x, size_t rows, size_t cols, float* d_running_max, void* stream) {
+  clear_error();
+  if (!d_running_max || (!x && rows && cols)) return fail(Q8_ERR_INVALID_ARG, "q8_calibrate_maxabs_rows: null pointer");
+  if (reinterpret_cast<uintptr_t>(x) & 3u) return fail(Q8_ERR_ALIGNMENT, "q8_calibrate_maxabs_rows: x not 4-byte aligned");
+  if (rows == 0 || cols == 0) return Q8_OK;
+  const int grid = (int)(rows < (size_t)sm_count() * 8 ? rows : (size_t)sm_count() * 8);
+  maxabs_rows_kernel<<<grid, 256, 0, as_stream(stream)>>>(x, rows, cols, reinterpret_cast<unsigned int*>(d_running_max));
+  return check_launch("maxabs_rows_kernel");
+}
+
+int q8_quantize_rows(const float* x, size_t rows, size_t cols, const float* d_q, int out_type, void* z, void* stream) {
+  clear_error();
+  if ((!x || !z || !d_q) && rows && cols) return fail(Q8_ERR_INVALID_ARG, "q8_quantize_rows: null pointer");
+  if (out_type != Q8_U8 && out_type != Q8_S8 && out_type != Q8_S32) return fail(Q8_ERR_INVALID_ARG, "q8_quantize_rows: bad out_type");
+  if (rows == 0 || cols == 0) return Q8_OK;
+  const int grid = (int)(rows < (size_t)sm_count() * 8 ? rows : (size_t)sm_count() * 8);
+  cudaStream_t s = as_stream(stream);
+  if (out_type == Q8_U8) quantize_rows_kernel<unsigned char><<<grid, 256, 0, s>>>(x, rows, cols, d_q, 0, 255, static_cast<unsigned char*>(z));
+  else if (out_type == Q8_S8) quantize_rows_kernel<signed char><<<grid, 256, 0, s>>>(x, rows, cols, d_q, -128, 127, static_cast<signed char*>(z));
+  else quantize_rows_kernel<int><<<grid, 256, 0, s>>>(x, rows, cols, d_q, INT32_MIN, INT32_MAX, static_cast<int*>(z));
+  return check_launch("quantize_rows_kernel");
 }
 
 int q8_factor(float maxabs, int p, float* q) {

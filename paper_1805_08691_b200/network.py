@@ -26,9 +26,11 @@ from . import pipeline
 
 
 class QuantNetwork:
-    def __init__(self, layers, folded: Dict[str, tuple], maxima: Dict[str, float], in_shape, device="cuda"):
+    def __init__(self, layers, folded: Dict[str, tuple], maxima: Dict[str, float], in_shape, device="cuda",
+                 per_channel=False):
         """folded[name] = (w KRSC, b K) FP32 device tensors; maxima: calibrated max-abs of "input", every layer
-        output and "<name>:pre" of residual convolutions; in_shape = (N, H, W, 3)."""
+        output and "<name>:pre" of residual convolutions; in_shape = (N, H, W, 3); per_channel: one weight
+        factor per output channel instead of one per tensor."""
         self.layers = layers
         self.maxima = maxima
         self.by_name = {L.name: L for L in layers}
@@ -63,7 +65,7 @@ class QuantNetwork:
                     root, off = self.slot[L.name]
                     ldc = self.shape[root][3]
                 qc = pipeline.prepare_conv(wf.contiguous(), bf, (n, h, w_, c), q_in, q_y, t_in, y_type, sp.relu, sp.stride,
-                                           sp.pad, sp.dil, q_res, res_type, ldc, off)
+                                           sp.pad, sp.dil, q_res, res_type, ldc, off, per_channel=per_channel)
                 self.convs[L.name] = qc
                 self.info[L.name] = (y_type, qc.q_y)
                 ws_bytes = max(ws_bytes, q8.q8_conv2d_workspace_bytes(qc.desc))

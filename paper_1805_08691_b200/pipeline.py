@@ -43,7 +43,7 @@ class QuantConv:
     w_q: torch.Tensor
     b_q: Optional[torch.Tensor]
     scale: torch.Tensor
-    q_w: float
+    q_w: object  # float, or a list of K floats with per-channel factors
     q_x: float
     q_y: float
     res_scale: float = 0.0
@@ -53,26 +53,38 @@ class QuantConv:
 
 
 def prepare_conv(w, b, in_shape, q_x, q_y, x_type=q8.Q8_U8, y_type=q8.Q8_U8, relu=True, stride=(1, 1), pad=(0, 0),
-                 dil=(1, 1), q_res=None, res_type=q8.Q8_U8, y_ldc=0, y_c_offset=0, algo=q8.Q8_ALGO_AUTO) -> QuantConv:
+                 dil=(1, 1), q_res=None, res_type=q8.Q8_U8, y_ldc=0, y_c_offset=0, algo=q8.Q8_ALGO_AUTO,
+                 per_channel=False) -> QuantConv:
     """w: folded FP32 weights KRSC on the device, b: folded FP32 bias [K] or None.
 
     q_y is the output factor; for y_type F32 the layer dequantizes (q_y is taken as 1).
+    per_channel: one weight factor per output channel (max|w[k]| / 127) instead of the paper's one per tensor;
+    the bias and the requantisation multiplier then carry the factor of their channel.
     """
     N, H, W, Cin = in_shape
     K, R, S, C2 = w.shape
     assert C2 == Cin
-    q_w = q8.q8_factor(tensor_maxabs(w), 7)
-    w_q = q8.q8_quantize(w, q_w, q8.Q8_S8)
-    b_q = None
-    if b is not None:
-        b_q = q8.q8_quantize(b, q8.q8_bias_factor(q_x, q_w), q8.Q8_S32)
     if y_type == q8.Q8_F32:
         q_y = 1.0
-    s = q8.q8_requant_scale(q_x, q_w, q_y)
-    scale = torch.tensor([s], dtype=torch.float32, device=w.device)
+    b_q = None
+    if per_channel:
+        slots = torch.zeros(K, dtype=torch.float32, device=w.device)
+        q8.q8_calibrate_maxabs_rows(w, slots)
+        q_w = [q8.q8_factor(m, 7) for m in slots.cpu().tolist()]
+        w_q = q8.q8_quantize_rows(w, torch.tensor(q_w, dtype=torch.float32, device=w.device), q8.Q8_S8)
+        if b is not None:
+            q_b = torch.tensor([q8.q8_bias_factor(q_x, qk) for qk in q_w], dtype=torch.float32, device=w.device)
+            b_q = q8.q8_quantize_rows(b.reshape(K, 1).contiguous(), q_b, q8.Q8_S32).reshape(K)
+        scale = torch.tensor([q8.q8_requant_scale(q_x, qk, q_y) for qk in q_w], dtype=torch.float32, device=w.device)
+    else:
+        q_w = q8.q8_factor(tensor_maxabs(w), 7)
+        w_q = q8.q8_quantize(w, q_w, q8.Q8_S8)
+        if b is not None:
+            b_q = q8.q8_quantize(b, q8.q8_bias_factor(q_x, q_w), q8.Q8_S32)
+        scale = torch.tensor([q8.q8_requant_scale(q_x, q_w, q_y)], dtype=torch.float32, device=w.device)
     res_scale = q8.q8_requant_scale(q_res, 1.0, q_y) if q_res is not None else 0.0
-    desc = q8.make_conv_desc(N, H, W, Cin, K, R, S, stride, pad, dil, x_type, res_type, y_type, relu, 1, y_ldc,
-                             y_c_offset, algo)
+    desc = q8.make_conv_desc(N, H, W, Cin, K, R, S, stride, pad, dil, x_type, res_type, y_type, relu,
+                             K if per_channel else 1, y_ldc, y_c_offset, algo)
     return QuantConv(desc, w_q, b_q, scale, q_w, q_x, q_y, res_scale)
 
 

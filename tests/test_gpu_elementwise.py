@@ -138,3 +138,18 @@ def test_concat_branch_writes_only_its_slice(q8, signed, ch, ldc, off):
         want = y0.copy()
         want[..., off:off + ch] = o.concat([x], [q_in], q_out)
         assert np.array_equal(y.cpu().numpy(), want)
+
+
+@pytest.mark.parametrize("rows,cols", [(1, 1), (7, 33), (300, 1153), (2048, 64)])
+def test_per_row_maxabs_and_quantize(q8, rows, cols):
+    g = np.random.default_rng(rows + cols)
+    x = (g.standard_normal((rows, cols)) * g.uniform(0.01, 3.0, (rows, 1))).astype(np.float32)
+    running = torch.full((rows,), 0.001, dtype=torch.float32, device="cuda")
+    q8.q8_calibrate_maxabs_rows(_cuda(x), running)
+    want = np.array([o.maxabs(x[r], init=0.001) for r in range(rows)], dtype=np.float32)
+    assert np.array_equal(running.cpu().numpy(), want)
+    q = np.array([o.factor(m, 7) for m in want], dtype=np.float32)
+    for t, ot in ((1, o.S8), (0, o.U8), (2, o.S32)):
+        qq = q if t != 2 else (q * np.float32(1e-3)).astype(np.float32)
+        got = q8.q8_quantize_rows(_cuda(x), _cuda(qq), t).cpu().numpy()
+        assert np.array_equal(got, np.stack([o.quantize(x[r], float(qq[r]), ot) for r in range(rows)]))

@@ -19,7 +19,7 @@ def _cuda(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
-def _run_both(q8, layers, hw, batch, calib_batches, seed, check_layers=None):
+def _run_both(q8, layers, hw, batch, calib_batches, seed, check_layers=None, per_channel=False):
     from paper_1805_08691_b200 import network, pipeline
     # fold BN on both sides, must agree bit for bit
     folded_o, folded_g = {}, {}
@@ -52,9 +52,9 @@ def _run_both(q8, layers, hw, batch, calib_batches, seed, check_layers=None):
     assert max_g == max_o
     # prepare and run
     x = nets.images(seed + 1, batch, hw)
-    prep, info = oracle_net.network_prepare(layers, folded_o, max_o)
+    prep, info = oracle_net.network_prepare(layers, folded_o, max_o, per_channel)
     want = oracle_net.network_forward(layers, prep, info, x, threads=batch)
-    net = network.QuantNetwork(layers, folded_g, max_g, x.shape)
+    net = network.QuantNetwork(layers, folded_g, max_g, x.shape, per_channel=per_channel)
     got = net.forward(_cuda(x))
     q8.q8_read_status()
     for L in layers:
@@ -72,6 +72,14 @@ def _run_both(q8, layers, hw, batch, calib_batches, seed, check_layers=None):
 def test_bottleneck_stack_every_layer(q8):
     layers = nets.bottleneck_stack(C=64, blocks=2)
     _run_both(q8, layers, hw=32, batch=3, calib_batches=2, seed=3100)
+
+
+def test_per_channel_weight_factors_every_layer(q8):
+    """One weight factor per output channel (scale_count = K) through residual blocks and concat modules."""
+    from tests.test_oracle_network import _mini_inception
+    _run_both(q8, nets.bottleneck_stack(C=64, blocks=2), hw=32, batch=2, calib_batches=2, seed=3100, per_channel=True)
+    got, want, ref, net = _run_both(q8, _mini_inception(), hw=12, batch=2, calib_batches=2, seed=77, per_channel=True)
+    assert net.convs["m0_1x3"].scale.numel() == 16
 
 
 def test_resnet50_logits_bit_exact_and_close_to_fp32(q8):
@@ -123,3 +131,12 @@ def test_ssd300_heads_bit_exact_and_close_to_fp32(q8):
     rel = (num / den) ** 0.5
     print(f"SSD-300 int8 vs FP32 head outputs: relative L2 error {rel:.4f}")
     assert rel < 0.5
+
+
+def test_resnet50_with_sparsity_removed_bit_exact(q8):
+    """The rewritten ResNet-50 (stride moved into the producing 1x1, 1x1 stride-2 pooling on the skip branch)."""
+    from paper_1805_08691_b200 import graph
+    layers = graph.remove_sparsity(nets.resnet50())
+    got, want, ref, net = _run_both(q8, layers, hw=224, batch=2, calib_batches=2, seed=3000)
+    logits, fp32 = got["fc1000"].cpu().numpy().reshape(2, -1), ref["fc1000"].reshape(2, -1)
+    assert float(np.linalg.norm(logits - fp32) / np.linalg.norm(fp32)) < 0.5

@@ -121,3 +121,34 @@ def test_layer_lists_match_the_published_architectures():
     fc6 = next(L for L in ssd if L.name == "fc6").conv
     assert (fc6.R, fc6.dil, fc6.pad) == (3, (6, 6), (6, 6))
     assert next(L for L in ssd if L.name == "pool3").ceil_mode
+
+
+def test_per_channel_weight_factors():
+    """One factor per output channel: every channel uses its full code range, the multiplier and the bias follow
+    the channel's factor, and the quantized run tracks FP32 at least as well as with one factor per tensor."""
+    layers = nets.bottleneck_stack(C=16, blocks=2)
+    folded = _fold(layers)
+    maxima = _calibrate(layers, folded, 31, 2, 16)
+    pt, info_t = oracle_net.network_prepare(layers, folded, maxima)
+    pc, info_c = oracle_net.network_prepare(layers, folded, maxima, per_channel=True)
+    assert info_t == info_c                              # activation factors do not depend on the weight factors
+    name = "blk0_branch2b"
+    w, b = folded[name]
+    d = pc[name]
+    K = w.shape[0]
+    assert len(d["q_w"]) == K and d["scale"].shape == (K,)
+    q_in = info_c["blk0_branch2a"][1]
+    for k in range(K):
+        assert d["q_w"][k] == o.factor(o.maxabs(w[k]), 7)
+        assert np.abs(d["w_q"][k].astype(np.int32)).max() == 127
+        assert d["scale"][k] == o.requant_scale(q_in, d["q_w"][k], d["q_y"])
+        assert d["b_q"][k] == o.quantize(b[k:k + 1], o.bias_factor(q_in, d["q_w"][k]), o.S32)[0]
+    assert max(d["q_w"]) == pt[name]["q_w"]              # the per-tensor factor is the largest channel factor
+    x = nets.images(32, 2, 16)
+    ref = nets.fp32_forward(layers, x, folded)
+    out_t = oracle_net.network_forward(layers, pt, info_t, x)
+    out_c = oracle_net.network_forward(layers, pc, info_c, x)
+    last = layers[-1].name
+    err_t = _rel(o.dequantize(out_t[last], info_t[last][1]), ref[last])
+    err_c = _rel(o.dequantize(out_c[last], info_c[last][1]), ref[last])
+    assert err_c < 0.12 and err_c <= err_t * 1.05
