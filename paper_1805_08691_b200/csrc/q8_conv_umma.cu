@@ -112,7 +112,8 @@ struct UmmaParams {
   unsigned int desc_hi;      // high word of the shared-memory matrix descriptors
   unsigned int a_sub_bytes;  // plain/im2col: one 128 x bk block; halo: bytes of one patch load
   unsigned int b_tile_bytes; // bn * bk
-  unsigned int b_sub_bytes;  // b_tile_bytes rounded up to 1 KiB (placement inside a stage / the ring)
+  unsigned int b_sub_bytes;  // b_tile_bytes rounded up to 1 KiB (placement inside a stage); ring: one ring stage
+  int b_T, b_chunks;         // weight ring: filter taps per ring stage (one TMA operation), stages per channel block
   unsigned int a_stage_bytes;
   unsigned int tile8_bytes;
   unsigned int res_tx_bytes; // bytes one residual tile load delivers
@@ -589,7 +590,8 @@ __device__ __forceinline__ bool mma_role(const UmmaParams& p, const MmaRoleArgs&
   const bool halo = p.a_mode == kAHalo, ring = p.b_mode == kBRing, b_in_stage = p.b_mode == kBStage;
   // ring positions of tile lt = who, and how far the other lanes' tiles move them between two of ours
   const uint32_t spt = halo ? (uint32_t)c_blocks : (uint32_t)((k_iters + kb - 1) / kb);  // A stages per tile
-  const uint32_t bpt = (uint32_t)(taps * c_blocks);                                       // ring tiles per tile
+  const int bT = p.b_T;
+  const uint32_t bpt = (uint32_t)(p.b_chunks * c_blocks);                                 // ring stages per tile
   const uint32_t skip_a = (kMmaWarps - 1) * spt, skip_b = (kMmaWarps - 1) * bpt;
   uint32_t stage = ((uint32_t)who * spt) % nstages, phase = (((uint32_t)who * spt) / nstages) & 1u;
   uint32_t bs = 0, bphase = 0;
@@ -619,13 +621,29 @@ __device__ __forceinline__ bool mma_role(const UmmaParams& p, const MmaRoleArgs&
         const bool last_cb = cb == c_blocks - 1;
         if (last_cb && !ring) mbar_arrive(turn_next);  // this tile's last wait is behind us
         tcgen05_fence_after();
-        if (ring) {
+        if (ring && bT == 1) {
+          // (kept apart from the multi-tap loop below: every extra instruction of this lone lane costs ~6 cycles)
           for (int tap = 0; tap < taps; ++tap) {
             if (!mbar_wait(r.b_full + bs * 8u, bphase, r.abortp)) return false;
             if (last_cb && tap == taps - 1) mbar_arrive(turn_next);
             tcgen05_fence_after();
             umma_i8_block<kSteps>(d_tmem, a_d + r.tap_shift16[tap], bring_d, idesc, accum);
             accum = 1;
+            umma_commit(r.b_empty + bs * 8u);
+            bring_d += bsub16;
+            if (++bs == nbst) { bs = 0; bphase ^= 1u; bring_d = bring_d0; }
+          }
+        } else if (ring) {
+          for (int tap0 = 0; tap0 < taps; tap0 += bT) {
+            if (!mbar_wait(r.b_full + bs * 8u, bphase, r.abortp)) return false;
+            if (last_cb && tap0 + bT >= taps) mbar_arrive(turn_next);
+            tcgen05_fence_after();
+            const int nt = min(bT, taps - tap0);
+            uint64_t bd = bring_d;
+            for (int t = 0; t < nt; ++t, bd += btile16) {
+              umma_i8_block<kSteps>(d_tmem, a_d + r.tap_shift16[tap0 + t], bd, idesc, accum);
+              accum = 1;
+            }
             umma_commit(r.b_empty + bs * 8u);
             bring_d += bsub16;
             if (++bs == nbst) { bs = 0; bphase ^= 1u; bring_d = bring_d0; }
@@ -803,6 +821,7 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       }
     }
     if (p.a_mode == kAHalo) {
+      const uint32_t b_tx = (uint32_t)p.b_T * p.b_tile_bytes;
       for (; ti.tile < total_tiles && ok; ti.next(p)) {
         const int n0 = ti.nt * p.bn, q0 = ti.qt * p.tw - p.pad_w, p0 = ti.pt * p.th * p.stride_h - p.pad_h;
         for (int c = 0; c < p.C_pad && ok; c += p.bk) {
@@ -813,11 +832,13 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
           a_dst += p.a_stage_bytes;
           if (++stage == nstages) { stage = 0; phase ^= 1u; a_dst = a0; }
           if (p.b_mode == kBRing) {
-            for (int tap = 0; tap < p.taps; ++tap) {
+            // one operation brings the weight tiles of b_T taps (a box that runs past the last tap is zero filled
+            // and still counts in full): the copy engine spends ~600 cycles per operation whatever its size
+            for (int tap = 0; tap < p.taps; tap += p.b_T) {
               if (!mbar_wait(bempty0 + bs * 8u, bphase ^ 1u, abortp)) { ok = false; break; }
               const uint32_t bbar = bfull0 + bs * 8u;
-              mbar_arrive_expect_tx(bbar, p.b_tile_bytes);
-              tma_load_3d(b_dst, &tmB, bbar, c, tap, n0);
+              mbar_arrive_expect_tx(bbar, b_tx);
+              tma_load_3d(b_dst, &tmB, bbar, c, n0, tap);
               b_dst += p.b_sub_bytes;
               if (++bs == nbst) { bs = 0; bphase ^= 1u; b_dst = bring0; }
             }
@@ -1397,6 +1418,8 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
   const bool resident = tune_env("Q8_BRES", (b_all <= 80u * 1024u && p.taps <= 256 && p.b_tile_bytes % (8u * BK) == 0) ? 1 : 0) != 0;
   p.b_mode = resident ? kBResident : (p.a_mode == kAHalo ? kBRing : kBStage);
   const unsigned bres_bytes = resident ? round_up(b_all, 1024u) : 0u;
+  p.b_T = 1;
+  p.b_chunks = p.taps;
   unsigned min_pipe;
   if (p.a_mode == kAHalo) {
     // the taps read up to (ext_h * twb + ext_w) pixels beyond accumulator row 127
@@ -1404,7 +1427,24 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
     p.a_sub_bytes = (unsigned)(BK * ht.twb * ht.hb);
     p.a_stage_bytes = round_up(reach > p.a_sub_bytes ? reach : p.a_sub_bytes, 1024u);
     p.kb = 1;
-    min_pipe = 2u * p.a_stage_bytes + (p.b_mode == kBRing ? 3u * p.b_sub_bytes : 0u);
+    // (measured: a gain with four accumulators, i.e. tiles up to 128 columns; a loss with two)
+    if (p.b_mode == kBRing && p.b_tile_bytes % (8u * BK) == 0 && p.nacc >= 4) {
+      // Weight ring stages of several filter taps, one TMA operation each (the copy engine spends ~600 cycles
+      // per operation whatever its size): as many taps as fit in about 48 KiB while two such stages fit beside
+      // two activation stages and one tile buffer per epilogue group, spread evenly over a channel block.
+      const unsigned fixed = bres_bytes + (use_bufs ? (unsigned)G * p.tile8_bytes : 0u) + 2u * p.a_stage_bytes;
+      const unsigned avail = budget > fixed ? budget - fixed : 0u;
+      int T = (int)(48u * 1024u / p.b_tile_bytes);
+      if (T > (int)(avail / (2u * p.b_tile_bytes))) T = (int)(avail / (2u * p.b_tile_bytes));
+      T = tune_env("Q8_BT", T);
+      if (T > p.taps) T = p.taps;
+      if (T < 1) T = 1;
+      p.b_chunks = (p.taps + T - 1) / T;
+      p.b_T = (p.taps + p.b_chunks - 1) / p.b_chunks;
+      p.b_chunks = (p.taps + p.b_T - 1) / p.b_T;
+      p.b_sub_bytes = round_up((unsigned)p.b_T * p.b_tile_bytes, 1024u);
+    }
+    min_pipe = 2u * p.a_stage_bytes + (p.b_mode == kBRing ? (p.b_T > 1 ? 2u : 3u) * p.b_sub_bytes : 0u);
   } else {
     p.a_sub_bytes = (unsigned)(kBM * BK);
     const unsigned unit = p.a_sub_bytes + (p.b_mode == kBStage ? p.b_sub_bytes : 0u);
@@ -1485,6 +1525,13 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
     cuuint64_t dims[3] = {(cuuint64_t)d.C, (cuuint64_t)d.K, (cuuint64_t)p.taps};
     cuuint64_t strides[2] = {(cuuint64_t)p.taps * d.C, (cuuint64_t)d.C};
     cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)BN, (cuuint32_t)p.taps};
+    cr = fn.tiled(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(a.w), dims, strides, box, ones,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else if (p.b_mode == kBRing) {
+    // (C, K, taps) view: one box brings bn rows of b_T consecutive taps, one K-major tile per tap
+    cuuint64_t dims[3] = {(cuuint64_t)d.C, (cuuint64_t)d.K, (cuuint64_t)p.taps};
+    cuuint64_t strides[2] = {(cuuint64_t)p.taps * d.C, (cuuint64_t)d.C};
+    cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)BN, (cuuint32_t)p.b_T};
     cr = fn.tiled(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(a.w), dims, strides, box, ones,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   } else {
