@@ -158,6 +158,58 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------------------ GPU arm
+def bandwidth_kernel_numbers(dev, peak_gbs, reps=20):
+    """The memory-bound kernels of the path on tensors larger than L2: algorithmic bytes (max-abs 4 B/elem,
+    quantize and dequantize 5, concat 2, pooling input + output) over the CUDA-event time, against the measured
+    copy bandwidth."""
+    import torch
+    import paper_1805_08691_b200 as q8
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps * 1e-3
+
+    out = {}
+
+    def report(name, nbytes, fn):
+        t = timed(fn)
+        out[name] = {"GB/s": nbytes / t / 1e9, "frac": nbytes / t / 1e9 / peak_gbs, "us": t * 1e6}
+
+    n = 64 * 112 * 112 * 64 * 2                      # 102.8 M elements: conv1 output of two ResNet-50 batches
+    x = torch.randn(n, device=dev)
+    slot = torch.zeros(1, device=dev)
+    z = torch.empty(n, dtype=torch.uint8, device=dev)
+    r = torch.empty(n, dtype=torch.float32, device=dev)
+    report("maxabs", n * 4, lambda: q8.q8_calibrate_maxabs(x, slot))
+    report("quantize_u8", n * 5, lambda: q8.q8_quantize(x, 0.02, q8.Q8_U8, z))
+    report("dequantize_u8", n * 5, lambda: q8.q8_dequantize(z, 0.02, r))
+    del r
+    img = torch.randn((4 * 64, 224, 224, 3), device=dev)   # 154 MB fp32 in, 206 MB s8 out
+    zi = torch.empty((4 * 64, 224, 224, 16), dtype=torch.int8, device=dev)
+    report("quantize_pad_3_to_16", img.numel() * 4 + zi.numel(), lambda: q8.q8_quantize_pad_channels(img, 16, 0.02, q8.Q8_S8, out=zi))
+    del img, zi
+    rows = n // 2 // 192
+    a = z[:rows * 192].view(rows, 192)
+    b = z[n // 2:n // 2 + rows * 192].view(rows, 192)
+    cat = torch.empty((rows, 384), dtype=torch.uint8, device=dev)
+    report("concat_requant", rows * 384 * 2, lambda: q8.q8_concat([a, b], [0.01, 0.02], 0.02, out=cat))
+    xp = z.view(2 * 64, 112, 112, 64)
+    yp = torch.empty((2 * 64, 56, 56, 64), dtype=torch.uint8, device=dev)
+    report("maxpool_3x3_s2", xp.numel() + yp.numel(), lambda: q8.q8_maxpool2d(xp, (3, 3), (2, 2), (1, 1), out=yp))
+    xa = z[:4 * 64 * 35 * 35 * 288].view(4 * 64, 35, 35, 288)
+    ya = torch.empty_like(xa)
+    report("avgpool_3x3_s1", xa.numel() * 2, lambda: q8.q8_avgpool2d(xa, (3, 3), (1, 1), (1, 1), out=ya))
+    return out
+
+
 # The paper's own whole-network int8 figures (Tables 1 and 2: one 18-core Xeon socket; throughput at this
 # batch, latency at batch 1).  Another machine: context beside the numbers below, not a target.
 NETWORKS = {
@@ -412,6 +464,7 @@ def run_ours(args):
             "roofline": roofline, "kernels": kernels,
             "images_per_s": BATCH * world / ms_step * 1e3}
     if world == 1 and not args.skip_networks:
+        line["bandwidth_kernels"] = bandwidth_kernel_numbers(dev, peaks["hbm_gbs"])
         line["networks"] = {name: network_numbers(dev, name) for name in NETWORKS}
     if world == 1 and not args.skip_cpu_baseline:
         r = oracle_time_steps(steps=2, warmup=1)

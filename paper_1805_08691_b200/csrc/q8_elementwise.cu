@@ -200,6 +200,20 @@ __global__ void __launch_bounds__(kThreads) quantize_pad16_kernel(const float* _
   }
 }
 
+// Images: 3 channels -> 16.  Four pixels per thread: three 16-byte loads (12 floats), four 16-byte stores.
+__global__ void __launch_bounds__(kThreads) quantize_pad3_kernel(const float4* __restrict__ x, size_t quads, float q, int lo,
+                                                                 int hi, uint4* __restrict__ z) {
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < quads; i += nthreads) {
+    const float4 a = __ldcs(x + 3 * i), b = __ldcs(x + 3 * i + 1), c = __ldcs(x + 3 * i + 2);
+    uint4* out = z + 4 * i;
+    __stcs(out, make_uint4(pack4(quant1(a.x, q, lo, hi), quant1(a.y, q, lo, hi), quant1(a.z, q, lo, hi), 0), 0u, 0u, 0u));
+    __stcs(out + 1, make_uint4(pack4(quant1(a.w, q, lo, hi), quant1(b.x, q, lo, hi), quant1(b.y, q, lo, hi), 0), 0u, 0u, 0u));
+    __stcs(out + 2, make_uint4(pack4(quant1(b.z, q, lo, hi), quant1(b.w, q, lo, hi), quant1(c.x, q, lo, hi), 0), 0u, 0u, 0u));
+    __stcs(out + 3, make_uint4(pack4(quant1(c.y, q, lo, hi), quant1(c.z, q, lo, hi), quant1(c.w, q, lo, hi), 0), 0u, 0u, 0u));
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Eq. (D): r = q * float(z), one fp32 multiply.
 // ---------------------------------------------------------------------------------------------
@@ -286,9 +300,14 @@ __global__ void __launch_bounds__(kThreads) concat_vec_kernel(const uint4* __res
                                                               uint4* __restrict__ y) {
   const size_t total = pixels * (size_t)cvec;
   const size_t nthreads = (size_t)gridDim.x * blockDim.x;
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += nthreads) {
-    size_t px = i / cvec;
-    int c = (int)(i - px * cvec);
+  // (pixel, 16-byte group) of this thread's element, advanced by additions: one division per thread
+  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  size_t px = i / cvec;
+  int c = (int)(i - px * cvec);
+  const size_t dpx = nthreads / cvec;
+  const int dc = (int)(nthreads - dpx * cvec);
+#pragma unroll 4
+  for (; i < total; i += nthreads) {
     uint4 v = __ldcs(x + i);
     if (!copy_only) {
       v.x = requant_word<kSigned>(v.x, s);
@@ -297,6 +316,9 @@ __global__ void __launch_bounds__(kThreads) concat_vec_kernel(const uint4* __res
       v.w = requant_word<kSigned>(v.w, s);
     }
     y[px * ctot_vec + coff_vec + c] = v;
+    px += dpx;
+    c += dc;
+    if (c >= cvec) { c -= cvec; ++px; }
   }
 }
 
@@ -452,6 +474,92 @@ __global__ void __launch_bounds__(256) avgpool16_kernel(const uint4* __restrict_
   }
 }
 
+// 3x3 and 2x2 windows, 16 channels per thread, 32-bit index arithmetic: the window is unrolled so that all of
+// its (predicated) 16-byte loads are in flight together; cells outside the image do not take part.
+template <bool kSigned, bool kAvg, int KH, int KW>
+__global__ void __launch_bounds__(256) pool16_window_kernel(const uint4* __restrict__ x, int H, int W, int cg, int st_h,
+                                                            int st_w, int pad_h, int pad_w, int P, int Q, float inv,
+                                                            unsigned int total, uint4* __restrict__ y) {
+  // Average: the result is a function of the window sum alone, so each block tabulates it once, with the
+  // defining arithmetic clamp(Round(float(sum) * inv)); entry j is the code for sum j - kOff.  The kernel is
+  // bound by integer instructions, and the table replaces seven of them per element by one shared-memory load.
+  constexpr int kOff = kSigned ? 128 * KH * KW : 0;
+  constexpr int kEntries = 255 * KH * KW + 1;
+  __shared__ unsigned char table[kAvg ? kEntries : 1];
+  if (kAvg) {
+    for (int j = threadIdx.x; j < kEntries; j += blockDim.x) {
+      const int z = __float2int_rn(__fmul_rn((float)(j - kOff), inv));
+      table[j] = (unsigned char)(kSigned ? min(max(z, -128), 127) : min(max(z, 0), 255));
+    }
+    __syncthreads();
+  }
+  const unsigned int nthreads = gridDim.x * blockDim.x;
+  for (unsigned int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += nthreads) {
+    const unsigned int c = i % (unsigned)cg;
+    unsigned int t = i / (unsigned)cg;
+    const int q = (int)(t % (unsigned)Q);
+    t /= (unsigned)Q;
+    const int p = (int)(t % (unsigned)P);
+    const unsigned int n = t / (unsigned)P;
+    const int h0 = p * st_h - pad_h, w0 = q * st_w - pad_w;
+    const uint4* img = x + (size_t)n * H * W * cg + c;
+    uint4 v[KH * KW];
+    bool ok[KH * KW];
+#pragma unroll
+    for (int r = 0; r < KH; ++r)
+#pragma unroll
+      for (int s = 0; s < KW; ++s) {
+        const int h = h0 + r, w = w0 + s;
+        ok[r * KW + s] = h >= 0 && h < H && w >= 0 && w < W;
+        v[r * KW + s] = ok[r * KW + s] ? __ldg(img + ((size_t)h * W + w) * cg) : make_uint4(0u, 0u, 0u, 0u);
+      }
+    if (!kAvg) {
+      const unsigned int init = kSigned ? 0x80808080u : 0u;
+      uint4 m = make_uint4(init, init, init, init);
+#pragma unroll
+      for (int k = 0; k < KH * KW; ++k) {
+        if (!ok[k]) continue;
+        if (kSigned) { m.x = __vmaxs4(m.x, v[k].x); m.y = __vmaxs4(m.y, v[k].y); m.z = __vmaxs4(m.z, v[k].z); m.w = __vmaxs4(m.w, v[k].w); }
+        else { m.x = __vmaxu4(m.x, v[k].x); m.y = __vmaxu4(m.y, v[k].y); m.z = __vmaxu4(m.z, v[k].z); m.w = __vmaxu4(m.w, v[k].w); }
+      }
+      y[i] = m;
+    } else {
+      unsigned int even[4] = {0, 0, 0, 0}, odd[4] = {0, 0, 0, 0};
+      int cells = 0;
+#pragma unroll
+      for (int k = 0; k < KH * KW; ++k) {
+        if (!ok[k]) continue;
+        const unsigned int flip = kSigned ? 0x80808080u : 0u;
+        const unsigned int word[4] = {v[k].x ^ flip, v[k].y ^ flip, v[k].z ^ flip, v[k].w ^ flip};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          even[j] += word[j] & 0x00ff00ffu;
+          odd[j] += __byte_perm(word[j], 0u, 0x4341u);  // bytes 1 and 3 as 16-bit lanes
+        }
+        ++cells;
+      }
+      // table index = lane sum - 128 * cells + kOff (signed input was biased by 128 per cell)
+      const unsigned int adj = kSigned ? (unsigned int)(128 * (KH * KW - cells)) * 0x00010001u : 0u;
+      unsigned int out[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const unsigned int e = even[j] + adj, o = odd[j] + adj;
+        out[j] = (unsigned int)table[e & 0xffffu] | ((unsigned int)table[o & 0xffffu] << 8) |
+                 ((unsigned int)table[e >> 16] << 16) | ((unsigned int)table[o >> 16] << 24);
+      }
+      y[i] = make_uint4(out[0], out[1], out[2], out[3]);
+    }
+  }
+}
+
+template <bool kSigned, bool kAvg, int KH, int KW>
+void launch_pool16_window(const void* x, int N, int H, int W, int cg, int st_h, int st_w, int pad_h, int pad_w, int P, int Q,
+                          float inv, void* y, cudaStream_t s) {
+  const unsigned int total = (unsigned int)((size_t)N * P * Q * cg);
+  pool16_window_kernel<kSigned, kAvg, KH, KW><<<grid_for(total, 256, 8), 256, 0, s>>>(
+      static_cast<const uint4*>(x), H, W, cg, st_h, st_w, pad_h, pad_w, P, Q, inv, total, static_cast<uint4*>(y));
+}
+
 int pool_extent(int H, int k, int st, int pad, int ceil_mode) {
   int num = H + 2 * pad - k;
   int o = (ceil_mode ? (num + st - 1) / st : num / st) + 1;
@@ -472,6 +580,18 @@ int launch_pool(const void* x, int t, int N, int H, int W, int C, int kh, int kw
   if (P <= 0 || Q <= 0) return fail(Q8_ERR_INVALID_ARG, "pool: empty output");
   float inv = 1.0f / (float)(kh * kw);
   cudaStream_t s = as_stream(stream);
+  if (C % 16 == 0 && aligned16(x) && aligned16(y) && kh == kw && (kh == 3 || kh == 2) &&
+      (size_t)N * P * Q * (C / 16) < (1ull << 31) && (size_t)N * H * W * (C / 16) < (1ull << 31)) {
+    const int cg = C / 16;
+    if (kh == 3) {
+      if (t == Q8_S8) launch_pool16_window<true, kAvg, 3, 3>(x, N, H, W, cg, st_h, st_w, pad_h, pad_w, P, Q, inv, y, s);
+      else launch_pool16_window<false, kAvg, 3, 3>(x, N, H, W, cg, st_h, st_w, pad_h, pad_w, P, Q, inv, y, s);
+    } else {
+      if (t == Q8_S8) launch_pool16_window<true, kAvg, 2, 2>(x, N, H, W, cg, st_h, st_w, pad_h, pad_w, P, Q, inv, y, s);
+      else launch_pool16_window<false, kAvg, 2, 2>(x, N, H, W, cg, st_h, st_w, pad_h, pad_w, P, Q, inv, y, s);
+    }
+    return check_launch("pool16_window_kernel");
+  }
   if (!kAvg && C % 16 == 0 && aligned16(x) && aligned16(y)) {
     const int cg = C / 16;
     const int grid16 = grid_for((size_t)N * P * Q * cg, 256, 8);
@@ -604,6 +724,14 @@ int q8_quantize_pad_channels(const float* x, size_t pixels, int C, int C_pad, fl
   if (out_type != Q8_U8 && out_type != Q8_S8) return fail(Q8_ERR_INVALID_ARG, "q8_quantize_pad_channels: bad out_type");
   if (pixels == 0) return Q8_OK;
   const int lo = out_type == Q8_U8 ? 0 : -128, hi = out_type == Q8_U8 ? 255 : 127;
+  if (C == 3 && C_pad == 16 && aligned16(z) && aligned16(x)) {
+    const size_t quads = pixels / 4;
+    if (quads) quantize_pad3_kernel<<<grid_for(quads, kThreads, 8), kThreads, 0, as_stream(stream)>>>(
+        reinterpret_cast<const float4*>(x), quads, q, lo, hi, static_cast<uint4*>(z));
+    if (quads * 4 < pixels)  // the last one to three pixels
+      quantize_pad16_kernel<<<1, 32, 0, as_stream(stream)>>>(x + quads * 12, pixels - quads * 4, 3, 1, q, lo, hi, static_cast<uint4*>(z) + quads * 4);
+    return check_launch("quantize_pad3_kernel");
+  }
   if (C_pad % 16 == 0 && aligned16(z)) {
     const int groups = C_pad / 16;
     quantize_pad16_kernel<<<grid_for(pixels * groups, kThreads, 8), kThreads, 0, as_stream(stream)>>>(
