@@ -9,6 +9,11 @@ for the fused residual sum; all tensor arithmetic runs in the library's kernels.
   conv without ReLU                 : s8, q = max|y| / 127
   conv + residual sum + ReLU        : u8, q = max(max|conv|, max|residual|) / 255
   dequantized output (logits, heads): fp32
+  channel padding                   : a convolution output with a channel count that is not a multiple of 32 and is
+                                      read only by convolutions lives in a buffer padded with zero channels (to 64,
+                                      128 or the next multiple of 32), and its readers get zero weights there: exact,
+                                      and the readers' TMA rows start on 32-byte boundaries (48- and 80-byte rows
+                                      load up to 2.5x slower)
   pooling                           : type and factor of its input
   concat                            : one factor for the whole output, the largest factor among its branches.  A
                                       conv + ReLU read by nothing but the concat writes its channel slice of the
@@ -39,6 +44,10 @@ class QuantNetwork:
         N, H, W, _ = in_shape
         first = next(L for L in layers if L.op == "conv")
         self.c_pad_in = -(-first.conv.C // 16) * 16
+        self.uses: Dict[str, List] = {}
+        for L in layers:
+            for s in L.src + ([L.residual] if L.residual else []):
+                self.uses.setdefault(s, []).append(L)
         self._shapes((N, H, W, self.c_pad_in))
         self._place_concats()
         self._factors = {}
@@ -64,6 +73,8 @@ class QuantNetwork:
                 if L.name in self.in_place:
                     root, off = self.slot[L.name]
                     ldc = self.shape[root][3]
+                elif self.shape[L.name][3] != sp.K:
+                    ldc = self.shape[L.name][3]  # padded with zero channels
                 qc = pipeline.prepare_conv(wf.contiguous(), bf, (n, h, w_, c), q_in, q_y, t_in, y_type, sp.relu, sp.stride,
                                            sp.pad, sp.dil, q_res, res_type, ldc, off, per_channel=per_channel)
                 self.convs[L.name] = qc
@@ -78,11 +89,17 @@ class QuantNetwork:
             dt = q8.TORCH_DTYPES[self.info[L.name][0]]
             if L.name in self.in_place or (L.op == "concat" and self.slot[L.name][0] != L.name):
                 continue  # a slice of the outermost concat's buffer, bound below
-            self.bufs[L.name] = torch.empty(self.shape[L.name], dtype=dt, device=device)
+            padded = L.op == "conv" and self.shape[L.name][3] != L.conv.K
+            self.bufs[L.name] = (torch.zeros if padded else torch.empty)(self.shape[L.name], dtype=dt, device=device)
         for name, (root, off) in self.slot.items():
             if name in self.in_place or (self.by_name[name].op == "concat" and root != name):
                 self.bufs[name] = self.bufs[root][..., off:off + self.shape[name][3]]
         self.workspace = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device=device) if ws_bytes else None
+        # what a caller sees: every tensor with its own channel count (padding channels cut off)
+        self.outputs = {k: v for k, v in self.bufs.items()}
+        for L in layers:
+            if L.op == "conv" and L.name in self.bufs and self.bufs[L.name].shape[-1] != L.conv.K and L.name not in self.slot:
+                self.outputs[L.name] = self.bufs[L.name][..., :L.conv.K]
 
     # ---- host bookkeeping ---------------------------------------------------------------------------
     def _shapes(self, in_shape):
@@ -93,7 +110,12 @@ class QuantNetwork:
                 sp = L.conv
                 P = (h + 2 * sp.pad[0] - sp.dil[0] * (sp.R - 1) - 1) // sp.stride[0] + 1
                 Q = (w_ + 2 * sp.pad[1] - sp.dil[1] * (sp.S - 1) - 1) // sp.stride[1] + 1
-                self.shape[L.name] = (n, P, Q, sp.K)
+                k_out = sp.K
+                readers = self.uses.get(L.name, [])
+                if (sp.K > 32 and sp.K % 32 and not L.f32_out and readers
+                        and all(r.op == "conv" and r.src == [L.name] and r.residual != L.name for r in readers)):
+                    k_out = 64 if sp.K <= 64 else (128 if sp.K <= 128 else -(-sp.K // 32) * 32)
+                self.shape[L.name] = (n, P, Q, k_out)
             elif L.op in ("maxpool", "avgpool"):
                 P = q8.q8_pool_out_extent(h, L.k[0], L.stride[0], L.pad[0], L.ceil_mode)
                 Q = q8.q8_pool_out_extent(w_, L.k[1], L.stride[1], L.pad[1], L.ceil_mode)
@@ -106,10 +128,7 @@ class QuantNetwork:
     def _place_concats(self):
         """slot[name] = (outermost concat, channel offset) for every tensor that is part of a concat;
         in_place = the convolutions that write their slice themselves; members[root] = all non-concat parts."""
-        uses: Dict[str, List] = {}
-        for L in self.layers:
-            for s in L.src + ([L.residual] if L.residual else []):
-                uses.setdefault(s, []).append(L)
+        uses = self.uses
         self.slot, self.in_place, self.members = {}, set(), {}
 
         def place(cat, root, base):
@@ -161,7 +180,7 @@ class QuantNetwork:
         channel slices of a concat buffer)."""
         q8.q8_quantize_pad_channels(x_f32, self.c_pad_in, self.info["input"][1], q8.Q8_S8, out=self.bufs["input"])
         self.run_quantized()
-        return self.bufs
+        return self.outputs
 
     def run_quantized(self):
         """Everything after the input quantization (the part a CUDA graph replays)."""
