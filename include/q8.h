@@ -109,6 +109,13 @@ int q8_quantize_rows(const float* x, size_t rows, size_t cols, const float* d_q,
 int q8_quantize_pad_channels(const float* x, size_t pixels, int C, int C_pad, float q, int out_type,
                              void* z, void* stream);
 
+/* The same for an image batch x[N][H][W][C] written into z[N][H][W_pad][C_pad] (W_pad >= W, C_pad >= C): pixels
+ * beyond W and channels beyond C are zero.  A stride-2 first layer reads its input as pixel pairs, which needs
+ * an even row length; a zero column on the right is never read or acts as the zero padding it replaces, as long
+ * as it does not add an output column (the caller checks that).  Errors as q8_quantize_pad_channels. */
+int q8_quantize_pad_image(const float* x, int N, int H, int W, int C, int W_pad, int C_pad, float q, int out_type,
+                          void* z, void* stream);
+
 /* r[i] = q * float(z[i]).  in_type: Q8_U8, Q8_S8 or Q8_S32. */
 int q8_dequantize(const void* z, int in_type, size_t n, float q, float* r, void* stream);
 

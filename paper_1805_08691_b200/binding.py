@@ -21,7 +21,7 @@ TORCH_DTYPES = {Q8_U8: torch.uint8, Q8_S8: torch.int8, Q8_S32: torch.int32, Q8_F
 EXPORTS = ["q8_version", "q8_last_error", "q8_read_status", "q8_calibrate_maxabs", "q8_factor", "q8_requant_scale",
            "q8_bias_factor", "q8_quantize", "q8_quantize_pad_channels", "q8_dequantize", "q8_fold_bn",
            "q8_conv2d_workspace_bytes", "q8_conv2d_query_algo", "q8_conv2d", "q8_static_workspace_bytes",
-           "q8_conv2d_static_workspace", "q8_concat", "q8_concat_branch", "q8_calibrate_maxabs_rows", "q8_quantize_rows", "q8_pool_out_extent",
+           "q8_conv2d_static_workspace", "q8_concat", "q8_concat_branch", "q8_calibrate_maxabs_rows", "q8_quantize_rows", "q8_quantize_pad_image", "q8_pool_out_extent",
            "q8_maxpool2d", "q8_avgpool2d"]
 
 
@@ -69,6 +69,7 @@ lib.q8_static_workspace_bytes.argtypes = []
 lib.q8_conv2d_static_workspace.argtypes = [C.POINTER(q8_conv_desc), _vp, _vp, _vp, _vp, _vp, _f, _vp, _vp]
 lib.q8_concat.argtypes = [_i, C.POINTER(_vp), _ip, _fp, _f, _i, _sz, _vp, _vp]
 lib.q8_calibrate_maxabs_rows.argtypes = [_vp, _sz, _sz, _vp, _vp]
+lib.q8_quantize_pad_image.argtypes = [_vp, _i, _i, _i, _i, _i, _i, _f, _i, _vp, _vp]
 lib.q8_quantize_rows.argtypes = [_vp, _sz, _sz, _vp, _i, _vp, _vp]
 lib.q8_concat_branch.argtypes = [_vp, _i, _f, _f, _i, _sz, _vp, _i, _i, _vp]
 lib.q8_pool_out_extent.argtypes = [_i] * 5 + [_ip]
@@ -147,6 +148,16 @@ def q8_quantize_pad_channels(x, C_pad, q, out_type, out=None):
     if out is None:
         out = torch.empty(x.shape[:-1] + (C_pad,), dtype=TORCH_DTYPES[out_type], device=x.device)
     _check(lib.q8_quantize_pad_channels(_dev(x, "x"), pixels, Cc, C_pad, q, out_type, _dev(out, "out"), _stream()))
+    return out
+
+
+def q8_quantize_pad_image(x, W_pad, C_pad, q, out_type, out=None):
+    """x: [N, H, W, C] fp32 -> [N, H, W_pad, C_pad] codes, zero beyond W and C."""
+    assert x.dtype == torch.float32 and x.dim() == 4
+    N, H, W, Cc = (int(v) for v in x.shape)
+    if out is None:
+        out = torch.empty((N, H, W_pad, C_pad), dtype=TORCH_DTYPES[out_type], device=x.device)
+    _check(lib.q8_quantize_pad_image(_dev(x, "x"), N, H, W, Cc, W_pad, C_pad, q, out_type, _dev(out, "out"), _stream()))
     return out
 
 

@@ -200,6 +200,26 @@ __global__ void __launch_bounds__(kThreads) quantize_pad16_kernel(const float* _
   }
 }
 
+// Image batch with padded rows and channels: thread = (output pixel, group of 16 output channels).
+__global__ void __launch_bounds__(kThreads) quantize_pad_image_kernel(const float* __restrict__ x, size_t rows, int W, int C,
+                                                                      int W_pad, int groups, float q, int lo, int hi,
+                                                                      uint4* __restrict__ z) {
+  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+  const size_t per_row = (size_t)W_pad * groups;
+  const size_t total = rows * per_row;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += nthreads) {
+    const size_t row = i / per_row;
+    const unsigned int rem = (unsigned int)(i - row * per_row);
+    const int w = (int)(rem / (unsigned)groups), c0 = (int)(rem % (unsigned)groups) * 16;
+    int v[16];
+    const float* src = x + (row * W + w) * C + c0;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v[j] = (w < W && c0 + j < C) ? quant1(__ldcs(src + j), q, lo, hi) : 0;
+    z[i] = make_uint4(pack4(v[0], v[1], v[2], v[3]), pack4(v[4], v[5], v[6], v[7]), pack4(v[8], v[9], v[10], v[11]),
+                      pack4(v[12], v[13], v[14], v[15]));
+  }
+}
+
 // Images: 3 channels -> 16.  Four pixels per thread: three 16-byte loads (12 floats), four 16-byte stores.
 __global__ void __launch_bounds__(kThreads) quantize_pad3_kernel(const float4* __restrict__ x, size_t quads, float q, int lo,
                                                                  int hi, uint4* __restrict__ z) {
@@ -741,6 +761,25 @@ int q8_quantize_pad_channels(const float* x, size_t pixels, int C, int C_pad, fl
   quantize_pad_kernel<unsigned char><<<grid_for(pixels * C_pad, kThreads, 8), kThreads, 0, as_stream(stream)>>>(
       x, pixels, C, C_pad, q, lo, hi, static_cast<unsigned char*>(z));
   return check_launch("quantize_pad_kernel");
+}
+
+int q8_quantize_pad_image(const float* x, int N, int H, int W, int C, int W_pad, int C_pad, float q, int out_type, void* z,
+                          void* stream) {
+  clear_error();
+  if (N < 0 || H < 0 || W < 0 || C <= 0 || W_pad < W || C_pad < C || C_pad % 16)
+    return fail(Q8_ERR_INVALID_ARG, "q8_quantize_pad_image: need W_pad >= W, C_pad >= C > 0, C_pad a multiple of 16");
+  if (W_pad == W) return q8_quantize_pad_channels(x, (size_t)N * H * W, C, C_pad, q, out_type, z, stream);
+  const size_t rows = (size_t)N * H;
+  if ((!x || !z) && rows && W) return fail(Q8_ERR_INVALID_ARG, "q8_quantize_pad_image: null pointer");
+  if (!(q > 0.f) || std::isinf(q)) return fail(Q8_ERR_NONFINITE, "q8_quantize_pad_image: factor must be finite and positive");
+  if (out_type != Q8_U8 && out_type != Q8_S8) return fail(Q8_ERR_INVALID_ARG, "q8_quantize_pad_image: bad out_type");
+  if (!aligned16(z)) return fail(Q8_ERR_ALIGNMENT, "q8_quantize_pad_image: z not 16-byte aligned");
+  if (rows == 0 || W_pad == 0) return Q8_OK;
+  const int lo = out_type == Q8_U8 ? 0 : -128, hi = out_type == Q8_U8 ? 255 : 127;
+  const int groups = C_pad / 16;
+  quantize_pad_image_kernel<<<grid_for(rows * W_pad * groups, kThreads, 8), kThreads, 0, as_stream(stream)>>>(
+      x, rows, W, C, W_pad, groups, q, lo, hi, static_cast<uint4*>(z));
+  return check_launch("quantize_pad_image_kernel");
 }
 
 int q8_dequantize(const void* z, int in_type, size_t n, float q, float* r, void* stream) {

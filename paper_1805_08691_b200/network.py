@@ -4,7 +4,9 @@ q8_conv2d / pooling / concat calls on preallocated device tensors.
 Host logic only: per-tensor factors follow the paper's calibration rule (max-abs / (2^p - 1)) and its "+" rule
 for the fused residual sum; all tensor arithmetic runs in the library's kernels.
 
-  network input (signed)            : s8, q = max|x| / 127, 3 channels zero padded to 16
+  network input (signed)            : s8, q = max|x| / 127, 3 channels zero padded to 16; an odd image width is
+                                      padded with one zero column when the first layer has stride 2 and the column
+                                      adds no output (the kernel reads stride-2 inputs as pixel pairs)
   conv + ReLU                       : u8, q = max / 255
   conv without ReLU                 : s8, q = max|y| / 127
   conv + residual sum + ReLU        : u8, q = max(max|conv|, max|residual|) / 255
@@ -48,7 +50,13 @@ class QuantNetwork:
         for L in layers:
             for s in L.src + ([L.residual] if L.residual else []):
                 self.uses.setdefault(s, []).append(L)
-        self._shapes((N, H, W, self.c_pad_in))
+        self.w_pad_in = W
+        sp0 = first.conv
+        if first.src == ["input"] and sp0.stride[1] == 2 and W % 2 == 1 and sp0.dil[1] == 1:
+            q_of = lambda w: (w + 2 * sp0.pad[1] - (sp0.S - 1) - 1) // 2 + 1
+            if q_of(W + 1) == q_of(W) and all(L is first or "input" not in L.src for L in layers):
+                self.w_pad_in = W + 1
+        self._shapes((N, H, self.w_pad_in, self.c_pad_in))
         self._place_concats()
         self._factors = {}
         self.info = {"input": (q8.Q8_S8, self._factor("input"))}
@@ -178,7 +186,7 @@ class QuantNetwork:
     def forward(self, x_f32: torch.Tensor) -> Dict[str, torch.Tensor]:
         """Enqueues the whole network on the current stream; returns the tensors (preallocated buffers, or
         channel slices of a concat buffer)."""
-        q8.q8_quantize_pad_channels(x_f32, self.c_pad_in, self.info["input"][1], q8.Q8_S8, out=self.bufs["input"])
+        q8.q8_quantize_pad_image(x_f32, self.w_pad_in, self.c_pad_in, self.info["input"][1], q8.Q8_S8, out=self.bufs["input"])
         self.run_quantized()
         return self.outputs
 

@@ -153,3 +153,13 @@ def test_per_row_maxabs_and_quantize(q8, rows, cols):
         qq = q if t != 2 else (q * np.float32(1e-3)).astype(np.float32)
         got = q8.q8_quantize_rows(_cuda(x), _cuda(qq), t).cpu().numpy()
         assert np.array_equal(got, np.stack([o.quantize(x[r], float(qq[r]), ot) for r in range(rows)]))
+
+
+@pytest.mark.parametrize("W,W_pad,C,C_pad", [(41, 42, 3, 16), (40, 40, 3, 16), (7, 9, 20, 32)])
+def test_quantize_pad_image(q8, W, W_pad, C, C_pad):
+    g = np.random.default_rng(W + C)
+    x = (g.standard_normal((2, 5, W, C)) * 2).astype(np.float32)
+    got = q8.q8_quantize_pad_image(_cuda(x), W_pad, C_pad, 0.02, 1).cpu().numpy()
+    assert got.shape == (2, 5, W_pad, C_pad)
+    assert np.array_equal(got[:, :, :W, :C], o.quantize(x, 0.02, o.S8))
+    assert np.all(got[:, :, W:, :] == 0) and np.all(got[..., C:] == 0)
