@@ -263,7 +263,8 @@ def network_numbers(dev, name, reps=20):
                 cal.observe(k, cuda(v))
             maxima = cal.maxima()
             del acts
-        net = network.QuantNetwork(net_layers, folded, maxima, (batch, hw, hw, 3), device=dev)
+        net = network.QuantNetwork(net_layers, folded, maxima, (batch, hw, hw, 3), device=dev,
+                                   streams=int(os.environ.get("Q8_BENCH_STREAMS", "4")))
         x = cuda(nets.images(cfg["seed"] + 1, batch, hw))
         net.forward(x)
         torch.cuda.synchronize()

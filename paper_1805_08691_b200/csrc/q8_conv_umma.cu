@@ -1142,7 +1142,11 @@ FastDiv make_fastdiv(int d) {
   return f;
 }
 
+// Developer knobs for sweeps of tile shapes and pipeline depths: honoured only when Q8_TUNE is set in the
+// environment (looked up once per process), so that a normal launch never reads the environment.
 int tune_env(const char* name, int dflt) {
+  static const bool enabled = getenv("Q8_TUNE") != nullptr;
+  if (!enabled) return dflt;
   const char* v = getenv(name);
   return v && *v ? atoi(v) : dflt;
 }

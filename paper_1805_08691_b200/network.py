@@ -34,10 +34,13 @@ from . import pipeline
 
 class QuantNetwork:
     def __init__(self, layers, folded: Dict[str, tuple], maxima: Dict[str, float], in_shape, device="cuda",
-                 per_channel=False):
+                 per_channel=False, streams=1):
         """folded[name] = (w KRSC, b K) FP32 device tensors; maxima: calibrated max-abs of "input", every layer
         output and "<name>:pre" of residual convolutions; in_shape = (N, H, W, 3); per_channel: one weight
-        factor per output channel instead of one per tensor."""
+        factor per output channel instead of one per tensor; streams: independent branches (the
+        branches of an Inception module, a projection shortcut beside its residual branch, detection heads beside
+        the trunk) are enqueued on up to this many CUDA streams, so that one branch's kernels start on SMs that
+        another branch's kernel has already left."""
         self.layers = layers
         self.maxima = maxima
         self.by_name = {L.name: L for L in layers}
@@ -102,7 +105,11 @@ class QuantNetwork:
         for name, (root, off) in self.slot.items():
             if name in self.in_place or (self.by_name[name].op == "concat" and root != name):
                 self.bufs[name] = self.bufs[root][..., off:off + self.shape[name][3]]
-        self.workspace = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device=device) if ws_bytes else None
+        self._assign_streams(max(1, int(streams)))
+        # split-K scratch: one per stream, layers on different streams may run at the same time
+        self.workspaces = [torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device=device) if ws_bytes else None
+                           for _ in range(self.n_streams)]
+        self.side_streams = [torch.cuda.Stream(device=device) for _ in range(self.n_streams - 1)]
         # what a caller sees: every tensor with its own channel count (padding channels cut off)
         self.outputs = {k: v for k, v in self.bufs.items()}
         for L in layers:
@@ -182,6 +189,43 @@ class QuantNetwork:
             return q8.q8_factor(max(m[name + ":pre"], m[L.residual]), 8)
         return q8.q8_factor(m[name], 8 if L.conv.relu else 7)
 
+    def _assign_streams(self, limit):
+        """stream_of[layer]: a layer continues on the stream of its first input if it is that tensor's first
+        reader, otherwise it opens the least recently used other stream.  deps[layer]: the tensors it must wait
+        for (concat members count through their leaves)."""
+        self.stream_of, self.deps = {"input": 0}, {}
+        first_reader_done = set()
+        next_side = 0
+
+        def leaves(name):
+            L = self.by_name.get(name)
+            if L is not None and L.op == "concat":
+                out = []
+                for s in L.src:
+                    out += leaves(s)
+                return out + [name]   # the concat layer itself (copies of pooled branches)
+            return [name]
+
+        used = 1
+        for L in self.layers:
+            ins = list(L.src) + ([L.residual] if L.residual else [])
+            deps = []
+            for t in ins:
+                deps += leaves(t)
+            self.deps[L.name] = deps
+            src0 = L.src[0]
+            if limit == 1:
+                sid = 0
+            elif src0 not in first_reader_done:
+                sid = self.stream_of[src0]
+                first_reader_done.add(src0)
+            else:
+                next_side = next_side % (limit - 1) + 1
+                sid = next_side
+                used = max(used, sid + 1)
+            self.stream_of[L.name] = sid
+        self.n_streams = used if limit > 1 else 1
+
     # ---- device work --------------------------------------------------------------------------------
     def forward(self, x_f32: torch.Tensor) -> Dict[str, torch.Tensor]:
         """Enqueues the whole network on the current stream; returns the tensors (preallocated buffers, or
@@ -192,21 +236,48 @@ class QuantNetwork:
 
     def run_quantized(self):
         """Everything after the input quantization (the part a CUDA graph replays)."""
-        b = self.bufs
+        if self.n_streams == 1:
+            for L in self.layers:
+                self._launch(L, self.workspaces[0])
+            return
+        main = torch.cuda.current_stream()
+        streams = [main] + self.side_streams
+        fork = torch.cuda.Event()
+        fork.record(main)
+        for st in self.side_streams:
+            st.wait_event(fork)
+        done: Dict[str, torch.cuda.Event] = {}
         for L in self.layers:
-            x = b[L.src[0]]
-            if L.op == "conv":
-                qc = self.convs[L.name]
-                res = b[L.residual] if L.residual is not None else None
-                y = b[self.slot[L.name][0]] if L.name in self.in_place else b[L.name]
-                q8.q8_conv2d(qc.desc, x, qc.w_q, qc.b_q, qc.scale, res, qc.res_scale, y, self.workspace)
-            elif L.op == "maxpool":
-                q8.q8_maxpool2d(x, L.k, L.stride, L.pad, L.ceil_mode, out=b[L.name])
-            elif L.op == "avgpool":
-                q8.q8_avgpool2d(x, L.k, L.stride, L.pad, L.ceil_mode, out=b[L.name])
-            elif L.op == "concat":
-                for s in L.src:
-                    if s in self.in_place or self.by_name[s].op == "concat":
-                        continue
-                    root, off = self.slot[s]
-                    q8.q8_concat_branch(b[s], self.info[s][1], self.info[L.name][1], b[root], off)
+            sid = self.stream_of[L.name]
+            st = streams[sid]
+            for t in self.deps[L.name]:
+                if t in done and self.stream_of[t] != sid:
+                    st.wait_event(done[t])
+            with torch.cuda.stream(st):
+                self._launch(L, self.workspaces[sid])
+            ev = torch.cuda.Event()
+            ev.record(st)
+            done[L.name] = ev
+        for st in self.side_streams:
+            join = torch.cuda.Event()
+            join.record(st)
+            main.wait_event(join)
+
+    def _launch(self, L, workspace):
+        b = self.bufs
+        x = b[L.src[0]]
+        if L.op == "conv":
+            qc = self.convs[L.name]
+            res = b[L.residual] if L.residual is not None else None
+            y = b[self.slot[L.name][0]] if L.name in self.in_place else b[L.name]
+            q8.q8_conv2d(qc.desc, x, qc.w_q, qc.b_q, qc.scale, res, qc.res_scale, y, workspace)
+        elif L.op == "maxpool":
+            q8.q8_maxpool2d(x, L.k, L.stride, L.pad, L.ceil_mode, out=b[L.name])
+        elif L.op == "avgpool":
+            q8.q8_avgpool2d(x, L.k, L.stride, L.pad, L.ceil_mode, out=b[L.name])
+        elif L.op == "concat":
+            for s in L.src:
+                if s in self.in_place or self.by_name[s].op == "concat":
+                    continue
+                root, off = self.slot[s]
+                q8.q8_concat_branch(b[s], self.info[s][1], self.info[L.name][1], b[root], off)

@@ -19,7 +19,7 @@ def _cuda(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
-def _run_both(q8, layers, hw, batch, calib_batches, seed, check_layers=None, per_channel=False):
+def _run_both(q8, layers, hw, batch, calib_batches, seed, check_layers=None, per_channel=False, streams=1):
     from paper_1805_08691_b200 import network, pipeline
     # fold BN on both sides, must agree bit for bit
     folded_o, folded_g = {}, {}
@@ -54,7 +54,7 @@ def _run_both(q8, layers, hw, batch, calib_batches, seed, check_layers=None, per
     x = nets.images(seed + 1, batch, hw)
     prep, info = oracle_net.network_prepare(layers, folded_o, max_o, per_channel)
     want = oracle_net.network_forward(layers, prep, info, x, threads=batch)
-    net = network.QuantNetwork(layers, folded_g, max_g, x.shape, per_channel=per_channel)
+    net = network.QuantNetwork(layers, folded_g, max_g, x.shape, per_channel=per_channel, streams=streams)
     got = net.forward(_cuda(x))
     q8.q8_read_status()
     for L in layers:
@@ -72,6 +72,7 @@ def _run_both(q8, layers, hw, batch, calib_batches, seed, check_layers=None, per
 def test_bottleneck_stack_every_layer(q8):
     layers = nets.bottleneck_stack(C=64, blocks=2)
     _run_both(q8, layers, hw=32, batch=3, calib_batches=2, seed=3100)
+    _run_both(q8, layers, hw=32, batch=3, calib_batches=2, seed=3100, streams=2)
 
 
 def test_per_channel_weight_factors_every_layer(q8):
@@ -106,7 +107,8 @@ def test_inception_v3_bit_exact_and_close_to_fp32(q8):
     """Config 4 at batch 2: 95 affine layers, 15 concatenations (11 modules, 4 nested), 1x7 / 7x1 / 5x5 filters,
     stride-2 reductions with a pooled branch, 3x3 average pools, dequantized logits."""
     layers = nets.inception_v3()
-    got, want, ref, net = _run_both(q8, layers, hw=299, batch=2, calib_batches=2, seed=4000)
+    got, want, ref, net = _run_both(q8, layers, hw=299, batch=2, calib_batches=2, seed=4000, streams=4)
+    assert net.n_streams == 4       # module branches on their own streams, joined at the concatenations
     logits, fp32 = got["fc"].cpu().numpy().reshape(2, -1), ref["fc"].reshape(2, -1)
     rel = float(np.linalg.norm(logits - fp32) / np.linalg.norm(fp32))
     print(f"Inception-v3 int8 vs FP32 logits: relative L2 error {rel:.4f}")
@@ -117,7 +119,7 @@ def test_ssd300_heads_bit_exact_and_close_to_fp32(q8):
     """Config 5 at batch 1: VGG-16 base with ceil-mode pool3, dilation-6 fc6, extra stages, and the twelve
     dequantized 3x3 heads (16/24 and 84/126 output channels) over 8732 boxes."""
     layers = nets.ssd300()
-    got, want, ref, net = _run_both(q8, layers, hw=300, batch=1, calib_batches=1, seed=5000)
+    got, want, ref, net = _run_both(q8, layers, hw=300, batch=1, calib_batches=1, seed=5000, streams=3)
     boxes = 0
     num = den = 0.0
     for L in layers:
