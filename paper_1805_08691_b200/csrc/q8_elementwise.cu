@@ -580,6 +580,44 @@ void launch_pool16_window(const void* x, int N, int H, int W, int cg, int st_h, 
       static_cast<const uint4*>(x), H, W, cg, st_h, st_w, pad_h, pad_w, P, Q, inv, total, static_cast<uint4*>(y));
 }
 
+// Global average pooling (the window is the whole image, one output pixel): a block takes one image and 64
+// channels; thread (g, c) sums every 16th pixel of channel word c, the 16 partial sums meet in shared memory.
+template <bool kSigned>
+__global__ void __launch_bounds__(256) global_avgpool_kernel(const unsigned int* __restrict__ x, int pixels, int cw,
+                                                             float inv, unsigned int* __restrict__ y) {
+  __shared__ int part[16][16][4];
+  const int c = threadIdx.x & 15, g = threadIdx.x >> 4;
+  const int word = blockIdx.x * 16 + c;          // 32-bit word (4 channels) of a pixel
+  const int n = blockIdx.y;
+  int sum[4] = {0, 0, 0, 0};
+  if (word < cw) {
+    const unsigned int* img = x + (size_t)n * pixels * cw + word;
+    for (int p = g; p < pixels; p += 16) {
+      const unsigned int w = __ldg(img + (size_t)p * cw);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const unsigned int b = (w >> (8 * j)) & 0xffu;
+        sum[j] += kSigned ? (int)(signed char)b : (int)b;
+      }
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < 4; ++j) part[g][c][j] = sum[j];
+  __syncthreads();
+  if (g == 0 && word < cw) {
+    int o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      int t = 0;
+#pragma unroll
+      for (int k = 0; k < 16; ++k) t += part[k][c][j];
+      const int z = __float2int_rn(__fmul_rn((float)t, inv));
+      o[j] = kSigned ? min(max(z, -128), 127) : min(max(z, 0), 255);
+    }
+    y[(size_t)n * cw + word] = pack4(o[0], o[1], o[2], o[3]);
+  }
+}
+
 int pool_extent(int H, int k, int st, int pad, int ceil_mode) {
   int num = H + 2 * pad - k;
   int o = (ceil_mode ? (num + st - 1) / st : num / st) + 1;
@@ -600,6 +638,14 @@ int launch_pool(const void* x, int t, int N, int H, int W, int C, int kh, int kw
   if (P <= 0 || Q <= 0) return fail(Q8_ERR_INVALID_ARG, "pool: empty output");
   float inv = 1.0f / (float)(kh * kw);
   cudaStream_t s = as_stream(stream);
+  if (kAvg && P == 1 && Q == 1 && kh == H && kw == W && pad_h == 0 && pad_w == 0 && C % 4 == 0 && N <= 65535 &&
+      (reinterpret_cast<uintptr_t>(x) & 3u) == 0 && (reinterpret_cast<uintptr_t>(y) & 3u) == 0) {
+    const int cw = C / 4;
+    const dim3 grid((unsigned)((cw + 15) / 16), (unsigned)N);
+    if (t == Q8_S8) global_avgpool_kernel<true><<<grid, 256, 0, s>>>(static_cast<const unsigned int*>(x), H * W, cw, inv, static_cast<unsigned int*>(y));
+    else global_avgpool_kernel<false><<<grid, 256, 0, s>>>(static_cast<const unsigned int*>(x), H * W, cw, inv, static_cast<unsigned int*>(y));
+    return check_launch("global_avgpool_kernel");
+  }
   if (C % 16 == 0 && aligned16(x) && aligned16(y) && kh == kw && (kh == 3 || kh == 2) &&
       (size_t)N * P * Q * (C / 16) < (1ull << 31) && (size_t)N * H * W * (C / 16) < (1ull << 31)) {
     const int cg = C / 16;

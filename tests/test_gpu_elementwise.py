@@ -163,3 +163,12 @@ def test_quantize_pad_image(q8, W, W_pad, C, C_pad):
     assert got.shape == (2, 5, W_pad, C_pad)
     assert np.array_equal(got[:, :, :W, :C], o.quantize(x, 0.02, o.S8))
     assert np.all(got[:, :, W:, :] == 0) and np.all(got[..., C:] == 0)
+
+
+@pytest.mark.parametrize("H,W,C,dt", [(7, 7, 2048, np.uint8), (8, 8, 2048, np.uint8), (5, 3, 20, np.int8), (1, 1, 4, np.int8)])
+def test_global_average_pool(q8, H, W, C, dt):
+    g = np.random.default_rng(H * W + C)
+    lo, hi = (0, 256) if dt == np.uint8 else (-128, 128)
+    x = g.integers(lo, hi, (3, H, W, C)).astype(dt)
+    got = q8.q8_avgpool2d(_cuda(x), (H, W), (1, 1), (0, 0), False).cpu().numpy()
+    assert np.array_equal(got, o.pool(x, "avg", (H, W), (1, 1), (0, 0), False))
