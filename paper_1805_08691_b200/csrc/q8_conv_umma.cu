@@ -21,7 +21,8 @@
 //              block, several of them per stage.
 //   B operand (KRSC weights), three sources
 //     resident : the whole layer's weights sit in shared memory for the CTA's lifetime;
-//     ring     : (halo) one BN x BK tile per tap and channel block through its own ring;
+//     ring     : (halo) BN x BK tiles per tap and channel block through their own ring, several taps per
+//                stage (one TMA operation) for tiles up to 128 columns;
 //     stage    : (plain, im2col) one BN x BK tile next to each A block of a stage.
 //
 // Roles (one lane each unless noted):
@@ -33,10 +34,13 @@
 //   warp 2     : hands 8-bit tile buffers to the epilogue groups, filled by TMA with the residual
 //                tile of the fused eltwise sum when there is one;
 //   warp 3     : sends finished 8-bit tiles to global memory with TMA stores, recycles the buffers;
-//   warps 6..  : G epilogue groups of four warps; group g owns every G-th tile of the CTA.  A thread
+//   warps 6..  : G epilogue groups of four warps; group g owns every G-th tile of the CTA, or, in launches
+//                with at most two tiles per CTA, a share of the columns of every tile.  A thread
 //                owns one accumulator row: tcgen05.ld, + bias, requantise, + residual, ReLU, round,
 //                clamp; the 16 bytes go back into the buffer the residual came from (same swizzled
 //                position), which then is the source of the TMA store.
+// The kernel is launched with programmatic stream serialization: its set-up overlaps the tail of the kernel
+// before it, and every global access comes after griddepcontrol.wait.
 // All hand-offs are mbarriers, there is no block-wide barrier after the prologue.  Every wait is
 // bounded in wall-clock time; on expiry a bit of the library's status word is set and all roles drain
 // instead of hanging.
@@ -113,6 +117,7 @@ struct UmmaParams {
   unsigned int a_sub_bytes;  // plain/im2col: one 128 x bk block; halo: bytes of one patch load
   unsigned int b_tile_bytes; // bn * bk
   unsigned int b_sub_bytes;  // b_tile_bytes rounded up to 1 KiB (placement inside a stage); ring: one ring stage
+  int epi_split;             // 1: every epilogue group takes a share of the columns of every tile (short launches)
   int b_T, b_chunks;         // weight ring: filter taps per ring stage (one TMA operation), stages per channel block
   unsigned int a_stage_bytes;
   unsigned int tile8_bytes;
@@ -527,12 +532,18 @@ __device__ __forceinline__ void epilogue_chunk(const UmmaParams& p, const EpiTil
 // is released (acc_empty) as soon as its last chunk is in registers.
 template <int kOut, int kRes>
 __device__ __forceinline__ void epilogue_row(const UmmaParams& p, const EpiTile& t, uint32_t taddr, uint32_t acc_empty_bar,
-                                             int lane) {
-  const int nchunk = p.bn >> 4;
+                                             int lane, const int ch0, const int nchunk) {
+  // chunks ch0 .. nchunk-1 of 16 columns each
   int ra[16], rb[16];
-  tmem_ld_16(taddr, ra);
+  if (ch0 >= nchunk) {  // no columns for this warp in this tile: it still hands the accumulator back
+    tcgen05_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(acc_empty_bar);
+    return;
+  }
+  tmem_ld_16(taddr + ch0 * 16, ra);
 #pragma unroll 1
-  for (int ch = 0; ch < nchunk; ch += 2) {
+  for (int ch = ch0; ch < nchunk; ch += 2) {
     tmem_ld_wait(ra);
     const bool more1 = ch + 1 < nchunk;
     if (more1) tmem_ld_16(taddr + (ch + 1) * 16, rb);
@@ -736,7 +747,7 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
   float* const s_scale = reinterpret_cast<float*>(base_ptr + p.off_chan) + p.k_pad;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int total_tiles = p.m_tiles * p.n_tiles * p.splits;  // work items
-  const int slots = G * p.nbuf;
+  const int slots = p.epi_split ? p.nbuf : G * p.nbuf;  // split mode: nbuf counts the buffers of the CTA
 
   // Programmatic dependent launch: the next kernel of the stream may be scheduled onto SMs as they fall idle
   // (it waits below, like this one, before it touches global memory), and this kernel's own set-up (barriers,
@@ -761,7 +772,8 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
     asm volatile("bar.arrive 1, %0;" ::"r"(nthreads) : "memory");
   } else {
     if (warp == 1) {
-      if (lane < p.nacc) { mbar_init(smem_u32(&acc_full[lane]), 1); mbar_init(smem_u32(&acc_empty[lane]), 4); }  // 4: one arrival per epilogue warp
+      // one arrival per epilogue warp that reads the accumulator: a group's four, or all of them in split mode
+      if (lane < p.nacc) { mbar_init(smem_u32(&acc_full[lane]), 1); mbar_init(smem_u32(&acc_empty[lane]), p.epi_split ? 4 * G : 4); }
       else if (lane >= 8 && lane - 8 < kMmaWarps) mbar_init(smem_u32(&mma_turn[lane - 8]), 1);
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     } else if (warp == 2) {
@@ -769,7 +781,7 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       else if (lane == 16 && p.res_mode == kResTma) prefetch_tensormap(&tmRes);
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     } else if (warp == 3) {
-      if (lane < slots) mbar_init(smem_u32(&store_ready[lane]), kGroupThreads);
+      if (lane < slots) mbar_init(smem_u32(&store_ready[lane]), p.epi_split ? G * kGroupThreads : kGroupThreads);
       else if (lane == 16 && p.out8) prefetch_tensormap(&tmY);
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -1006,10 +1018,16 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
     const uint32_t accf0 = smem_u32(&acc_full[0]), acce0 = smem_u32(&acc_empty[0]);
     const uint32_t bfull0 = smem_u32(&buf_full[0]), ready0 = smem_u32(&store_ready[0]);
     const uint32_t nslots = (uint32_t)slots, nacc = (uint32_t)p.nacc;
-    uint32_t ab = (uint32_t)g % nacc, acc_par = ((uint32_t)g / nacc) & 1u;
-    uint32_t slot = (uint32_t)g, slot_par = 0;
+    // split mode: every group works on every tile and takes the chunks [ch0, ch1) of its columns, so that a
+    // launch with one or two tiles per CTA does not leave three of four groups idle
+    const bool split = p.epi_split != 0;
+    const int tile_step = split ? 1 : G;
+    const int nchunk_all = p.bn >> 4;
+    const int ch0 = split ? (g * nchunk_all) / G : 0, ch1 = split ? ((g + 1) * nchunk_all) / G : nchunk_all;
+    uint32_t ab = split ? 0u : (uint32_t)g % nacc, acc_par = split ? 0u : ((uint32_t)g / nacc) & 1u;
+    uint32_t slot = split ? 0u : (uint32_t)g, slot_par = 0;
     TileIter ti;
-    ti.init(p, blockIdx.x + g * (int)gridDim.x, G * (int)gridDim.x);
+    ti.init(p, blockIdx.x + (split ? 0 : g) * (int)gridDim.x, tile_step * (int)gridDim.x);
     for (; ti.tile < total_tiles; ti.next(p)) {
       bool ok = mbar_wait(accf0 + ab * 8u, acc_par, abortp);
       if (p.nbuf > 0 && ok) ok = mbar_wait(bfull0 + slot * 8u, slot_par, abortp);
@@ -1034,15 +1052,15 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       }
       t.buf = p.nbuf > 0 ? base_ptr + p.off_bufs + (size_t)slot * p.tile8_bytes : nullptr;
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + ab * (uint32_t)p.acc_stride;
-      epilogue_row<kOut, kRes>(p, t, taddr, acce0 + ab * 8u, lane);
+      epilogue_row<kOut, kRes>(p, t, taddr, acce0 + ab * 8u, lane, ch0, ch1);
       if (p.nbuf > 0) {
         // this thread's reads and writes of the buffer are done; the store thread takes over
         if (p.out8) fence_proxy_async_smem();
         mbar_arrive(ready0 + slot * 8u);
       }
-      ab += (uint32_t)G;
+      ab += (uint32_t)tile_step;
       while (ab >= nacc) { ab -= nacc; acc_par ^= 1u; }
-      slot += (uint32_t)G;
+      slot += (uint32_t)tile_step;
       if (slot >= nslots) { slot -= nslots; slot_par ^= 1u; }
     }
   }
@@ -1412,8 +1430,15 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
 
   // ---- shared memory plan: [resident weights] [A stages] [weight ring] [8-bit tile buffers] [bias, scale]
   const bool use_bufs = out8 || res_mode == kResTma;
-  int G = tune_env("Q8_G", BN > 128 ? 2 : 4);
-  if (G > p.nacc) G = 2;  // a group may run at most one accumulator phase ahead of the MMA warp
+  // Launches with at most two work items per CTA cannot keep several groups busy on different tiles: there all
+  // four groups share every tile, each taking a quarter of its columns (any tile width, both accumulators).
+  {
+    const long long items = (long long)p.m_tiles * p.n_tiles * splits;
+    const long long ctas = items < sm_count() ? items : sm_count();
+    p.epi_split = tune_env("Q8_SPLIT", ((items + ctas - 1) / ctas <= 2 && BN >= 64 && d.y_type != Q8_S32) ? 1 : 0);
+  }
+  int G = tune_env("Q8_G", (BN > 128 && !p.epi_split) ? 2 : 4);
+  if (G > p.nacc && !p.epi_split) G = 2;  // a group may run at most one accumulator phase ahead of the MMA warp
   const unsigned chan_bytes = round_up((unsigned)p.k_pad * 8u, 1024u);
   const unsigned budget = (unsigned)(kSmemLimit - kStaticSmemReserve) - 1024u /* alignment slack */ - chan_bytes;
   // Weights stay resident when the whole layer's B operand is small: no per-tile weight traffic at all.
@@ -1436,7 +1461,7 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
       // Weight ring stages of several filter taps, one TMA operation each (the copy engine spends ~600 cycles
       // per operation whatever its size): as many taps as fit in about 48 KiB while two such stages fit beside
       // two activation stages and one tile buffer per epilogue group, spread evenly over a channel block.
-      const unsigned fixed = bres_bytes + (use_bufs ? (unsigned)G * p.tile8_bytes : 0u) + 2u * p.a_stage_bytes;
+      const unsigned fixed = bres_bytes + (use_bufs ? (unsigned)(p.epi_split ? 2 : G) * p.tile8_bytes : 0u) + 2u * p.a_stage_bytes;
       const unsigned avail = budget > fixed ? budget - fixed : 0u;
       int T = (int)(48u * 1024u / p.b_tile_bytes);
       if (T > (int)(avail / (2u * p.b_tile_bytes))) T = (int)(avail / (2u * p.b_tile_bytes));
@@ -1464,8 +1489,9 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
     // two buffers per group when that still leaves a comfortable pipeline
     p.nbuf = (budget >= bres_bytes + 2u * G * p.tile8_bytes + 2u * min_pipe && 2 * G <= kMaxSlots) ? 2 : 1;
     p.nbuf = tune_env("Q8_NBUF", p.nbuf);
+    if (p.epi_split) p.nbuf = 2;  // one buffer per tile in flight; a CTA has at most two tiles
   }
-  const unsigned buf_bytes = (unsigned)(G * p.nbuf) * p.tile8_bytes;
+  const unsigned buf_bytes = (unsigned)(p.epi_split ? p.nbuf : G * p.nbuf) * p.tile8_bytes;
   if (budget < bres_bytes + buf_bytes + min_pipe) return kPlanNoFit;
   unsigned rest = budget - bres_bytes - buf_bytes;
   p.b_stages = 0;
