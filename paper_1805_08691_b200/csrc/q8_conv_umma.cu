@@ -117,6 +117,9 @@ struct UmmaParams {
   unsigned int a_sub_bytes;  // plain/im2col: one 128 x bk block; halo: bytes of one patch load
   unsigned int b_tile_bytes; // bn * bk
   unsigned int b_sub_bytes;  // b_tile_bytes rounded up to 1 KiB (placement inside a stage); ring: one ring stage
+  int cta2;                  // 1: CTA pairs (clusters of two) issue tcgen05.mma.cta_group::2 over two m tiles that
+                             // share the n tile; each CTA holds its own A patch and half of the weight tile rows
+  int m_tiles_real;          // cta2: number of real m tiles (m_tiles counts pairs)
   int epi_split;             // 1: every epilogue group takes a share of the columns of every tile (short launches)
   int b_T, b_chunks;         // weight ring: filter taps per ring stage (one TMA operation), stages per channel block
   unsigned int a_stage_bytes;
@@ -139,15 +142,33 @@ struct UmmaParams {
 // Walks the tiles of one role: tile = first, first + step, ...; tile -> (m tile, n tile) with the
 // n tiles of one m tile adjacent (they share the A operand through L2), and for halo tiles
 // m tile -> (image, tile row, tile column).  Only additions after init().
-struct TileIter {
+template <bool kPair>
+struct TileIterT {
   int tile, step;    // work item index (tile * splits + split) and its stride
   int sp, d_sp;      // split-K part of the work item
   int mt, nt;        // m tile, n tile
   int img, pt, qt;   // halo: image, tile row, tile column
   int d_mt, d_nt, d_img, d_pt, d_qt;
+  int rank;          // cta2: this CTA's rank in its pair; work items are pairs of m tiles (2 * pair + rank)
+  bool valid;        // cta2: the m tile exists (the last pair of an odd count has a phantom second tile)
 
-  __device__ __forceinline__ void init(const UmmaParams& p, int first, int step_) {
+  // cta2: plain re-decoding, a handful of multiply-shift divisions per tile of several thousand cycles
+  __device__ __forceinline__ void decode_pair(const UmmaParams& p) {
+    const int mp = p.fd_ntiles.div(tile);
+    nt = tile - mp * p.n_tiles;
+    mt = 2 * mp + rank;
+    valid = mt < p.m_tiles_real;
+    const int per_img = p.p_tiles * p.q_tiles;
+    img = p.fd_perimg.div(mt);
+    const int r = mt - img * per_img;
+    pt = p.fd_qtiles.div(r);
+    qt = r - pt * p.q_tiles;
+  }
+
+  __device__ __forceinline__ void init(const UmmaParams& p, int first, int step_, int rank_ = 0) {
     tile = first; step = step_;
+    rank = rank_; valid = true;
+    if constexpr (kPair) { sp = d_sp = 0; decode_pair(p); return; }
     int t0 = first, dt = step_;  // output tile and its stride
     sp = d_sp = 0;
     if (p.splits > 1) {
@@ -169,6 +190,7 @@ struct TileIter {
   }
   __device__ __forceinline__ void next(const UmmaParams& p) {
     tile += step;
+    if constexpr (kPair) { decode_pair(p); return; }
     int carry = 0;
     sp += d_sp;
     if (sp >= p.splits) { sp -= p.splits; carry = 1; }
@@ -303,6 +325,60 @@ __device__ __forceinline__ void tmem_relinquish() {
 }
 __device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
   asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+
+// ---- CTA pairs (cta_group::2).  The leader (even rank) issues the MMAs; operands sit at the same shared-memory
+// offsets in both CTAs; loads of either CTA signal the leader's barrier; commits arrive in both CTAs.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, uint32_t leader_bar, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(leader_bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_pair(uint32_t dst, const CUtensorMap* map, uint32_t leader_bar, int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(leader_bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t holder_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(holder_smem), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t addr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void umma_i8_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrives on the barrier at this offset in both CTAs of the pair once the MMAs issued so far have completed
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((unsigned short)3)
+               : "memory");
 }
 
 // D[tmem] (+)= A[smem desc] * B[smem desc]^T, 8-bit integer inputs, int32 accumulate.  The issuing
@@ -530,7 +606,7 @@ __device__ __forceinline__ void epilogue_chunk(const UmmaParams& p, const EpiTil
 
 // All chunks of one accumulator row, TMEM loads one chunk ahead of the arithmetic.  The accumulator
 // is released (acc_empty) as soon as its last chunk is in registers.
-template <int kOut, int kRes>
+template <int kOut, int kRes, bool kPair>
 __device__ __forceinline__ void epilogue_row(const UmmaParams& p, const EpiTile& t, uint32_t taddr, uint32_t acc_empty_bar,
                                              int lane, const int ch0, const int nchunk) {
   // chunks ch0 .. nchunk-1 of 16 columns each
@@ -538,7 +614,7 @@ __device__ __forceinline__ void epilogue_row(const UmmaParams& p, const EpiTile&
   if (ch0 >= nchunk) {  // no columns for this warp in this tile: it still hands the accumulator back
     tcgen05_fence_before();
     __syncwarp();
-    if (lane == 0) mbar_arrive(acc_empty_bar);
+    if (lane == 0) { if constexpr (kPair) mbar_arrive_cluster(acc_empty_bar); else mbar_arrive(acc_empty_bar); }
     return;
   }
   tmem_ld_16(taddr + ch0 * 16, ra);
@@ -551,7 +627,7 @@ __device__ __forceinline__ void epilogue_row(const UmmaParams& p, const EpiTile&
       // every accumulator value of this warp is in registers: hand the TMEM buffer back
       tcgen05_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(acc_empty_bar);
+      if (lane == 0) { if constexpr (kPair) mbar_arrive_cluster(acc_empty_bar); else mbar_arrive(acc_empty_bar); }
     }
     epilogue_chunk<kOut, kRes>(p, t, ch, ra);
     if (more1) {
@@ -561,7 +637,7 @@ __device__ __forceinline__ void epilogue_row(const UmmaParams& p, const EpiTile&
       else {
         tcgen05_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(acc_empty_bar);
+        if (lane == 0) { if constexpr (kPair) mbar_arrive_cluster(acc_empty_bar); else mbar_arrive(acc_empty_bar); }
       }
       epilogue_chunk<kOut, kRes>(p, t, ch + 1, rb);
     }
@@ -586,7 +662,7 @@ __device__ __forceinline__ bool mma_role(const UmmaParams& p, const MmaRoleArgs&
   // the use of a barrier that is in flight, so a lane starts the stage waits of tile lt only after
   // the lane of tile lt - 1 has passed all of its own (the turn barriers); the per-tile bookkeeping
   // and the accumulator wait run ahead of that.
-  TileIter ti;
+  TileIterT<false> ti;
   ti.init(p, blockIdx.x + who * (int)gridDim.x, kMmaWarps * (int)gridDim.x);
   const uint32_t nstages = (uint32_t)p.stages, nbst = (uint32_t)p.b_stages;
   // descriptors: high word constant; low word = start address >> 4 (shared memory ends below 256 KiB,
@@ -718,10 +794,79 @@ __device__ __forceinline__ bool mma_role(const UmmaParams& p, const MmaRoleArgs&
   return true;
 }
 
+// The MMA lanes of the leader CTA of a pair (halo tiles, weight ring): the same schedule as mma_role, with
+// tcgen05.mma.cta_group::2 over both CTAs' tiles and commits that arrive in both CTAs.
+template <int kSteps>
+__device__ __forceinline__ bool mma_role_pair(const UmmaParams& p, const MmaRoleArgs& r, const int who, const int vblock,
+                                              const int vgrid) {
+  TileIterT<true> ti;
+  ti.init(p, vblock + who * vgrid, kMmaWarps * vgrid, 0);
+  const uint32_t nstages = (uint32_t)p.stages, nbst = (uint32_t)p.b_stages;
+  const uint64_t hi = ((uint64_t)p.desc_hi << 32) | (1ull << 16);
+  const uint64_t a_d0 = hi | (((r.base + p.off_a) >> 4) & 0x3fffu), bring_d0 = hi | (((r.base + p.off_bring) >> 4) & 0x3fffu);
+  const uint32_t stage16 = p.a_stage_bytes >> 4, bsub16 = p.b_sub_bytes >> 4, btile16 = p.b_tile_bytes >> 4;
+  const uint32_t idesc = p.idesc;
+  const int taps = p.taps, c_blocks = p.c_blocks, bT = p.b_T;
+  const uint32_t spt = (uint32_t)c_blocks, bpt = (uint32_t)(p.b_chunks * c_blocks);
+  const uint32_t skip_a = (kMmaWarps - 1) * spt, skip_b = (kMmaWarps - 1) * bpt;
+  uint32_t stage = ((uint32_t)who * spt) % nstages, phase = (((uint32_t)who * spt) / nstages) & 1u;
+  uint32_t bs = ((uint32_t)who * bpt) % nbst, bphase = (((uint32_t)who * bpt) / nbst) & 1u;
+  uint64_t a_d = a_d0 + stage * stage16, bring_d = bring_d0 + bs * bsub16;
+  const uint32_t nacc = (uint32_t)p.nacc;
+  uint32_t ab = (uint32_t)who % nacc, acc_par = 1u ^ (((uint32_t)who / nacc) & 1u);
+  uint32_t my_k = 0;
+  const uint32_t turn_next = r.turn + (who == 0 ? 8u : 0u);
+  for (; ti.tile < r.total_tiles; ti.next(p)) {
+    if (!mbar_wait(r.acc_empty + ab * 8u, acc_par, r.abortp)) return false;
+    if (who == 0) { if (my_k > 0 && !mbar_wait(r.turn, (my_k - 1) & 1u, r.abortp)) return false; }
+    else if (!mbar_wait(r.turn + 8u, my_k & 1u, r.abortp)) return false;
+    tcgen05_fence_after();
+    const uint32_t d_tmem = r.tmem_base + ab * (uint32_t)p.acc_stride;
+    uint32_t accum = 0;
+    for (int cb = 0; cb < c_blocks; ++cb) {
+      if (!mbar_wait(r.a_full + stage * 8u, phase, r.abortp)) return false;
+      const bool last_cb = cb == c_blocks - 1;
+      tcgen05_fence_after();
+      for (int tap0 = 0; tap0 < taps; tap0 += bT) {
+        if (!mbar_wait(r.b_full + bs * 8u, bphase, r.abortp)) return false;
+        if (last_cb && tap0 + bT >= taps) mbar_arrive(turn_next);
+        tcgen05_fence_after();
+        const int nt = min(bT, taps - tap0);
+        uint64_t bd = bring_d;
+        for (int t = 0; t < nt; ++t, bd += btile16) {
+          const uint64_t ad = a_d + r.tap_shift16[tap0 + t];
+          umma_i8_pair(d_tmem, ad, bd, idesc, accum);
+#pragma unroll
+          for (int k = 1; k < kSteps; ++k) umma_i8_pair(d_tmem, ad + 2 * k, bd + 2 * k, idesc, 1u);
+          accum = 1;
+        }
+        umma_commit_pair(r.b_empty + bs * 8u);
+        bring_d += bsub16;
+        if (++bs == nbst) { bs = 0; bphase ^= 1u; bring_d = bring_d0; }
+      }
+      umma_commit_pair(r.a_empty + stage * 8u);
+      a_d += stage16;
+      if (++stage == nstages) { stage = 0; phase ^= 1u; a_d = a_d0; }
+    }
+    ++my_k;
+    umma_commit_pair(r.acc_full + ab * 8u);
+    ab += kMmaWarps;
+    while (ab >= nacc) { ab -= nacc; acc_par ^= 1u; }
+    stage += skip_a;
+    while (stage >= nstages) { stage -= nstages; phase ^= 1u; }
+    a_d = a_d0 + stage * stage16;
+    bs += skip_b;
+    while (bs >= nbst) { bs -= nbst; bphase ^= 1u; }
+    bring_d = bring_d0 + bs * bsub16;
+  }
+  return true;
+}
+
 // ------------------------------------------------------------------------------------------ kernel
 // G epilogue groups; one instantiation per output type and residual source keeps a single epilogue
 // body in each kernel (several of them in one kernel made the register allocator spill).
-template <int G, int kOut, int kRes>
+// kCta2: the CTA-pair variant (its cta_group::2 instructions make the kernel launchable as clusters of two only).
+template <int G, int kOut, int kRes, bool kCta2>
 __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
     conv_umma_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                      const __grid_constant__ CUtensorMap tmRes, const __grid_constant__ CUtensorMap tmY,
@@ -746,6 +891,11 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
   int* const s_bias = reinterpret_cast<int*>(base_ptr + p.off_chan);
   float* const s_scale = reinterpret_cast<float*>(base_ptr + p.off_chan) + p.k_pad;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // CTA pairs: both CTAs walk the same sequence of work items (pairs of m tiles); rank 1 takes the second tile
+  int cta_rank = 0;
+  if constexpr (kCta2) cta_rank = (int)cluster_ctarank();
+  const int vblock = kCta2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int vgrid = kCta2 ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   const int total_tiles = p.m_tiles * p.n_tiles * p.splits;  // work items
   const int slots = p.epi_split ? p.nbuf : G * p.nbuf;  // split mode: nbuf counts the buffers of the CTA
 
@@ -769,11 +919,12 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncwarp();
     asm volatile("griddepcontrol.wait;" ::: "memory");  // everything the previous kernel wrote is visible from here
+    if constexpr (kCta2) cluster_sync_all();  // the peer's barriers exist before anything signals them
     asm volatile("bar.arrive 1, %0;" ::"r"(nthreads) : "memory");
   } else {
     if (warp == 1) {
       // one arrival per epilogue warp that reads the accumulator: a group's four, or all of them in split mode
-      if (lane < p.nacc) { mbar_init(smem_u32(&acc_full[lane]), 1); mbar_init(smem_u32(&acc_empty[lane]), p.epi_split ? 4 * G : 4); }
+      if (lane < p.nacc) { mbar_init(smem_u32(&acc_full[lane]), 1); mbar_init(smem_u32(&acc_empty[lane]), (p.epi_split ? 4 * G : 4) * (kCta2 ? 2 : 1)); }
       else if (lane >= 8 && lane - 8 < kMmaWarps) mbar_init(smem_u32(&mma_turn[lane - 8]), 1);
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     } else if (warp == 2) {
@@ -787,8 +938,13 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
     }
     if (warp == 1) {
       __syncwarp();
-      tmem_alloc(smem_u32(&tmem_holder), (uint32_t)p.tmem_cols);
-      tmem_relinquish();
+      if constexpr (kCta2) {
+        tmem_alloc_pair(smem_u32(&tmem_holder), (uint32_t)p.tmem_cols);
+        tmem_relinquish_pair();
+      } else {
+        tmem_alloc(smem_u32(&tmem_holder), (uint32_t)p.tmem_cols);
+        tmem_relinquish();
+      }
     }
     if (p.a_mode == kAHalo && threadIdx.x >= 32 && threadIdx.x - 32 < p.taps) tap_shift16[threadIdx.x - 32] = p.tap_shift16[threadIdx.x - 32];
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -798,6 +954,10 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       s_scale[i] = p.scale ? (p.scale_count == 1 ? p.scale[0] : (i < p.K ? p.scale[i] : 0.f)) : 0.f;
     }
     tcgen05_fence_before();
+    if constexpr (kCta2) {
+      __syncwarp();
+      cluster_sync_all();
+    }
     asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
     tcgen05_fence_after();
   }
@@ -806,8 +966,8 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
 
   if (threadIdx.x == 0) {
     // ------------------------------------------------------------------ A / B producer
-    TileIter ti;
-    ti.init(p, blockIdx.x, gridDim.x);
+    TileIterT<kCta2> ti;
+    ti.init(p, vblock, vgrid, cta_rank);
     const uint32_t nstages = (uint32_t)p.stages, nbst = (uint32_t)p.b_stages;
     const uint32_t afull0 = smem_u32(&a_full[0]), aempty0 = smem_u32(&a_empty[0]);
     const uint32_t bfull0 = smem_u32(&b_full[0]), bempty0 = smem_u32(&b_empty[0]);
@@ -835,12 +995,19 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
     if (p.a_mode == kAHalo) {
       const uint32_t b_tx = (uint32_t)p.b_T * p.b_tile_bytes;
       for (; ti.tile < total_tiles && ok; ti.next(p)) {
-        const int n0 = ti.nt * p.bn, q0 = ti.qt * p.tw - p.pad_w, p0 = ti.pt * p.th * p.stride_h - p.pad_h;
+        const int n0 = ti.nt * p.bn + (kCta2 ? cta_rank * (p.bn >> 1) : 0);
+        const int q0 = ti.qt * p.tw - p.pad_w, p0 = ti.pt * p.th * p.stride_h - p.pad_h;
         for (int c = 0; c < p.C_pad && ok; c += p.bk) {
           if (!mbar_wait(aempty0 + stage * 8u, phase ^ 1u, abortp)) { ok = false; break; }
           const uint32_t bar = afull0 + stage * 8u;
-          mbar_arrive_expect_tx(bar, p.a_sub_bytes);
-          tma_load_4d(a_dst, &tmA, bar, c, q0, p0, ti.img);
+          if constexpr (kCta2) {
+            // the leader's barrier counts the bytes of both CTAs' patches
+            if (cta_rank == 0) mbar_arrive_expect_tx(bar, 2u * p.a_sub_bytes);
+            tma_load_4d_pair(a_dst, &tmA, map_to_cta(bar, 0), c, q0, p0, ti.img);
+          } else {
+            mbar_arrive_expect_tx(bar, p.a_sub_bytes);
+            tma_load_4d(a_dst, &tmA, bar, c, q0, p0, ti.img);
+          }
           a_dst += p.a_stage_bytes;
           if (++stage == nstages) { stage = 0; phase ^= 1u; a_dst = a0; }
           if (p.b_mode == kBRing) {
@@ -849,8 +1016,13 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
             for (int tap = 0; tap < p.taps; tap += p.b_T) {
               if (!mbar_wait(bempty0 + bs * 8u, bphase ^ 1u, abortp)) { ok = false; break; }
               const uint32_t bbar = bfull0 + bs * 8u;
-              mbar_arrive_expect_tx(bbar, b_tx);
-              tma_load_3d(b_dst, &tmB, bbar, c, n0, tap);
+              if constexpr (kCta2) {
+                if (cta_rank == 0) mbar_arrive_expect_tx(bbar, 2u * b_tx);
+                tma_load_3d_pair(b_dst, &tmB, map_to_cta(bbar, 0), c, n0, tap);
+              } else {
+                mbar_arrive_expect_tx(bbar, b_tx);
+                tma_load_3d(b_dst, &tmB, bbar, c, n0, tap);
+              }
               b_dst += p.b_sub_bytes;
               if (++bs == nbst) { bs = 0; bphase ^= 1u; b_dst = bring0; }
             }
@@ -916,10 +1088,14 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
     ra.b_full = smem_u32(&b_full[0]); ra.b_empty = smem_u32(&b_empty[0]);
     ra.acc_full = smem_u32(&acc_full[0]); ra.acc_empty = smem_u32(&acc_empty[0]);
     ra.bres_full = smem_u32(&bres_full); ra.tap_shift16 = tap_shift16; ra.turn = smem_u32(&mma_turn[0]);
-    bool ok;
-    if (p.ksteps == 4) ok = mma_role<4>(p, ra, who);
-    else if (p.ksteps == 2) ok = mma_role<2>(p, ra, who);
-    else ok = mma_role<1>(p, ra, who);
+    bool ok = true;
+    if constexpr (kCta2) {
+      if (cta_rank == 0) ok = p.ksteps == 4 ? mma_role_pair<4>(p, ra, who, vblock, vgrid) : mma_role_pair<2>(p, ra, who, vblock, vgrid);
+    } else {
+      if (p.ksteps == 4) ok = mma_role<4>(p, ra, who);
+      else if (p.ksteps == 2) ok = mma_role<2>(p, ra, who);
+      else ok = mma_role<1>(p, ra, who);
+    }
     if (!ok) {
       abort_flag = 1;
       atomicOr(p.status, kTimeoutMma);
@@ -927,8 +1103,8 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
   } else if (threadIdx.x == 64) {
     // ------------------------------------------------------------------ tile-buffer / residual producer
     if (p.nbuf > 0) {
-      TileIter ti;
-      ti.init(p, blockIdx.x, gridDim.x);
+      TileIterT<kCta2> ti;
+      ti.init(p, vblock, vgrid, cta_rank);
       const uint32_t bfull0 = smem_u32(&buf_full[0]), bempty0 = smem_u32(&buf_empty[0]);
       const uint32_t nslots = (uint32_t)slots;
       uint32_t slot = 0, par = 1;  // slots are used round robin over all groups: tile lt -> slot lt % (G*nbuf)
@@ -938,7 +1114,7 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       for (; ti.tile < total_tiles; ti.next(p)) {
         if (!mbar_wait(bempty0 + slot * 8u, par, abortp)) { ok = false; break; }
         const uint32_t bar = bfull0 + slot * 8u;
-        if (p.res_mode == kResTma) {
+        if (p.res_mode == kResTma && ti.valid) {
           uint32_t dst = base + p.off_bufs + slot * p.tile8_bytes;
           mbar_arrive_expect_tx(bar, p.res_tx_bytes);
           if (p.a_mode == kAHalo) {
@@ -959,8 +1135,8 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
   } else if (threadIdx.x == 96) {
     // ------------------------------------------------------------------ output store / buffer recycler
     if (p.nbuf > 0) {
-      TileIter ti;
-      ti.init(p, blockIdx.x, gridDim.x);
+      TileIterT<kCta2> ti;
+      ti.init(p, vblock, vgrid, cta_rank);
       const uint32_t bempty0 = smem_u32(&buf_empty[0]), ready0 = smem_u32(&store_ready[0]);
       const uint32_t nslots = (uint32_t)slots;
       uint32_t slot = 0, spar = 0;  // tile lt uses buffer lt % (G*nbuf); its use number (lt / (G*nbuf)) gives the parity
@@ -972,7 +1148,9 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
         if (!mbar_wait(ready0 + slot * 8u, spar, abortp)) { ok = false; break; }
         if (p.out8) {
           uint32_t src = base + p.off_bufs + slot * p.tile8_bytes;
-          if (p.a_mode == kAHalo) {
+          if (!ti.valid) {
+            // second tile of the last pair of an odd count: nothing to store
+          } else if (p.a_mode == kAHalo) {
             for (int pn = 0, c = p.c_off + ti.nt * p.bn; pn < p.panels; ++pn, c += pw, src += panel_bytes) tma_store_4d(&tmY, src, c, ti.qt * p.tw, ti.pt * p.th, ti.img);
           } else {
             for (int pn = 0, c = p.c_off + ti.nt * p.bn; pn < p.panels; ++pn, c += pw, src += panel_bytes) tma_store_2d(&tmY, src, c, ti.mt * kBM);
@@ -1015,7 +1193,10 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       t.srow = t.smem_ok ? pp * p.tw + qq : 0;
     }
     // this group's tiles are lt = g, g + G, ... of the CTA's sequence; ring positions advance by additions
-    const uint32_t accf0 = smem_u32(&acc_full[0]), acce0 = smem_u32(&acc_empty[0]);
+    // pair mode: the accumulators of both CTAs are handed back on the leader's barriers
+    const uint32_t accf0 = smem_u32(&acc_full[0]);
+    uint32_t acce0 = smem_u32(&acc_empty[0]);
+    if constexpr (kCta2) acce0 = map_to_cta(acce0, 0);
     const uint32_t bfull0 = smem_u32(&buf_full[0]), ready0 = smem_u32(&store_ready[0]);
     const uint32_t nslots = (uint32_t)slots, nacc = (uint32_t)p.nacc;
     // split mode: every group works on every tile and takes the chunks [ch0, ch1) of its columns, so that a
@@ -1026,8 +1207,8 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
     const int ch0 = split ? (g * nchunk_all) / G : 0, ch1 = split ? ((g + 1) * nchunk_all) / G : nchunk_all;
     uint32_t ab = split ? 0u : (uint32_t)g % nacc, acc_par = split ? 0u : ((uint32_t)g / nacc) & 1u;
     uint32_t slot = split ? 0u : (uint32_t)g, slot_par = 0;
-    TileIter ti;
-    ti.init(p, blockIdx.x + (split ? 0 : g) * (int)gridDim.x, tile_step * (int)gridDim.x);
+    TileIterT<kCta2> ti;
+    ti.init(p, vblock + (split ? 0 : g) * vgrid, tile_step * vgrid, cta_rank);
     for (; ti.tile < total_tiles; ti.next(p)) {
       bool ok = mbar_wait(accf0 + ab * 8u, acc_par, abortp);
       if (p.nbuf > 0 && ok) ok = mbar_wait(bfull0 + slot * 8u, slot_par, abortp);
@@ -1044,7 +1225,7 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       t.y_off = (long long)ti.sp * p.split_stride;
       if (p.a_mode == kAHalo) {
         const int pr = ti.pt * p.th + pp, qc = ti.qt * p.tw + qq;
-        t.row_ok = t.smem_ok && pr < p.P && qc < p.Q;
+        t.row_ok = t.smem_ok && pr < p.P && qc < p.Q && ti.valid;
         t.m = ((long long)ti.img * p.P + pr) * p.Q + qc;
       } else {
         t.m = (long long)ti.mt * kBM + row;
@@ -1052,7 +1233,7 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       }
       t.buf = p.nbuf > 0 ? base_ptr + p.off_bufs + (size_t)slot * p.tile8_bytes : nullptr;
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + ab * (uint32_t)p.acc_stride;
-      epilogue_row<kOut, kRes>(p, t, taddr, acce0 + ab * 8u, lane, ch0, ch1);
+      epilogue_row<kOut, kRes, kCta2>(p, t, taddr, acce0 + ab * 8u, lane, ch0, ch1);
       if (p.nbuf > 0) {
         // this thread's reads and writes of the buffer are done; the store thread takes over
         if (p.out8) fence_proxy_async_smem();
@@ -1067,10 +1248,12 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
 
   tcgen05_fence_before();
   __syncthreads();
+  if constexpr (kCta2) cluster_sync_all();  // the peer may still read this CTA's weight halves and signal its barriers until here
   if (warp == 1) {
     __syncwarp();
     tcgen05_fence_after();
-    tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+    if constexpr (kCta2) tmem_dealloc_pair(tmem_base, (uint32_t)p.tmem_cols);
+    else tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
   }
 }
 
@@ -1225,10 +1408,10 @@ bool choose_halo_tile(const q8_conv_desc& d, int P, int Q, HaloTile* out) {
   return true;
 }
 
-template <int G, int kOut, int kRes>
+template <int G, int kOut, int kRes, bool kCta2>
 int launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmRes, const CUtensorMap& tmY,
                    const UmmaParams& p, size_t dyn, int grid, cudaStream_t stream) {
-  auto kernel = conv_umma_kernel<G, kOut, kRes>;
+  auto kernel = conv_umma_kernel<G, kOut, kRes, kCta2>;
   static bool configured = false;  // per instantiation
   if (!configured) {
     int rc = check_cuda(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit - kStaticSmemReserve),
@@ -1248,15 +1431,26 @@ int launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtenso
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = tune_env("Q8_PDL", 1) ? 1 : 0;
-  int rc = check_cuda(cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, tmRes, tmY, p), "conv_umma: launch");
-  if (rc != Q8_OK) return rc;
+  if (p.cta2) {  // CTA pairs: clusters of two, no dependent launch
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.numAttrs = 1;
+  }
+  const cudaError_t le = cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, tmRes, tmY, p);
+  if (le != cudaSuccess) {
+    cudaGetLastError();
+    return fail(Q8_ERR_CUDA, "conv_umma: launch failed (%s; grid %d, block %d, shared memory %zu, cluster %d)", cudaGetErrorString(le),
+                grid, kCtrlThreads + G * kGroupThreads, dyn, p.cta2 ? 2 : 1);
+  }
   return check_launch("conv_umma_kernel");
 }
 
 template <int G>
 int launch_groups(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmRes, const CUtensorMap& tmY,
                   const UmmaParams& p, size_t dyn, int grid, cudaStream_t stream) {
-#define Q8_LAUNCH(OUT, RES) return launch_variant<G, OUT, RES>(tmA, tmB, tmRes, tmY, p, dyn, grid, stream)
+#define Q8_LAUNCH(OUT, RES) return launch_variant<G, OUT, RES, false>(tmA, tmB, tmRes, tmY, p, dyn, grid, stream)
   switch (p.y_type * 3 + p.res_mode) {
     case Q8_U8 * 3 + kResNone: Q8_LAUNCH(Q8_U8, kResNone);
     case Q8_U8 * 3 + kResTma: Q8_LAUNCH(Q8_U8, kResTma);
@@ -1447,6 +1641,23 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
   const bool resident = tune_env("Q8_BRES", (b_all <= 80u * 1024u && p.taps <= 256 && p.b_tile_bytes % (8u * BK) == 0) ? 1 : 0) != 0;
   p.b_mode = resident ? kBResident : (p.a_mode == kAHalo ? kBRing : kBStage);
   const unsigned bres_bytes = resident ? round_up(b_all, 1024u) : 0u;
+  // CTA pairs for the large layers with 256-wide tiles and streamed weights.  There the shared-memory port is
+  // the limit: every 128 x 256 x 128 block reads 48 KB of operands while TMA writes 32 KB of weights.  With
+  // tcgen05.mma.cta_group::2 two CTAs work on two m tiles of the same n tile, each holds half of the weight
+  // rows, and both the operand reads and the weight writes per SM drop by a third and a half.
+  p.cta2 = 0;
+  p.m_tiles_real = p.m_tiles;
+  {
+    const bool can = p.a_mode == kAHalo && !paired && p.b_mode == kBRing && BN == 256 && out8 && res_mode != kResGlobal &&
+                     splits == 1 && (BK == 128 || BK == 64) && !p.epi_split &&
+                     (long long)((p.m_tiles + 1) / 2) * p.n_tiles >= (long long)tune_env("Q8_CTA2MIN", 2 * (sm_count() / 2));
+    if (can && tune_env("Q8_CTA2", 1)) {
+      p.cta2 = 1;
+      p.m_tiles = (p.m_tiles + 1) / 2;              // work items are pairs of m tiles
+      p.b_tile_bytes = (unsigned)((BN / 2) * BK);   // this CTA's half of the weight rows
+      p.b_sub_bytes = round_up(p.b_tile_bytes, 1024u);
+    }
+  }
   p.b_T = 1;
   p.b_chunks = p.taps;
   unsigned min_pipe;
@@ -1457,7 +1668,7 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
     p.a_stage_bytes = round_up(reach > p.a_sub_bytes ? reach : p.a_sub_bytes, 1024u);
     p.kb = 1;
     // (measured: a gain with four accumulators, i.e. tiles up to 128 columns; a loss with two)
-    if (p.b_mode == kBRing && p.b_tile_bytes % (8u * BK) == 0 && p.nacc >= 4) {
+    if (p.b_mode == kBRing && p.b_tile_bytes % (8u * BK) == 0 && (p.nacc >= 4 || p.cta2)) {
       // Weight ring stages of several filter taps, one TMA operation each (the copy engine spends ~600 cycles
       // per operation whatever its size): as many taps as fit in about 48 KiB while two such stages fit beside
       // two activation stages and one tile buffer per epilogue group, spread evenly over a channel block.
@@ -1561,7 +1772,7 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
     // (C, K, taps) view: one box brings bn rows of b_T consecutive taps, one K-major tile per tap
     cuuint64_t dims[3] = {(cuuint64_t)d.C, (cuuint64_t)d.K, (cuuint64_t)p.taps};
     cuuint64_t strides[2] = {(cuuint64_t)p.taps * d.C, (cuuint64_t)d.C};
-    cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)BN, (cuuint32_t)p.b_T};
+    cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)(p.cta2 ? BN / 2 : BN), (cuuint32_t)p.b_T};
     cr = fn.tiled(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(a.w), dims, strides, box, ones,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   } else {
@@ -1602,7 +1813,8 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
 
   // instruction descriptor: D = s32 (2 << 4); A format at bit 7 (0 = u8, 1 = s8); B = s8 at bit 10;
   // both operands K-major; N/8 at bit 17; M/16 at bit 24.
-  p.idesc = (2u << 4) | ((d.x_type == Q8_S8 ? 1u : 0u) << 7) | (1u << 10) | ((unsigned)(BN >> 3) << 17) | ((unsigned)(kBM >> 4) << 24);
+  p.idesc = (2u << 4) | ((d.x_type == Q8_S8 ? 1u : 0u) << 7) | (1u << 10) | ((unsigned)(BN >> 3) << 17) |
+            ((unsigned)((p.cta2 ? 2 * kBM : kBM) >> 4) << 24);
   // shared-memory matrix descriptor of a K-major operand tile whose rows are BK bytes (= one swizzle
   // span): 8-row groups are 8*BK bytes apart (stride byte offset, bits 32-45), the leading byte offset
   // (bits 16-29) is unused for swizzled K-major tiles and set to 1, descriptor version 1 (bit 46),
@@ -1625,6 +1837,18 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
   const long long tiles = (long long)p.m_tiles * p.n_tiles * splits;  // work items
   int grid = (int)(tiles < sm_count() ? tiles : sm_count());
   grid = tune_env("Q8_GRID", grid);
+  if (p.cta2) {  // one cluster of two CTAs per work item in flight
+    const long long pairs = sm_count() / 2;
+    grid = 2 * (int)(tiles < pairs ? tiles : pairs);
+  }
+  if (p.cta2) {  // planned only for 8-bit outputs, two groups, residual by TMA or none
+    if (d.y_type == Q8_U8) {
+      if (res_mode == kResTma) return launch_variant<2, Q8_U8, kResTma, true>(tmA, tmB, tmRes, tmY, p, dyn, grid, a.stream);
+      return launch_variant<2, Q8_U8, kResNone, true>(tmA, tmB, tmRes, tmY, p, dyn, grid, a.stream);
+    }
+    if (res_mode == kResTma) return launch_variant<2, Q8_S8, kResTma, true>(tmA, tmB, tmRes, tmY, p, dyn, grid, a.stream);
+    return launch_variant<2, Q8_S8, kResNone, true>(tmA, tmB, tmRes, tmY, p, dyn, grid, a.stream);
+  }
   if (G == 2) return launch_groups<2>(tmA, tmB, tmRes, tmY, p, dyn, grid, a.stream);
   return launch_groups<4>(tmA, tmB, tmRes, tmY, p, dyn, grid, a.stream);
 }

@@ -140,6 +140,30 @@ def test_short_reduction_extreme_accumulators(q8, xs8, extra):
         assert np.array_equal(_bits(y.cpu().numpy()), _bits(want))
 
 
+PAIR_CASES = [
+    # enough 128 x 256 tiles for every SM pair: these run as clusters of two CTAs (tcgen05.mma.cta_group::2);
+    # an odd number of m tiles leaves the last pair with a phantom second tile
+    ("pair_3x3_c256_k256", 7, 75, 75, 256, 256, 3, 3, 1, 1, 1, False, U8, None, True),
+    ("pair_3x3_c128_k512_res", 10, 38, 38, 128, 512, 3, 3, 1, 1, 1, False, U8, "u8", True),
+    ("pair_3x3_c256_k256_s8", 7, 75, 75, 256, 256, 3, 3, 1, 1, 1, True, S8, "s8", False),
+]
+
+
+@pytest.mark.parametrize("case", PAIR_CASES, ids=[c[0] for c in PAIR_CASES])
+def test_cta_pair_layers_match_oracle(q8, case):
+    name, N, H, W, C, K, R, S, _, _, _, xs8, ytype, res, relu = case
+    x, w, bias, acc, resid, (st, pad, dil) = _make(case)
+    scale = np.float32(100.0 / max(1, np.abs(acc).max()))
+    rs = 0.37 if resid is not None else 0.0
+    want = o.epilogue(acc, scale, resid, rs, relu, OT[ytype])
+    d = q8.make_conv_desc(N, H, W, C, K, R, S, st, pad, dil, S8 if xs8 else U8, S8 if res == "s8" else U8, ytype, relu)
+    for _ in range(2):   # twice: the second launch follows a cluster launch in the stream
+        y = q8.q8_conv2d(d, _cuda(x), _cuda(w), _cuda(bias), torch.tensor([scale], device="cuda"),
+                         _cuda(resid) if resid is not None else None, rs)
+    q8.q8_read_status()
+    assert np.array_equal(y.cpu().numpy(), want)
+
+
 def test_tensor_core_kernel_is_selected(q8):
     """The shapes of the paper's networks must run on tcgen05, not on the fallback."""
     for (N, H, W, C, K, R, S, st, pad) in [(32, 56, 56, 256, 64, 1, 1, 1, 0), (32, 56, 56, 64, 64, 3, 3, 1, 1),
