@@ -1648,9 +1648,14 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
   p.cta2 = 0;
   p.m_tiles_real = p.m_tiles;
   {
-    const bool can = p.a_mode == kAHalo && !paired && p.b_mode == kBRing && BN == 256 && out8 && res_mode != kResGlobal &&
-                     splits == 1 && (BK == 128 || BK == 64) && !p.epi_split &&
-                     (long long)((p.m_tiles + 1) / 2) * p.n_tiles >= (long long)tune_env("Q8_CTA2MIN", 2 * (sm_count() / 2));
+    // 256-wide tiles gain as soon as every SM pair has a work item; 128-wide ones (measured: 150x150 128->128
+    // 113 -> 100 us, 28x28 128->128 16.1 -> 16.7 us) only when the launch is long enough to pay for the cluster
+    // set-up and the lost dependent launch
+    const long long pair_items = (long long)((p.m_tiles + 1) / 2) * p.n_tiles;
+    const long long pair_min = (long long)(sm_count() / 2) * (BN == 256 ? 2 : 8);
+    const bool can = p.a_mode == kAHalo && !paired && p.b_mode == kBRing && (BN == 256 || BN == 128) && out8 &&
+                     res_mode != kResGlobal && splits == 1 && (BK == 128 || BK == 64) && !p.epi_split &&
+                     pair_items >= tune_env("Q8_CTA2MIN", (int)pair_min);
     if (can && tune_env("Q8_CTA2", 1)) {
       p.cta2 = 1;
       p.m_tiles = (p.m_tiles + 1) / 2;              // work items are pairs of m tiles
@@ -1841,13 +1846,19 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
     const long long pairs = sm_count() / 2;
     grid = 2 * (int)(tiles < pairs ? tiles : pairs);
   }
-  if (p.cta2) {  // planned only for 8-bit outputs, two groups, residual by TMA or none
-    if (d.y_type == Q8_U8) {
-      if (res_mode == kResTma) return launch_variant<2, Q8_U8, kResTma, true>(tmA, tmB, tmRes, tmY, p, dyn, grid, a.stream);
-      return launch_variant<2, Q8_U8, kResNone, true>(tmA, tmB, tmRes, tmY, p, dyn, grid, a.stream);
-    }
-    if (res_mode == kResTma) return launch_variant<2, Q8_S8, kResTma, true>(tmA, tmB, tmRes, tmY, p, dyn, grid, a.stream);
-    return launch_variant<2, Q8_S8, kResNone, true>(tmA, tmB, tmRes, tmY, p, dyn, grid, a.stream);
+  if (p.cta2) {  // planned only for 8-bit outputs, residual by TMA or none
+#define Q8_PAIR(GG)                                                                                                      \
+  do {                                                                                                                   \
+    if (d.y_type == Q8_U8) {                                                                                             \
+      if (res_mode == kResTma) return launch_variant<GG, Q8_U8, kResTma, true>(tmA, tmB, tmRes, tmY, p, dyn, grid, a.stream); \
+      return launch_variant<GG, Q8_U8, kResNone, true>(tmA, tmB, tmRes, tmY, p, dyn, grid, a.stream);                    \
+    }                                                                                                                    \
+    if (res_mode == kResTma) return launch_variant<GG, Q8_S8, kResTma, true>(tmA, tmB, tmRes, tmY, p, dyn, grid, a.stream); \
+    return launch_variant<GG, Q8_S8, kResNone, true>(tmA, tmB, tmRes, tmY, p, dyn, grid, a.stream);                      \
+  } while (0)
+    if (G == 2) Q8_PAIR(2);
+    Q8_PAIR(4);
+#undef Q8_PAIR
   }
   if (G == 2) return launch_groups<2>(tmA, tmB, tmRes, tmY, p, dyn, grid, a.stream);
   return launch_groups<4>(tmA, tmB, tmRes, tmY, p, dyn, grid, a.stream);

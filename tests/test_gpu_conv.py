@@ -146,6 +146,7 @@ PAIR_CASES = [
     ("pair_3x3_c256_k256", 7, 75, 75, 256, 256, 3, 3, 1, 1, 1, False, U8, None, True),
     ("pair_3x3_c128_k512_res", 10, 38, 38, 128, 512, 3, 3, 1, 1, 1, False, U8, "u8", True),
     ("pair_3x3_c256_k256_s8", 7, 75, 75, 256, 256, 3, 3, 1, 1, 1, True, S8, "s8", False),
+    ("pair_3x3_c128_k128", 7, 150, 150, 128, 128, 3, 3, 1, 1, 1, False, U8, None, True),   # 128-wide tiles, four groups
 ]
 
 
