@@ -27,7 +27,7 @@ def _worker(rank, world, port, out):
 
 def test_maxima_are_reduced_with_max_and_shards_tile_the_batch():
     world = 2
-    mgr = mp.Manager()
+    mgr = mp.get_context("spawn").Manager()
     out = mgr.dict()
     mp.spawn(_worker, args=(world, _free_port(), out), nprocs=world, join=True)
     want = {"x": 2.0, "a": 5.0, "b": 0.25, "c": 6.0}
