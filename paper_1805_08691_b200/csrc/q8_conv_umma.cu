@@ -1426,17 +1426,18 @@ int launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtenso
   cfg.dynamicSmemBytes = dyn;
   cfg.stream = stream;
   // let this kernel's set-up overlap the tail of the kernel before it in the stream
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = tune_env("Q8_PDL", 1) ? 1 : 0;
-  if (p.cta2) {  // CTA pairs: clusters of two, no dependent launch
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.numAttrs = 1;
+  if (p.cta2) {  // CTA pairs: clusters of two, beside the dependent launch
+    const int pdl = (int)cfg.numAttrs;
+    attr[pdl].id = cudaLaunchAttributeClusterDimension;
+    attr[pdl].val.clusterDim.x = 2;
+    attr[pdl].val.clusterDim.y = 1;
+    attr[pdl].val.clusterDim.z = 1;
+    cfg.numAttrs = pdl + 1;
   }
   const cudaError_t le = cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, tmRes, tmY, p);
   if (le != cudaSuccess) {
@@ -1648,11 +1649,9 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
   p.cta2 = 0;
   p.m_tiles_real = p.m_tiles;
   {
-    // 256-wide tiles gain as soon as every SM pair has a work item; 128-wide ones (measured: 150x150 128->128
-    // 113 -> 100 us, 28x28 128->128 16.1 -> 16.7 us) only when the launch is long enough to pay for the cluster
-    // set-up and the lost dependent launch
+    // worth it once every SM pair has two work items (28x28 128->128, batch 64: 16.0 -> 15.0 us)
     const long long pair_items = (long long)((p.m_tiles + 1) / 2) * p.n_tiles;
-    const long long pair_min = (long long)(sm_count() / 2) * (BN == 256 ? 2 : 8);
+    const long long pair_min = (long long)(sm_count() / 2) * 2;
     const bool can = p.a_mode == kAHalo && !paired && p.b_mode == kBRing && (BN == 256 || BN == 128) && out8 &&
                      res_mode != kResGlobal && splits == 1 && (BK == 128 || BK == 64) && !p.epi_split &&
                      pair_items >= tune_env("Q8_CTA2MIN", (int)pair_min);
