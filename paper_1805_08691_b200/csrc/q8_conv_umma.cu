@@ -1649,15 +1649,25 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
   p.cta2 = 0;
   p.m_tiles_real = p.m_tiles;
   {
-    // worth it once every SM pair has two work items (28x28 128->128, batch 64: 16.0 -> 15.0 us)
+    // Worth it once every SM pair has two work items (28x28 3x3 128->128, batch 64: 16.0 -> 15.0 us).  Shorter
+    // launches gain a microsecond alone but lose inside a network whose branches run on several streams
+    // (clusters need two free SMs of one pair at the same time), so they stay single CTAs.  Tile widths whose
+    // halves keep whole 16-row groups.
     const long long pair_items = (long long)((p.m_tiles + 1) / 2) * p.n_tiles;
-    const long long pair_min = (long long)(sm_count() / 2) * 2;
-    const bool can = p.a_mode == kAHalo && !paired && p.b_mode == kBRing && (BN == 256 || BN == 128) && out8 &&
-                     res_mode != kResGlobal && splits == 1 && (BK == 128 || BK == 64) && !p.epi_split &&
-                     pair_items >= tune_env("Q8_CTA2MIN", (int)pair_min);
+    const bool can = p.a_mode == kAHalo && !paired && p.b_mode == kBRing && BN >= 96 && BN % 32 == 0 && out8 &&
+                     res_mode != kResGlobal && splits == 1 && (BK == 128 || BK == 64) &&
+                     (!p.epi_split || tune_env("Q8_CTA2SPLIT", 0)) &&
+                     pair_items >= tune_env("Q8_CTA2MIN", 2 * (sm_count() / 2));
     if (can && tune_env("Q8_CTA2", 1)) {
       p.cta2 = 1;
       p.m_tiles = (p.m_tiles + 1) / 2;              // work items are pairs of m tiles
+      {
+        const long long items = (long long)p.m_tiles * p.n_tiles, clusters = sm_count() / 2;
+        const long long per = (items + (items < clusters ? items : clusters) - 1) / (items < clusters ? items : clusters);
+        p.epi_split = tune_env("Q8_SPLIT", per <= 2 ? 1 : 0);
+        G = tune_env("Q8_G", (BN > 128 && !p.epi_split) ? 2 : 4);
+        if (G > p.nacc && !p.epi_split) G = 2;
+      }
       p.b_tile_bytes = (unsigned)((BN / 2) * BK);   // this CTA's half of the weight rows
       p.b_sub_bytes = round_up(p.b_tile_bytes, 1024u);
     }

@@ -147,6 +147,11 @@ PAIR_CASES = [
     ("pair_3x3_c128_k512_res", 10, 38, 38, 128, 512, 3, 3, 1, 1, 1, False, U8, "u8", True),
     ("pair_3x3_c256_k256_s8", 7, 75, 75, 256, 256, 3, 3, 1, 1, 1, True, S8, "s8", False),
     ("pair_3x3_c128_k128", 7, 150, 150, 128, 128, 3, 3, 1, 1, 1, False, U8, None, True),   # 128-wide tiles, four groups
+    # 160-, 192- and 96-wide tiles whose halves are 80, 96 and 48 weight rows, ragged tap groups (7 taps in
+    # stages of 4 + 3)
+    ("pair_1x7_c160_k160", 100, 17, 17, 160, 160, 1, 7, 1, (0, 3), 1, False, U8, None, True),
+    ("pair_7x1_c192_k192_res", 100, 17, 17, 192, 192, 7, 1, 1, (3, 0), 1, False, U8, "u8", True),
+    ("pair_3x3_c96_k96_s8", 16, 35, 35, 96, 96, 3, 3, 1, 1, 1, True, S8, None, False),
 ]
 
 
