@@ -32,6 +32,8 @@ CASES = [
     ("1x1_c64_k64_raw", 2, 15, 15, 64, 64, 1, 1, 1, 0, 1, False, S32, None, False),
     ("1x1_c256_k64", 2, 15, 15, 256, 64, 1, 1, 1, 0, 1, False, U8, None, True),
     ("1x1_c64_k256_res", 2, 15, 15, 64, 256, 1, 1, 1, 0, 1, False, U8, "u8", True),
+    ("1x1_c384_k64_three_blocks", 3, 21, 21, 384, 64, 1, 1, 1, 0, 1, False, U8, None, True),   # stages of 2 + 1 channel blocks
+    ("1x1_c512_k128_res", 3, 21, 21, 512, 128, 1, 1, 1, 0, 1, False, U8, "u8", True),
     ("1x1_c128_k128_s8", 2, 15, 15, 128, 128, 1, 1, 1, 0, 1, True, S8, "s8", False),
     ("1x1_c32_k16", 2, 15, 15, 32, 16, 1, 1, 1, 0, 1, False, U8, None, True),
     ("1x1_c16_k24_f32", 2, 15, 15, 16, 24, 1, 1, 1, 0, 1, False, F32, None, False),
