@@ -11,6 +11,12 @@ for the fused residual sum; all tensor arithmetic runs in the library's kernels.
   conv without ReLU                 : s8, q = max|y| / 127
   conv + residual sum + ReLU        : u8, q = max(max|conv|, max|residual|) / 255
   dequantized output (logits, heads): fp32
+  sibling heads                     : dequantized convolutions that read the same tensor with the same filter
+                                      geometry (the localisation and confidence heads of an SSD source map) run as
+                                      ONE convolution over the concatenated output channels with per-channel
+                                      multipliers and biases (each channel keeps its own layer's factors, so
+                                      every value is the one the separate layers give); the layers' outputs are
+                                      channel slices of its result
   channel padding                   : a convolution output with a channel count that is not a multiple of 32 and is
                                       read only by convolutions lives in a buffer padded with zero channels (to 64,
                                       128 or the next multiple of 32), and its readers get zero weights there: exact,
@@ -105,6 +111,7 @@ class QuantNetwork:
         for name, (root, off) in self.slot.items():
             if name in self.in_place or (self.by_name[name].op == "concat" and root != name):
                 self.bufs[name] = self.bufs[root][..., off:off + self.shape[name][3]]
+        ws_bytes = max(ws_bytes, self._merge_sibling_heads(device))
         self._assign_streams(max(1, int(streams)))
         # split-K scratch: one per stream, layers on different streams may run at the same time
         self.workspaces = [torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device=device) if ws_bytes else None
@@ -189,6 +196,44 @@ class QuantNetwork:
             return q8.q8_factor(max(m[name + ":pre"], m[L.residual]), 8)
         return q8.q8_factor(m[name], 8 if L.conv.relu else 7)
 
+    def _merge_sibling_heads(self, device):
+        """Groups of FP32-output convolutions on one input with one geometry become one launch (see the module
+        docstring).  merged[leader] = member names; self.skip = the members that no longer launch."""
+        self.merged, self.skip = {}, set()
+        ws_bytes = 0
+        groups = {}
+        for L in self.layers:
+            if L.op == "conv" and L.f32_out and L.residual is None and L.name not in self.slot and not self.uses.get(L.name):
+                sp = L.conv
+                key = (L.src[0], sp.R, sp.S, tuple(sp.stride), tuple(sp.pad), tuple(sp.dil), bool(sp.relu))
+                groups.setdefault(key, []).append(L.name)
+        for names in groups.values():
+            if len(names) < 2:
+                continue
+            parts = [self.convs[n] for n in names]
+            ks = [int(qc.w_q.shape[0]) for qc in parts]
+            K = sum(ks)
+            d0 = parts[0].desc
+            w_q = torch.cat([qc.w_q for qc in parts], dim=0).contiguous()
+            b_q = torch.cat([qc.b_q if qc.b_q is not None else torch.zeros(k, dtype=torch.int32, device=device)
+                             for qc, k in zip(parts, ks)]).contiguous()
+            scale = torch.cat([qc.scale if qc.scale.numel() == k else qc.scale.expand(k) for qc, k in zip(parts, ks)]).contiguous()
+            desc = q8.make_conv_desc(d0.N, d0.H, d0.W, d0.C, K, d0.R, d0.S, (d0.stride_h, d0.stride_w), (d0.pad_h, d0.pad_w),
+                                     (d0.dil_h, d0.dil_w), d0.x_type, d0.res_type, q8.Q8_F32, bool(d0.relu), K, 0, 0)
+            leader = names[0]
+            self.convs[leader] = pipeline.QuantConv(desc, w_q, b_q, scale, None, parts[0].q_x, 1.0, 0.0)
+            n, P, Q, _ = self.shape[leader]
+            buf = torch.empty((n, P, Q, K), dtype=torch.float32, device=device)
+            off = 0
+            for name, k in zip(names, ks):
+                self.bufs[name] = buf[..., off:off + k]
+                off += k
+            self.bufs[leader + ":merged"] = buf
+            self.merged[leader] = names
+            self.skip.update(names[1:])
+            ws_bytes = max(ws_bytes, q8.q8_conv2d_workspace_bytes(desc))
+        return ws_bytes
+
     def _assign_streams(self, limit):
         """stream_of[layer]: a layer continues on the stream of its first input if it is that tensor's first
         reader, otherwise it opens the least recently used other stream.  deps[layer]: the tensors it must wait
@@ -269,7 +314,11 @@ class QuantNetwork:
         if L.op == "conv":
             qc = self.convs[L.name]
             res = b[L.residual] if L.residual is not None else None
+            if L.name in self.skip:
+                return  # computed by the merged launch of its first sibling
             y = b[self.slot[L.name][0]] if L.name in self.in_place else b[L.name]
+            if L.name in self.merged:
+                y = b[L.name + ":merged"]
             q8.q8_conv2d(qc.desc, x, qc.w_q, qc.b_q, qc.scale, res, qc.res_scale, y, workspace)
         elif L.op == "maxpool":
             q8.q8_maxpool2d(x, L.k, L.stride, L.pad, L.ceil_mode, out=b[L.name])
