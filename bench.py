@@ -9,10 +9,13 @@ of the tcgen05 convolution kernel through the C ABI.  Prints ONE JSON line (rank
 
 * value      : int8 conv TOPS (2 * MACs / time), inputs resident in HBM, steps replayed as CUDA
                graphs over rotating buffer sets whose total size exceeds L2.
-* e2e        : same metric with the u8 input copied from pinned host memory and the u8 output copied
-               back inside the timed region.
+* e2e        : same metric with the u8 input of every step copied from pinned host memory and its u8 output
+               copied back inside the timed region (three streams: the copies overlap the kernels).
 * roofline   : dominant kernel, algorithmic bytes / CUDA-event duration against the measured copy peak.
 * cpu_baseline: the CPU oracle timed on a bounded sample of the same workload on the host cores.
+* bandwidth_kernels: the memory-bound kernels (max-abs, quantize, dequantize, concat, pooling) against the measured
+               copy bandwidth; networks: int8 forward of ResNet-50, Inception-v3 and SSD-300 (images/s), with the
+               paper's Xeon figures beside them as context.  Both only at N = 1; --skip-networks leaves them out.
 * --impl reference: the oracle alone (there is no reference implementation to install for this paper).
 With N > 1 every rank runs its own batch (weak scaling, replicated weights, no data-path collective).
 """
