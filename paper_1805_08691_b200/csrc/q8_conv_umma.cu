@@ -810,12 +810,16 @@ __device__ __forceinline__ bool mma_role_pair(const UmmaParams& p, const MmaRole
   const uint32_t spt = (uint32_t)c_blocks, bpt = (uint32_t)(p.b_chunks * c_blocks);
   const uint32_t skip_a = (kMmaWarps - 1) * spt, skip_b = (kMmaWarps - 1) * bpt;
   uint32_t stage = ((uint32_t)who * spt) % nstages, phase = (((uint32_t)who * spt) / nstages) & 1u;
-  uint32_t bs = ((uint32_t)who * bpt) % nbst, bphase = (((uint32_t)who * bpt) / nbst) & 1u;
+  uint32_t bs = 0, bphase = 0;
+  if (p.b_mode == kBRing) { bs = ((uint32_t)who * bpt) % nbst; bphase = (((uint32_t)who * bpt) / nbst) & 1u; }
   uint64_t a_d = a_d0 + stage * stage16, bring_d = bring_d0 + bs * bsub16;
   const uint32_t nacc = (uint32_t)p.nacc;
   uint32_t ab = (uint32_t)who % nacc, acc_par = 1u ^ (((uint32_t)who / nacc) & 1u);
   uint32_t my_k = 0;
   const uint32_t turn_next = r.turn + (who == 0 ? 8u : 0u);
+  const bool ring = p.b_mode == kBRing;
+  const uint64_t bres_d0 = hi | ((r.base >> 4) & 0x3fffu);
+  if (!ring && !mbar_wait(r.bres_full, 0u, r.abortp)) return false;
   for (; ti.tile < r.total_tiles; ti.next(p)) {
     if (!mbar_wait(r.acc_empty + ab * 8u, acc_par, r.abortp)) return false;
     if (who == 0) { if (my_k > 0 && !mbar_wait(r.turn, (my_k - 1) & 1u, r.abortp)) return false; }
@@ -823,11 +827,22 @@ __device__ __forceinline__ bool mma_role_pair(const UmmaParams& p, const MmaRole
     tcgen05_fence_after();
     const uint32_t d_tmem = r.tmem_base + ab * (uint32_t)p.acc_stride;
     uint32_t accum = 0;
+    uint64_t bres = bres_d0 + (uint32_t)(ti.nt * c_blocks * taps) * btile16;  // resident: (cb, tap) order
     for (int cb = 0; cb < c_blocks; ++cb) {
       if (!mbar_wait(r.a_full + stage * 8u, phase, r.abortp)) return false;
       const bool last_cb = cb == c_blocks - 1;
+      if (last_cb && !ring) mbar_arrive(turn_next);
       tcgen05_fence_after();
-      for (int tap0 = 0; tap0 < taps; tap0 += bT) {
+      if (!ring) {
+        for (int tap = 0; tap < taps; ++tap, bres += btile16) {
+          const uint64_t ad = a_d + r.tap_shift16[tap];
+          umma_i8_pair(d_tmem, ad, bres, idesc, accum);
+#pragma unroll
+          for (int k = 1; k < kSteps; ++k) umma_i8_pair(d_tmem, ad + 2 * k, bres + 2 * k, idesc, 1u);
+          accum = 1;
+        }
+      }
+      for (int tap0 = 0; ring && tap0 < taps; tap0 += bT) {
         if (!mbar_wait(r.b_full + bs * 8u, bphase, r.abortp)) return false;
         if (last_cb && tap0 + bT >= taps) mbar_arrive(turn_next);
         tcgen05_fence_after();
@@ -855,9 +870,11 @@ __device__ __forceinline__ bool mma_role_pair(const UmmaParams& p, const MmaRole
     stage += skip_a;
     while (stage >= nstages) { stage -= nstages; phase ^= 1u; }
     a_d = a_d0 + stage * stage16;
-    bs += skip_b;
-    while (bs >= nbst) { bs -= nbst; bphase ^= 1u; }
-    bring_d = bring_d0 + bs * bsub16;
+    if (ring) {
+      bs += skip_b;
+      while (bs >= nbst) { bs -= nbst; bphase ^= 1u; }
+      bring_d = bring_d0 + bs * bsub16;
+    }
   }
   return true;
 }
@@ -979,8 +996,16 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       // every weight tile of the layer, once: one load per (n tile, channel block) brings all taps,
       // laid out [tap][bn rows][bk bytes], i.e. one K-major operand tile per tap
       const uint32_t bar = smem_u32(&bres_full);
-      mbar_arrive_expect_tx(bar, (uint32_t)(p.n_tiles * p.c_blocks * p.taps) * p.b_tile_bytes);
       uint32_t dst = base;
+      if constexpr (kCta2) {
+        // each CTA keeps its half of the rows of every weight tile; the leader's barrier counts both halves
+        if (cta_rank == 0) mbar_arrive_expect_tx(bar, 2u * (uint32_t)(p.n_tiles * p.c_blocks * p.taps) * p.b_tile_bytes);
+        const uint32_t lbar = map_to_cta(bar, 0);
+        for (int nt = 0; nt < p.n_tiles; ++nt)
+          for (int c = 0; c < p.C_pad; c += p.bk, dst += (uint32_t)p.taps * p.b_tile_bytes)
+            tma_load_3d_pair(dst, &tmB, lbar, c, nt * p.bn + cta_rank * (p.bn >> 1), 0);
+      } else {
+      mbar_arrive_expect_tx(bar, (uint32_t)(p.n_tiles * p.c_blocks * p.taps) * p.b_tile_bytes);
       if (p.a_mode == kAHalo && p.halo_sw == 2) {
         // pixel-pair taps: tap t' of a filter row covers s = 2t' - e and 2t' - e + 1, whose weights are 2C
         // contiguous bytes of the (s, c) axis; a start left of s = 0 is zero filled.  One load per t' brings
@@ -990,6 +1015,7 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       } else {
         for (int nt = 0; nt < p.n_tiles; ++nt)
           for (int c = 0; c < p.C_pad; c += p.bk, dst += (uint32_t)p.taps * p.b_tile_bytes) tma_load_3d(dst, &tmB, bar, c, nt * p.bn, 0);
+      }
       }
     }
     if (p.a_mode == kAHalo) {
@@ -1652,12 +1678,14 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
     // Worth it once every SM pair has two work items (28x28 3x3 128->128, batch 64: 16.0 -> 15.0 us).  Shorter
     // launches gain a microsecond alone but lose inside a network whose branches run on several streams
     // (clusters need two free SMs of one pair at the same time), so they stay single CTAs.  Tile widths whose
-    // halves keep whole 16-row groups.
+    // halves keep whole 16-row groups.  With resident weights the pair only saves MMA issue slots (one 256-row
+    // instruction instead of two 128-row ones): 300x300 64->64 157 against 167 us, but 56x56 batch 32 12.7
+    // against 12.0 us, so only launches of many tiles per SM pair take it.
     const long long pair_items = (long long)((p.m_tiles + 1) / 2) * p.n_tiles;
-    const bool can = p.a_mode == kAHalo && !paired && p.b_mode == kBRing && BN >= 96 && BN % 32 == 0 && out8 &&
+    const bool can = p.a_mode == kAHalo && !paired && (p.b_mode == kBRing ? (BN >= 96 && BN % 32 == 0) : (BN >= 32 && BN % 16 == 0)) && out8 &&
                      res_mode != kResGlobal && splits == 1 && (BK == 128 || BK == 64) &&
                      (!p.epi_split || tune_env("Q8_CTA2SPLIT", 0)) &&
-                     pair_items >= tune_env("Q8_CTA2MIN", 2 * (sm_count() / 2));
+                     pair_items >= tune_env("Q8_CTA2MIN", (p.b_mode == kBRing ? 2 : 16) * (sm_count() / 2));
     if (can && tune_env("Q8_CTA2", 1)) {
       p.cta2 = 1;
       p.m_tiles = (p.m_tiles + 1) / 2;              // work items are pairs of m tiles
@@ -1776,10 +1804,10 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
     cr = fn.tiled(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(a.w), dims, strides, box, ones,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   } else if (resident) {
-    // (C, K, taps) view of the KRSC weights: one box brings bn rows of every tap
+    // (C, K, taps) view of the KRSC weights: one box brings bn rows (CTA pairs: this CTA's half) of every tap
     cuuint64_t dims[3] = {(cuuint64_t)d.C, (cuuint64_t)d.K, (cuuint64_t)p.taps};
     cuuint64_t strides[2] = {(cuuint64_t)p.taps * d.C, (cuuint64_t)d.C};
-    cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)BN, (cuuint32_t)p.taps};
+    cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)(p.cta2 ? BN / 2 : BN), (cuuint32_t)p.taps};
     cr = fn.tiled(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(a.w), dims, strides, box, ones,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   } else if (p.b_mode == kBRing) {
