@@ -58,7 +58,7 @@ namespace {
 constexpr int kBM = 128;
 constexpr int kCtrlWarps = 6;            // producer, MMA 0, buffers/residual, store, MMA 1, spare
 constexpr int kCtrlThreads = kCtrlWarps * 32;
-constexpr int kMmaWarps = 2;             // MMA-issuing lanes, tile lt belongs to lane lt % kMmaWarps
+constexpr int kMmaWarps = 3;             // at most this many MMA-issuing lanes; tile lt belongs to lane lt % mma_lanes
 constexpr int kGroupThreads = 128;      // one epilogue group
 constexpr int kMaxStages = 8;           // A stages
 constexpr int kMaxBStages = 8;          // weight ring
@@ -120,6 +120,7 @@ struct UmmaParams {
   int cta2;                  // 1: CTA pairs (clusters of two) issue tcgen05.mma.cta_group::2 over two m tiles that
                              // share the n tile; each CTA holds its own A patch and half of the weight tile rows
   int m_tiles_real;          // cta2: number of real m tiles (m_tiles counts pairs)
+  int mma_lanes;             // 3 with four accumulators (narrow tiles are bound by the issue rate of a lone lane), else 2
   int epi_split;             // 1: every epilogue group takes a share of the columns of every tile (short launches)
   int b_T, b_chunks;         // weight ring: filter taps per ring stage (one TMA operation), stages per channel block
   unsigned int a_stage_bytes;
@@ -663,7 +664,8 @@ __device__ __forceinline__ bool mma_role(const UmmaParams& p, const MmaRoleArgs&
   // the lane of tile lt - 1 has passed all of its own (the turn barriers); the per-tile bookkeeping
   // and the accumulator wait run ahead of that.
   TileIterT<false> ti;
-  ti.init(p, blockIdx.x + who * (int)gridDim.x, kMmaWarps * (int)gridDim.x);
+  const int L = p.mma_lanes;
+  ti.init(p, blockIdx.x + who * (int)gridDim.x, L * (int)gridDim.x);
   const uint32_t nstages = (uint32_t)p.stages, nbst = (uint32_t)p.b_stages;
   // descriptors: high word constant; low word = start address >> 4 (shared memory ends below 256 KiB,
   // the 14-bit field never wraps) plus the leading-byte-offset field (bits 16-29), unused for swizzled
@@ -679,7 +681,7 @@ __device__ __forceinline__ bool mma_role(const UmmaParams& p, const MmaRoleArgs&
   const uint32_t spt = halo ? (uint32_t)c_blocks : (uint32_t)((k_iters + kb - 1) / kb);  // A stages per tile
   const int bT = p.b_T;
   const uint32_t bpt = (uint32_t)(p.b_chunks * c_blocks);                                 // ring stages per tile
-  const uint32_t skip_a = (kMmaWarps - 1) * spt, skip_b = (kMmaWarps - 1) * bpt;
+  const uint32_t skip_a = (uint32_t)(L - 1) * spt, skip_b = (uint32_t)(L - 1) * bpt;
   uint32_t stage = ((uint32_t)who * spt) % nstages, phase = (((uint32_t)who * spt) / nstages) & 1u;
   uint32_t bs = 0, bphase = 0;
   if (ring) { bs = ((uint32_t)who * bpt) % nbst; bphase = (((uint32_t)who * bpt) / nbst) & 1u; }
@@ -688,14 +690,15 @@ __device__ __forceinline__ bool mma_role(const UmmaParams& p, const MmaRoleArgs&
   const uint32_t nacc = (uint32_t)p.nacc;
   uint32_t ab = (uint32_t)who % nacc, acc_par = 1u ^ (((uint32_t)who / nacc) & 1u);  // accumulator and the parity of its empty barrier
   uint32_t my_k = 0;  // number of tiles this lane has issued
-  const uint32_t turn_next = r.turn + (who == 0 ? 8u : 0u);  // the other lane's turn barrier
+  const uint32_t turn_next = r.turn + (uint32_t)((who + 1) % L) * 8u;  // the next lane's turn barrier
+  const uint32_t turn_mine = r.turn + (uint32_t)who * 8u;
   if (p.b_mode == kBResident && !mbar_wait(r.bres_full, 0u, r.abortp)) return false;
   for (; ti.tile < r.total_tiles; ti.next(p)) {
     if (!mbar_wait(r.acc_empty + ab * 8u, acc_par, r.abortp)) return false;
     // turn[w] counts the tiles the other lane has finished waiting for: tile number k of lane 0 needs
     // k of them, tile number k of lane 1 needs k + 1
-    if (who == 0) { if (my_k > 0 && !mbar_wait(r.turn, (my_k - 1) & 1u, r.abortp)) return false; }
-    else if (!mbar_wait(r.turn + 8u, my_k & 1u, r.abortp)) return false;
+    if (who == 0) { if (my_k > 0 && !mbar_wait(turn_mine, (my_k - 1) & 1u, r.abortp)) return false; }
+    else if (!mbar_wait(turn_mine, my_k & 1u, r.abortp)) return false;
     tcgen05_fence_after();
     const uint32_t d_tmem = r.tmem_base + ab * (uint32_t)p.acc_stride;
     uint32_t accum = 0;
@@ -779,7 +782,7 @@ __device__ __forceinline__ bool mma_role(const UmmaParams& p, const MmaRoleArgs&
     }
     ++my_k;
     umma_commit(r.acc_full + ab * 8u);
-    ab += kMmaWarps;
+    ab += (uint32_t)L;
     while (ab >= nacc) { ab -= nacc; acc_par ^= 1u; }
     // step over the stages and ring tiles of the other lanes' tiles
     stage += skip_a;
@@ -800,7 +803,8 @@ template <int kSteps>
 __device__ __forceinline__ bool mma_role_pair(const UmmaParams& p, const MmaRoleArgs& r, const int who, const int vblock,
                                               const int vgrid) {
   TileIterT<true> ti;
-  ti.init(p, vblock + who * vgrid, kMmaWarps * vgrid, 0);
+  const int L = p.mma_lanes;
+  ti.init(p, vblock + who * vgrid, L * vgrid, 0);
   const uint32_t nstages = (uint32_t)p.stages, nbst = (uint32_t)p.b_stages;
   const uint64_t hi = ((uint64_t)p.desc_hi << 32) | (1ull << 16);
   const uint64_t a_d0 = hi | (((r.base + p.off_a) >> 4) & 0x3fffu), bring_d0 = hi | (((r.base + p.off_bring) >> 4) & 0x3fffu);
@@ -808,41 +812,27 @@ __device__ __forceinline__ bool mma_role_pair(const UmmaParams& p, const MmaRole
   const uint32_t idesc = p.idesc;
   const int taps = p.taps, c_blocks = p.c_blocks, bT = p.b_T;
   const uint32_t spt = (uint32_t)c_blocks, bpt = (uint32_t)(p.b_chunks * c_blocks);
-  const uint32_t skip_a = (kMmaWarps - 1) * spt, skip_b = (kMmaWarps - 1) * bpt;
+  const uint32_t skip_a = (uint32_t)(L - 1) * spt, skip_b = (uint32_t)(L - 1) * bpt;
   uint32_t stage = ((uint32_t)who * spt) % nstages, phase = (((uint32_t)who * spt) / nstages) & 1u;
-  uint32_t bs = 0, bphase = 0;
-  if (p.b_mode == kBRing) { bs = ((uint32_t)who * bpt) % nbst; bphase = (((uint32_t)who * bpt) / nbst) & 1u; }
+  uint32_t bs = ((uint32_t)who * bpt) % nbst, bphase = (((uint32_t)who * bpt) / nbst) & 1u;
   uint64_t a_d = a_d0 + stage * stage16, bring_d = bring_d0 + bs * bsub16;
   const uint32_t nacc = (uint32_t)p.nacc;
   uint32_t ab = (uint32_t)who % nacc, acc_par = 1u ^ (((uint32_t)who / nacc) & 1u);
   uint32_t my_k = 0;
-  const uint32_t turn_next = r.turn + (who == 0 ? 8u : 0u);
-  const bool ring = p.b_mode == kBRing;
-  const uint64_t bres_d0 = hi | ((r.base >> 4) & 0x3fffu);
-  if (!ring && !mbar_wait(r.bres_full, 0u, r.abortp)) return false;
+  const uint32_t turn_next = r.turn + (uint32_t)((who + 1) % L) * 8u;
+  const uint32_t turn_mine = r.turn + (uint32_t)who * 8u;
   for (; ti.tile < r.total_tiles; ti.next(p)) {
     if (!mbar_wait(r.acc_empty + ab * 8u, acc_par, r.abortp)) return false;
-    if (who == 0) { if (my_k > 0 && !mbar_wait(r.turn, (my_k - 1) & 1u, r.abortp)) return false; }
-    else if (!mbar_wait(r.turn + 8u, my_k & 1u, r.abortp)) return false;
+    if (who == 0) { if (my_k > 0 && !mbar_wait(turn_mine, (my_k - 1) & 1u, r.abortp)) return false; }
+    else if (!mbar_wait(turn_mine, my_k & 1u, r.abortp)) return false;
     tcgen05_fence_after();
     const uint32_t d_tmem = r.tmem_base + ab * (uint32_t)p.acc_stride;
     uint32_t accum = 0;
-    uint64_t bres = bres_d0 + (uint32_t)(ti.nt * c_blocks * taps) * btile16;  // resident: (cb, tap) order
     for (int cb = 0; cb < c_blocks; ++cb) {
       if (!mbar_wait(r.a_full + stage * 8u, phase, r.abortp)) return false;
       const bool last_cb = cb == c_blocks - 1;
-      if (last_cb && !ring) mbar_arrive(turn_next);
       tcgen05_fence_after();
-      if (!ring) {
-        for (int tap = 0; tap < taps; ++tap, bres += btile16) {
-          const uint64_t ad = a_d + r.tap_shift16[tap];
-          umma_i8_pair(d_tmem, ad, bres, idesc, accum);
-#pragma unroll
-          for (int k = 1; k < kSteps; ++k) umma_i8_pair(d_tmem, ad + 2 * k, bres + 2 * k, idesc, 1u);
-          accum = 1;
-        }
-      }
-      for (int tap0 = 0; ring && tap0 < taps; tap0 += bT) {
+      for (int tap0 = 0; tap0 < taps; tap0 += bT) {
         if (!mbar_wait(r.b_full + bs * 8u, bphase, r.abortp)) return false;
         if (last_cb && tap0 + bT >= taps) mbar_arrive(turn_next);
         tcgen05_fence_after();
@@ -865,16 +855,14 @@ __device__ __forceinline__ bool mma_role_pair(const UmmaParams& p, const MmaRole
     }
     ++my_k;
     umma_commit_pair(r.acc_full + ab * 8u);
-    ab += kMmaWarps;
+    ab += (uint32_t)L;
     while (ab >= nacc) { ab -= nacc; acc_par ^= 1u; }
     stage += skip_a;
     while (stage >= nstages) { stage -= nstages; phase ^= 1u; }
     a_d = a_d0 + stage * stage16;
-    if (ring) {
-      bs += skip_b;
-      while (bs >= nbst) { bs -= nbst; bphase ^= 1u; }
-      bring_d = bring_d0 + bs * bsub16;
-    }
+    bs += skip_b;
+    while (bs >= nbst) { bs -= nbst; bphase ^= 1u; }
+    bring_d = bring_d0 + bs * bsub16;
   }
   return true;
 }
@@ -997,14 +985,6 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       // laid out [tap][bn rows][bk bytes], i.e. one K-major operand tile per tap
       const uint32_t bar = smem_u32(&bres_full);
       uint32_t dst = base;
-      if constexpr (kCta2) {
-        // each CTA keeps its half of the rows of every weight tile; the leader's barrier counts both halves
-        if (cta_rank == 0) mbar_arrive_expect_tx(bar, 2u * (uint32_t)(p.n_tiles * p.c_blocks * p.taps) * p.b_tile_bytes);
-        const uint32_t lbar = map_to_cta(bar, 0);
-        for (int nt = 0; nt < p.n_tiles; ++nt)
-          for (int c = 0; c < p.C_pad; c += p.bk, dst += (uint32_t)p.taps * p.b_tile_bytes)
-            tma_load_3d_pair(dst, &tmB, lbar, c, nt * p.bn + cta_rank * (p.bn >> 1), 0);
-      } else {
       mbar_arrive_expect_tx(bar, (uint32_t)(p.n_tiles * p.c_blocks * p.taps) * p.b_tile_bytes);
       if (p.a_mode == kAHalo && p.halo_sw == 2) {
         // pixel-pair taps: tap t' of a filter row covers s = 2t' - e and 2t' - e + 1, whose weights are 2C
@@ -1015,7 +995,6 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       } else {
         for (int nt = 0; nt < p.n_tiles; ++nt)
           for (int c = 0; c < p.C_pad; c += p.bk, dst += (uint32_t)p.taps * p.b_tile_bytes) tma_load_3d(dst, &tmB, bar, c, nt * p.bn, 0);
-      }
       }
     }
     if (p.a_mode == kAHalo) {
@@ -1105,9 +1084,9 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       abort_flag = 1;
       atomicOr(p.status, kTimeoutProducer);
     }
-  } else if (threadIdx.x == 32 || threadIdx.x == 128) {
-    // ------------------------------------------------------------------ MMA issuers (lane 0 of warps 1 and 4)
-    const int who = threadIdx.x == 32 ? 0 : 1;
+  } else if (threadIdx.x == 32 || threadIdx.x == 128 || (threadIdx.x == 160 && p.mma_lanes == 3)) {
+    // ------------------------------------------------------------------ MMA issuers (lane 0 of warps 1, 4 and 5)
+    const int who = threadIdx.x == 32 ? 0 : (threadIdx.x == 128 ? 1 : 2);
     MmaRoleArgs ra;
     ra.base = base; ra.tmem_base = tmem_base; ra.total_tiles = total_tiles; ra.abortp = abortp;
     ra.a_full = smem_u32(&a_full[0]); ra.a_empty = smem_u32(&a_empty[0]);
@@ -1646,6 +1625,11 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
   while (p.acc_stride < BN) p.acc_stride *= 2;
   p.nacc = 512 / p.acc_stride < kMaxAcc ? 512 / p.acc_stride : kMaxAcc;
   p.tmem_cols = p.nacc * p.acc_stride;  // a power of two in [32, 512]
+  // With two accumulators a third lane could wait on an accumulator barrier two phases ahead (the release it waits
+  // for may belong to a tile that another lane has not issued yet); with four, the tile that last used the
+  // accumulator was issued before this lane's previous tile.
+  p.mma_lanes = tune_env("Q8_LANES", p.nacc >= 4 ? 3 : 2);
+  if (p.mma_lanes > 2 && p.nacc < 4) p.mma_lanes = 2;
   p.b_tile_bytes = (unsigned)(BN * BK);
   p.b_sub_bytes = round_up(p.b_tile_bytes, 1024u);
 
@@ -1678,14 +1662,14 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
     // Worth it once every SM pair has two work items (28x28 3x3 128->128, batch 64: 16.0 -> 15.0 us).  Shorter
     // launches gain a microsecond alone but lose inside a network whose branches run on several streams
     // (clusters need two free SMs of one pair at the same time), so they stay single CTAs.  Tile widths whose
-    // halves keep whole 16-row groups.  With resident weights the pair only saves MMA issue slots (one 256-row
-    // instruction instead of two 128-row ones): 300x300 64->64 157 against 167 us, but 56x56 batch 32 12.7
-    // against 12.0 us, so only launches of many tiles per SM pair take it.
+    // halves keep whole 16-row groups.  Layers with resident weights stay single CTAs: they are bound by the
+    // issue rate of the MMA lanes, which a third lane cures better (300x300 64->64: 167 us with two lanes, 154 us
+    // as pairs, 135 us with three lanes).
     const long long pair_items = (long long)((p.m_tiles + 1) / 2) * p.n_tiles;
-    const bool can = p.a_mode == kAHalo && !paired && (p.b_mode == kBRing ? (BN >= 96 && BN % 32 == 0) : (BN >= 32 && BN % 16 == 0)) && out8 &&
+    const bool can = p.a_mode == kAHalo && !paired && p.b_mode == kBRing && BN >= 96 && BN % 32 == 0 && out8 &&
                      res_mode != kResGlobal && splits == 1 && (BK == 128 || BK == 64) &&
                      (!p.epi_split || tune_env("Q8_CTA2SPLIT", 0)) &&
-                     pair_items >= tune_env("Q8_CTA2MIN", (p.b_mode == kBRing ? 2 : 16) * (sm_count() / 2));
+                     pair_items >= tune_env("Q8_CTA2MIN", 2 * (sm_count() / 2));
     if (can && tune_env("Q8_CTA2", 1)) {
       p.cta2 = 1;
       p.m_tiles = (p.m_tiles + 1) / 2;              // work items are pairs of m tiles
@@ -1804,10 +1788,10 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
     cr = fn.tiled(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(a.w), dims, strides, box, ones,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   } else if (resident) {
-    // (C, K, taps) view of the KRSC weights: one box brings bn rows (CTA pairs: this CTA's half) of every tap
+    // (C, K, taps) view of the KRSC weights: one box brings bn rows of every tap
     cuuint64_t dims[3] = {(cuuint64_t)d.C, (cuuint64_t)d.K, (cuuint64_t)p.taps};
     cuuint64_t strides[2] = {(cuuint64_t)p.taps * d.C, (cuuint64_t)d.C};
-    cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)(p.cta2 ? BN / 2 : BN), (cuuint32_t)p.taps};
+    cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)BN, (cuuint32_t)p.taps};
     cr = fn.tiled(&tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(a.w), dims, strides, box, ones,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   } else if (p.b_mode == kBRing) {

@@ -154,9 +154,9 @@ PAIR_CASES = [
     ("pair_1x7_c160_k160", 100, 17, 17, 160, 160, 1, 7, 1, (0, 3), 1, False, U8, None, True),
     ("pair_7x1_c192_k192_res", 100, 17, 17, 192, 192, 7, 1, 1, (3, 0), 1, False, U8, "u8", True),
     ("pair_3x3_c96_k96_s8", 16, 35, 35, 96, 96, 3, 3, 1, 1, 1, True, S8, None, False),
-    # weights resident in shared memory, each CTA of a pair keeping half of the rows of every weight tile
-    ("pair_3x3_c64_k64_resident", 24, 112, 112, 64, 64, 3, 3, 1, 1, 1, False, U8, None, True),
-    ("pair_5x5_c64_k64_resident_res", 100, 35, 35, 64, 64, 5, 5, 1, 2, 1, False, U8, "u8", True),
+    # long launches with resident weights (single CTAs, three MMA lanes)
+    ("long_3x3_c64_k64_resident", 24, 112, 112, 64, 64, 3, 3, 1, 1, 1, False, U8, None, True),
+    ("long_5x5_c64_k64_resident_res", 100, 35, 35, 64, 64, 5, 5, 1, 2, 1, False, U8, "u8", True),
 ]
 
 
