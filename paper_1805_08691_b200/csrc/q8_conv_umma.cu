@@ -120,6 +120,8 @@ struct UmmaParams {
   int cta2;                  // 1: CTA pairs (clusters of two) issue tcgen05.mma.cta_group::2 over two m tiles that
                              // share the n tile; each CTA holds its own A patch and half of the weight tile rows
   int m_tiles_real;          // cta2: number of real m tiles (m_tiles counts pairs)
+  int fast_taps;             // halo: tap count of a filter whose issue loop is unrolled (3x3, 5x5, 7 x 4 pairs), else 0
+  unsigned int row16, col16; // halo: descriptor shift, in 16-byte units, of one filter row / one filter column
   int mma_lanes;             // 3 with four accumulators (narrow tiles are bound by the issue rate of a lone lane), else 2
   int epi_split;             // 1: every epilogue group takes a share of the columns of every tile (short launches)
   int b_T, b_chunks;         // weight ring: filter taps per ring stage (one TMA operation), stages per channel block
@@ -411,6 +413,27 @@ __device__ __forceinline__ void umma_i8_block(uint32_t d_tmem, uint64_t a_desc, 
   for (int k = 1; k < kSteps; ++k) umma_i8_acc(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc);
 }
 
+// All taps of an R x S filter (kTrans: tap order (s, r) of the pixel-pair view, else (r, s)) on one channel block
+// against resident weight tiles, fully unrolled: the descriptor shift of tap (r, s) is r * row16 + s * col16.
+template <int kR, int kS, bool kTrans, int kSteps>
+__device__ __forceinline__ void issue_taps(uint32_t d_tmem, uint64_t a_d, uint32_t row16, uint32_t col16, uint64_t bres,
+                                           uint32_t btile16, uint32_t idesc, uint32_t accumulate_first) {
+  uint32_t coff[kS];
+#pragma unroll
+  for (int t = 0; t < kS; ++t) coff[t] = (uint32_t)t * col16;
+  uint64_t rowb = a_d;  // descriptor of filter row r, advanced by additions
+#pragma unroll
+  for (int r = 0; r < kR; ++r) {
+#pragma unroll
+    for (int t = 0; t < kS; ++t) {
+      const int tap = kTrans ? t * kR + r : r * kS + t;  // position of the tap's weight tile
+      umma_i8_block<kSteps>(d_tmem, rowb + coff[t], bres + (uint32_t)tap * btile16, idesc,
+                            (r == 0 && t == 0) ? accumulate_first : 1u);
+    }
+    rowb += row16;
+  }
+}
+
 // The mbarrier gets one arrival once every tcgen05.mma issued so far by this thread has completed.
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -693,6 +716,10 @@ __device__ __forceinline__ bool mma_role(const UmmaParams& p, const MmaRoleArgs&
   const uint32_t turn_next = r.turn + (uint32_t)((who + 1) % L) * 8u;  // the next lane's turn barrier
   const uint32_t turn_mine = r.turn + (uint32_t)who * 8u;
   if (p.b_mode == kBResident && !mbar_wait(r.bres_full, 0u, r.abortp)) return false;
+  const int fast_taps = halo ? p.fast_taps : 0;  // 9: 3x3, 25: 5x5, 28: 7x7 as pixel pairs, else 0
+  uint32_t shift9[9];
+#pragma unroll
+  for (int t = 0; t < 9; ++t) shift9[t] = fast_taps == 9 ? r.tap_shift16[t] : 0u;
   for (; ti.tile < r.total_tiles; ti.next(p)) {
     if (!mbar_wait(r.acc_empty + ab * 8u, acc_par, r.abortp)) return false;
     // turn[w] counts the tiles the other lane has finished waiting for: tile number k of lane 0 needs
@@ -738,6 +765,23 @@ __device__ __forceinline__ bool mma_role(const UmmaParams& p, const MmaRoleArgs&
             bring_d += bsub16;
             if (++bs == nbst) { bs = 0; bphase ^= 1u; bring_d = bring_d0; }
           }
+        } else if (fast_taps == 9) {
+          // common filters: tap shifts in registers, straight-line issue (this lane pays ~6 cycles per
+          // instruction, more per branch, and a shared-memory load per tap otherwise)
+          // 3x3: the nine shifts live in registers (measured faster than forming them by additions)
+#pragma unroll
+          for (int tap = 0; tap < 9; ++tap)
+            umma_i8_block<kSteps>(d_tmem, a_d + shift9[tap], bres + (uint32_t)tap * btile16, idesc, tap == 0 ? accum : 1u);
+          accum = 1;
+          bres += 9u * btile16;
+        } else if (fast_taps == 25) {
+          issue_taps<5, 5, false, kSteps>(d_tmem, a_d, p.row16, p.col16, bres, btile16, idesc, accum);
+          accum = 1;
+          bres += 25u * btile16;
+        } else if (fast_taps == 28) {
+          issue_taps<7, 4, true, kSteps>(d_tmem, a_d, p.row16, p.col16, bres, btile16, idesc, accum);
+          accum = 1;
+          bres += 28u * btile16;
         } else {
 #pragma unroll 3
           for (int tap = 0; tap < taps; ++tap) {
@@ -1582,6 +1626,9 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
     p.S = ht.s_eff; p.taps = d.R * ht.s_eff; p.pad_w = ht.pad_w_eff;
     p.halo_sw = ht.sw; p.halo_e = ht.e;
     const int dil_w = paired ? 1 : d.dil_w;
+    p.row16 = (unsigned)(d.dil_h * ht.twb) * (unsigned)(BK >> 4);
+    p.col16 = (unsigned)dil_w * (unsigned)(BK >> 4);
+    p.fast_taps = (!paired && d.R == 3 && ht.s_eff == 3) ? 9 : ((!paired && d.R == 5 && ht.s_eff == 5) ? 25 : ((paired && d.R == 7 && ht.s_eff == 4) ? 28 : 0));
     for (int r = 0; r < d.R; ++r)
       for (int t = 0; t < ht.s_eff; ++t) {
         // tap order = order of the weight tiles in shared memory: (r, s) normally, (t', r) for pixel pairs
