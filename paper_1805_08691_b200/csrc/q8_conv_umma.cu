@@ -750,6 +750,21 @@ __device__ __forceinline__ bool mma_role(const UmmaParams& p, const MmaRoleArgs&
             bring_d += bsub16;
             if (++bs == nbst) { bs = 0; bphase ^= 1u; bring_d = bring_d0; }
           }
+        } else if (ring && fast_taps == 9 && bT == 3) {
+          // 3x3 in ring stages of one filter row each: straight-line issue with the shifts in registers
+#pragma unroll
+          for (int row = 0; row < 3; ++row) {
+            if (!mbar_wait(r.b_full + bs * 8u, bphase, r.abortp)) return false;
+            if (last_cb && row == 2) mbar_arrive(turn_next);
+            tcgen05_fence_after();
+#pragma unroll
+            for (int t = 0; t < 3; ++t)
+              umma_i8_block<kSteps>(d_tmem, a_d + shift9[3 * row + t], bring_d + (uint32_t)t * btile16, idesc, (row == 0 && t == 0) ? accum : 1u);
+            accum = 1;
+            umma_commit(r.b_empty + bs * 8u);
+            bring_d += bsub16;
+            if (++bs == nbst) { bs = 0; bphase ^= 1u; bring_d = bring_d0; }
+          }
         } else if (ring) {
           for (int tap0 = 0; tap0 < taps; tap0 += bT) {
             if (!mbar_wait(r.b_full + bs * 8u, bphase, r.abortp)) return false;
@@ -865,6 +880,10 @@ __device__ __forceinline__ bool mma_role_pair(const UmmaParams& p, const MmaRole
   uint32_t my_k = 0;
   const uint32_t turn_next = r.turn + (uint32_t)((who + 1) % L) * 8u;
   const uint32_t turn_mine = r.turn + (uint32_t)who * 8u;
+  const bool fast9 = p.fast_taps == 9 && bT == 3;
+  uint32_t shift9[9];
+#pragma unroll
+  for (int t = 0; t < 9; ++t) shift9[t] = fast9 ? r.tap_shift16[t] : 0u;
   for (; ti.tile < r.total_tiles; ti.next(p)) {
     if (!mbar_wait(r.acc_empty + ab * 8u, acc_par, r.abortp)) return false;
     if (who == 0) { if (my_k > 0 && !mbar_wait(turn_mine, (my_k - 1) & 1u, r.abortp)) return false; }
@@ -876,7 +895,27 @@ __device__ __forceinline__ bool mma_role_pair(const UmmaParams& p, const MmaRole
       if (!mbar_wait(r.a_full + stage * 8u, phase, r.abortp)) return false;
       const bool last_cb = cb == c_blocks - 1;
       tcgen05_fence_after();
-      for (int tap0 = 0; tap0 < taps; tap0 += bT) {
+      if (fast9) {
+        // 3x3 in ring stages of one filter row each: straight-line issue with the shifts in registers
+#pragma unroll
+        for (int row = 0; row < 3; ++row) {
+          if (!mbar_wait(r.b_full + bs * 8u, bphase, r.abortp)) return false;
+          if (last_cb && row == 2) mbar_arrive(turn_next);
+          tcgen05_fence_after();
+#pragma unroll
+          for (int t = 0; t < 3; ++t) {
+            const uint64_t ad = a_d + shift9[3 * row + t], bd = bring_d + (uint32_t)t * btile16;
+            umma_i8_pair(d_tmem, ad, bd, idesc, (row == 0 && t == 0) ? accum : 1u);
+#pragma unroll
+            for (int k = 1; k < kSteps; ++k) umma_i8_pair(d_tmem, ad + 2 * k, bd + 2 * k, idesc, 1u);
+          }
+          accum = 1;
+          umma_commit_pair(r.b_empty + bs * 8u);
+          bring_d += bsub16;
+          if (++bs == nbst) { bs = 0; bphase ^= 1u; bring_d = bring_d0; }
+        }
+      }
+      for (int tap0 = 0; !fast9 && tap0 < taps; tap0 += bT) {
         if (!mbar_wait(r.b_full + bs * 8u, bphase, r.abortp)) return false;
         if (last_cb && tap0 + bT >= taps) mbar_arrive(turn_next);
         tcgen05_fence_after();
