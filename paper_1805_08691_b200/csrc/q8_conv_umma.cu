@@ -508,7 +508,12 @@ struct EpiTile {
   bool smem_ok;            // this accumulator row maps to a pixel of the tile (always, except halo tiles)
 };
 
-// One 16-column chunk of one accumulator row.  kOut: Q8_U8, Q8_S8, Q8_S32 or Q8_F32.
+// One 16-column chunk of one accumulator row.  kOut: Q8_U8, Q8_S8, Q8_S32 or Q8_F32.  kRes: kResNone, kResTma
+// (a residual from the tile buffer if p.res_mode says so, else none: decided at run time) or kResGlobal.  Fewer
+// distinct kernels matter more than one uniform branch per chunk: a launch of another kernel function than
+// the one before it starts with cold instruction caches, which costs a layer of a network 2 to 6 us, so the
+// layers with and without a residual sum share their kernels.  (One straight-line arm per case, chosen per
+// chunk or per row, made the register allocator spill.)
 //   v = float(acc + bias) * s;  v += float(res) * s_res;  v = max(v, 0);  y = clamp(Round(v))
 // Each step is one IEEE fp32 operation (the library is built without FMA contraction).
 template <int kOut, int kRes>
@@ -542,7 +547,7 @@ __device__ __forceinline__ void epilogue_chunk(const UmmaParams& p, const EpiTil
   }
   // position of this thread's 16 bytes inside the swizzled 8-bit tile buffer
   uint32_t off = 0;
-  if (kOut == Q8_U8 || kOut == Q8_S8 || kRes == kResTma) {
+  if (kOut == Q8_U8 || kOut == Q8_S8 || (kRes == kResTma && p.res_mode == kResTma)) {
     const int pn = c16 >> p.pw_shift;
     off = ((uint32_t)t.srow << p.pw_shift) + (uint32_t)(c16 & ((1 << p.pw_shift) - 1));
     off ^= ((off >> 7) & (uint32_t)p.pmask) << 4;
@@ -559,11 +564,19 @@ __device__ __forceinline__ void epilogue_chunk(const UmmaParams& p, const EpiTil
       v2[2 * j + 1] = fmul2(pack_f2(__int2float_rn(acc[4 * j + 2]), __int2float_rn(acc[4 * j + 3])), pack_f2(s.z, s.w));
     }
   }
-  if (kRes != kResNone) {
-    unsigned int rw[4] = {0u, 0u, 0u, 0u};
+  unsigned int rw[4] = {0u, 0u, 0u, 0u};
+  if (kRes == kResTma && (kOut == Q8_U8 || kOut == Q8_S8)) {
+    // the tile buffer always exists for 8-bit outputs: its bytes are read ahead of the (uniform) branch on
+    // whether they are a residual, so that the load is in flight with those of bias and scale
+    const uint4 rv = *reinterpret_cast<const uint4*>(t.buf + off);
+    rw[0] = rv.x; rw[1] = rv.y; rw[2] = rv.z; rw[3] = rv.w;
+  }
+  if (kRes == kResGlobal || (kRes == kResTma && p.res_mode != kResNone)) {
     if (kRes == kResTma) {
-      const uint4 rv = *reinterpret_cast<const uint4*>(t.buf + off);
-      rw[0] = rv.x; rw[1] = rv.y; rw[2] = rv.z; rw[3] = rv.w;
+      if (kOut != Q8_U8 && kOut != Q8_S8) {
+        const uint4 rv = *reinterpret_cast<const uint4*>(t.buf + off);
+        rw[0] = rv.x; rw[1] = rv.y; rw[2] = rv.z; rw[3] = rv.w;
+      }
     } else if (t.row_ok && nb < p.K) {
       const int valid = min(16, p.K - nb);
       const unsigned char* rp = p.res + (size_t)t.m * p.K + nb;
@@ -1540,18 +1553,21 @@ template <int G>
 int launch_groups(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmRes, const CUtensorMap& tmY,
                   const UmmaParams& p, size_t dyn, int grid, cudaStream_t stream) {
 #define Q8_LAUNCH(OUT, RES) return launch_variant<G, OUT, RES, false>(tmA, tmB, tmRes, tmY, p, dyn, grid, stream)
-  switch (p.y_type * 3 + p.res_mode) {
-    case Q8_U8 * 3 + kResNone: Q8_LAUNCH(Q8_U8, kResNone);
-    case Q8_U8 * 3 + kResTma: Q8_LAUNCH(Q8_U8, kResTma);
-    case Q8_U8 * 3 + kResGlobal: Q8_LAUNCH(Q8_U8, kResGlobal);
-    case Q8_S8 * 3 + kResNone: Q8_LAUNCH(Q8_S8, kResNone);
-    case Q8_S8 * 3 + kResTma: Q8_LAUNCH(Q8_S8, kResTma);
-    case Q8_S8 * 3 + kResGlobal: Q8_LAUNCH(Q8_S8, kResGlobal);
-    case Q8_F32 * 3 + kResNone: Q8_LAUNCH(Q8_F32, kResNone);
-    case Q8_F32 * 3 + kResTma: Q8_LAUNCH(Q8_F32, kResTma);
-    case Q8_F32 * 3 + kResGlobal: Q8_LAUNCH(Q8_F32, kResGlobal);
-    default: Q8_LAUNCH(Q8_S32, kResNone);
+  // kResTma stands for "a residual through the tile buffers, or none"
+  const bool global_res = p.res_mode == kResGlobal;
+  if (p.y_type == Q8_U8) {
+    if (global_res) Q8_LAUNCH(Q8_U8, kResGlobal);
+    Q8_LAUNCH(Q8_U8, kResTma);
   }
+  if (p.y_type == Q8_S8) {
+    if (global_res) Q8_LAUNCH(Q8_S8, kResGlobal);
+    Q8_LAUNCH(Q8_S8, kResTma);
+  }
+  if (p.y_type == Q8_F32) {
+    if (global_res) Q8_LAUNCH(Q8_F32, kResGlobal);
+    Q8_LAUNCH(Q8_F32, kResTma);
+  }
+  Q8_LAUNCH(Q8_S32, kResTma);
 #undef Q8_LAUNCH
 }
 
@@ -1953,7 +1969,9 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
     const long long pairs = sm_count() / 2;
     grid = 2 * (int)(tiles < pairs ? tiles : pairs);
   }
-  if (p.cta2) {  // planned only for 8-bit outputs, residual by TMA or none
+  if (p.cta2) {
+    // planned only for 8-bit outputs, residual by TMA or none.  These are the large 3x3 layers, which seldom
+    // take a residual: their kernels keep that choice at compile time.
 #define Q8_PAIR(GG)                                                                                                      \
   do {                                                                                                                   \
     if (d.y_type == Q8_U8) {                                                                                             \
