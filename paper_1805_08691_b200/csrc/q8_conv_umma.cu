@@ -564,6 +564,8 @@ __device__ __forceinline__ void epilogue_chunk(const UmmaParams& p, const EpiTil
       v2[2 * j + 1] = fmul2(pack_f2(__int2float_rn(acc[4 * j + 2]), __int2float_rn(acc[4 * j + 3])), pack_f2(s.z, s.w));
     }
   }
+#pragma unroll
+  for (int j = 0; j < 8; ++j) unpack_f2(v2[j], v[2 * j], v[2 * j + 1]);
   unsigned int rw[4] = {0u, 0u, 0u, 0u};
   if (kRes == kResTma && (kOut == Q8_U8 || kOut == Q8_S8)) {
     // the tile buffer always exists for 8-bit outputs: its bytes are read ahead of the (uniform) branch on
@@ -598,13 +600,9 @@ __device__ __forceinline__ void epilogue_chunk(const UmmaParams& p, const EpiTil
       // fused operation (one rounding instead of two), which would break the two-rounding definition
       float t0, t1;
       unpack_f2(fmul2(fsub2(pack_f2(r0, r1), magic2), rs2), t0, t1);
-      unpack_f2(v2[j], v[2 * j], v[2 * j + 1]);
       v[2 * j] = __fadd_rn(v[2 * j], t0);
       v[2 * j + 1] = __fadd_rn(v[2 * j + 1], t1);
     }
-  } else {
-#pragma unroll
-    for (int j = 0; j < 8; ++j) unpack_f2(v2[j], v[2 * j], v[2 * j + 1]);
   }
   if (kOut == Q8_F32) {
     if (p.relu) {
