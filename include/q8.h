@@ -197,11 +197,17 @@ int q8_conv2d(const q8_conv_desc* d, const void* x, const int8_t* w, const int32
  * handed out before this library is called, or where cudaMalloc is off limits because it stalls the
  * device: the scratch of the split reduction (see q8_conv2d_workspace_bytes) is a fixed array of
  * q8_static_workspace_bytes() = 16 MiB inside the library image instead of a caller buffer.
- *  - Every GPU on which the library is loaded holds that array until the process exits.
+ *  - Every GPU on which the library is used holds that array until the process exits.  Under CUDA's default
+ *    lazy module loading the device sets the 16 MiB (and the library's kernel images) aside at the first call
+ *    into the library on that device, not when the process starts: a host that hands out all remaining device
+ *    memory must make that first call before it does so, or the call fails with Q8_ERR_CUDA (out of memory).
+ *    q8_static_workspace_bytes() is such a first call: besides returning the size it looks the array up on
+ *    the current device (and returns the size alone where there is no usable device).
  *  - A layer that would need more scratch is refused with Q8_ERR_WORKSPACE (nothing is launched);
  *    q8_conv2d with workspace = NULL still runs it, unsplit.  Layers that need none just run.
- *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that
- *    device current).  Make that first call outside any stream capture.
+ *  - The first call on each device (of q8_static_workspace_bytes or q8_conv2d_static_workspace) looks up
+ *    the array's device address (cudaGetSymbolAddress, with that device current).  Make that first call
+ *    outside any stream capture.  Later calls leave the amount of free device memory unchanged.
  *  - All calls share the one array and it keeps the previous call's contents.  Nothing needs clearing
  *    (each call writes every partial sum before reading it), but two calls whose kernels overlap on the
  *    GPU (different streams, or threads) race on it: serialise them.

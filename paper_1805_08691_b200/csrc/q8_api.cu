@@ -1,5 +1,6 @@
 // Host entry points of libq8 that are not tied to one kernel file: errors, status word,
 // descriptor validation and dispatch of q8_conv2d.
+#include <atomic>
 #include <cstdio>
 #include <cstring>
 
@@ -28,6 +29,24 @@ int check_cuda(cudaError_t e, const char* what) {
 }
 
 int check_launch(const char* kernel) { return check_cuda(cudaGetLastError(), kernel); }
+
+int current_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+  return dev;
+}
+
+int sm_count() {
+  static std::atomic<int> cached[kMaxDevices];  // zero-initialised; racing threads store the same value
+  const int dev = current_device();
+  int n = dev >= 0 ? cached[dev].load(std::memory_order_relaxed) : 0;
+  if (n == 0) {
+    int cur = 0;
+    if (cudaGetDevice(&cur) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, cur) != cudaSuccess || n <= 0) n = 148;
+    if (dev >= 0) cached[dev].store(n, std::memory_order_relaxed);
+  }
+  return n;
+}
 
 unsigned int* status_word_device_ptr() {
   // One lookup per device; the symbol address is a device address obtained from the runtime.

@@ -12,17 +12,6 @@ namespace {
 
 constexpr int kThreads = 512;
 
-int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    if (n <= 0) n = 148;
-  }
-  return n;
-}
-
 int grid_for(size_t work_items, int per_block, int blocks_per_sm) {
   size_t need = (work_items + per_block - 1) / per_block;
   size_t cap = (size_t)sm_count() * blocks_per_sm;

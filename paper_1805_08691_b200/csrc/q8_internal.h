@@ -22,6 +22,14 @@ int check_launch(const char* kernel);
 // Device status word (bit mask of timeout sites), zero when healthy.
 unsigned int* status_word_device_ptr();
 
+// Host-side caches are kept per device (function attributes, the SM count and symbol addresses belong to a
+// device, and one process may drive several from several threads).
+constexpr int kMaxDevices = 64;
+// Index of the current device, or -1 if it cannot be read or is not below kMaxDevices (callers then skip their cache).
+int current_device();
+// Multiprocessor count of the current device (148 if it cannot be read).
+int sm_count();
+
 inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

@@ -4,11 +4,14 @@ It exists for hosts that must not allocate device memory while they call this li
 out up front, or cudaMalloc forbidden because it stalls the device): the scratch of the split reduction is a
 fixed array inside the library.  This file is named to be collected last, so that a failure here cannot hide
 the result of any other test.  Every check goes through the C ABI and compares with q8_conv2d given an
-ordinary workspace: same bits, on two calls in a row (the array keeps the previous call's contents).
+ordinary workspace and with the CPU oracle: same bits, on two calls in a row (the array keeps the previous
+call's contents).  A call after the first must also leave the amount of free device memory unchanged.
 """
 import numpy as np
 import pytest
 import torch
+
+import oracle as o
 
 pytestmark = pytest.mark.gpu
 
@@ -39,10 +42,20 @@ def test_static_workspace_matches_caller_workspace_twice(q8, shape):
         want = q8.q8_conv2d(d, x, w, b, scale, res, 0.41, workspace=ws)
         got = q8.q8_conv2d_static_workspace(d, x, w, b, scale, res, 0.41)
         q8.q8_read_status()
+        ref = o.conv2d(x.cpu().numpy(), w.cpu().numpy(), b.cpu().numpy(), np.float32(3e-5), pad=(pad, pad),
+                       residual=None if res is None else res.cpu().numpy(), res_scale=np.float32(0.41), relu=True,
+                       y_type={U8: o.U8, F32: o.F32}[ytype], threads=o.hw_threads())
         a, e = got.cpu().numpy(), want.cpu().numpy()
         if a.dtype == np.float32:
-            a, e = a.view(np.uint32), e.view(np.uint32)
+            a, e, ref = a.view(np.uint32), e.view(np.uint32), ref.view(np.uint32)
         assert np.array_equal(a, e)
+        assert np.array_equal(a, ref)
+        # the entry point allocates nothing: with the output preallocated, free device memory does not move
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
+        q8.q8_conv2d_static_workspace(d, x, w, b, scale, res, 0.41, y=got)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before
 
 
 def test_static_workspace_refuses_oversized_layers_and_runs_unsplit_ones(q8):
