@@ -192,6 +192,28 @@ int q8_conv2d(const q8_conv_desc* d, const void* x, const int8_t* w, const int32
               const float* scale, const void* residual, float residual_scale, void* y,
               void* workspace, size_t workspace_bytes, void* stream);
 
+/* Two convolutions in one launch: layer 1 (descriptor d1: any filter with stride 1 that the tensor-core kernel
+ * tiles with halo patches, 32, 64 or 128 output channels, 8-bit output, no residual) followed by layer 2 (d2: 1x1,
+ * stride 1, no padding, reading exactly layer 1's output tensor, 8-bit output, optional fused residual sum).
+ * Each layer computes what q8_conv2d computes for its descriptor (Eq. int8_affine / int8_affine_fused, bias,
+ * requantization, ReLU, residual rule of Eq. arithmetics); the 8-bit tensor between them stays in shared memory
+ * and is never written (the paper's "Model Optimization" section fuses the element-wise operations into the
+ * convolution before them; this keeps the tensor between two convolutions on chip as well).  The result in y
+ * equals q8_conv2d(d2, q8_conv2d(d1, x, ...), ...) bit for bit.
+ * x: device, d1's input.  w1/bias1/scale1 and w2/bias2/scale2: device, as for q8_conv2d (bias nullable,
+ * scale_count 1 or K entries).  residual: device [N][P][Q][d2->K] of d2->res_type or NULL.  y: device, d2's
+ * output (y_ldc / y_c_offset of d2 honoured; d1's are ignored).  All pointers 16-byte aligned.
+ * Ordering contract: weights, biases and multipliers are read BEFORE the kernel orders itself behind the
+ * previous kernel of the stream, so they must not be produced by the library call enqueued immediately
+ * before on the same stream (activations and the residual may be).
+ * q8_conv2d_then_1x1_supported sets *supported to 1 if the pair can run this way (host only, no launch).
+ * Errors: Q8_ERR_INVALID_ARG, Q8_ERR_UNSUPPORTED (pair not eligible: the message names the reason; run the two
+ * layers with q8_conv2d instead), Q8_ERR_CUDA.  Nothing is launched on error. */
+int q8_conv2d_then_1x1_supported(const q8_conv_desc* d1, const q8_conv_desc* d2, int* supported);
+int q8_conv2d_then_1x1(const q8_conv_desc* d1, const q8_conv_desc* d2, const void* x, const int8_t* w1,
+                       const int32_t* bias1, const float* scale1, const int8_t* w2, const int32_t* bias2,
+                       const float* scale2, const void* residual, float residual_scale, void* y, void* stream);
+
 /* q8_conv2d for callers that cannot allocate device memory (the paper has no counterpart; this is a
  * property of the library, not of the method).  Meant for hosts where every byte of device memory was
  * handed out before this library is called, or where cudaMalloc is off limits because it stalls the

@@ -21,7 +21,7 @@ TORCH_DTYPES = {Q8_U8: torch.uint8, Q8_S8: torch.int8, Q8_S32: torch.int32, Q8_F
 EXPORTS = ["q8_version", "q8_last_error", "q8_read_status", "q8_calibrate_maxabs", "q8_factor", "q8_requant_scale",
            "q8_bias_factor", "q8_quantize", "q8_quantize_pad_channels", "q8_dequantize", "q8_fold_bn",
            "q8_conv2d_workspace_bytes", "q8_conv2d_query_algo", "q8_conv2d", "q8_static_workspace_bytes",
-           "q8_conv2d_static_workspace", "q8_concat", "q8_concat_branch", "q8_calibrate_maxabs_rows", "q8_quantize_rows", "q8_quantize_pad_image", "q8_pool_out_extent",
+           "q8_conv2d_static_workspace", "q8_conv2d_then_1x1_supported", "q8_conv2d_then_1x1", "q8_concat", "q8_concat_branch", "q8_calibrate_maxabs_rows", "q8_quantize_rows", "q8_quantize_pad_image", "q8_pool_out_extent",
            "q8_maxpool2d", "q8_avgpool2d"]
 
 
@@ -66,6 +66,8 @@ lib.q8_conv2d_workspace_bytes.argtypes = [C.POINTER(q8_conv_desc), C.POINTER(_sz
 lib.q8_conv2d_query_algo.argtypes = [C.POINTER(q8_conv_desc), _ip]
 lib.q8_conv2d.argtypes = [C.POINTER(q8_conv_desc), _vp, _vp, _vp, _vp, _vp, _f, _vp, _vp, _sz, _vp]
 lib.q8_static_workspace_bytes.argtypes = []
+lib.q8_conv2d_then_1x1_supported.argtypes = [C.POINTER(q8_conv_desc), C.POINTER(q8_conv_desc), _ip]
+lib.q8_conv2d_then_1x1.argtypes = [C.POINTER(q8_conv_desc), C.POINTER(q8_conv_desc), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _f, _vp, _vp]
 lib.q8_conv2d_static_workspace.argtypes = [C.POINTER(q8_conv_desc), _vp, _vp, _vp, _vp, _vp, _f, _vp, _vp]
 lib.q8_concat.argtypes = [_i, C.POINTER(_vp), _ip, _fp, _f, _i, _sz, _vp, _vp]
 lib.q8_calibrate_maxabs_rows.argtypes = [_vp, _sz, _sz, _vp, _vp]
@@ -211,6 +213,23 @@ def q8_conv2d(d, x, w, bias, scale, residual=None, residual_scale=0.0, y=None, w
     _check(lib.q8_conv2d(C.byref(d), _dev(x, "x"), _dev(w, "w"), _dev(bias, "bias"), _dev(scale, "scale"),
                          _dev(residual, "residual"), residual_scale, _dev(y, "y"), _dev(workspace, "workspace"),
                          ws_bytes, _stream()))
+    return y
+
+
+def q8_conv2d_then_1x1_supported(d1, d2):
+    ok = C.c_int(0)
+    _check(lib.q8_conv2d_then_1x1_supported(C.byref(d1), C.byref(d2), C.byref(ok)))
+    return bool(ok.value)
+
+
+def q8_conv2d_then_1x1(d1, d2, x, w1, bias1, scale1, w2, bias2, scale2, residual=None, residual_scale=0.0, y=None):
+    """Layer d1 followed by the 1x1 layer d2 in one launch; the tensor between them is never written."""
+    if y is None:
+        P, Q = conv_out_shape(d2)
+        y = torch.empty((d2.N, P, Q, d2.y_ldc or d2.K), dtype=TORCH_DTYPES[d2.y_type], device=x.device)
+    _check(lib.q8_conv2d_then_1x1(C.byref(d1), C.byref(d2), _dev(x, "x"), _dev(w1, "w1"), _dev(bias1, "bias1"),
+                                  _dev(scale1, "scale1"), _dev(w2, "w2"), _dev(bias2, "bias2"), _dev(scale2, "scale2"),
+                                  _dev(residual, "residual"), residual_scale, _dev(y, "y"), _stream()))
     return y
 
 

@@ -180,4 +180,32 @@ int q8_conv2d(const q8_conv_desc* d, const void* x, const int8_t* w, const int32
   return launch_conv_umma(a);
 }
 
+int q8_conv2d_then_1x1_supported(const q8_conv_desc* d1, const q8_conv_desc* d2, int* supported) {
+  clear_error();
+  int P, Q;
+  int rc = validate_desc(d1, &P, &Q);
+  if (rc != Q8_OK) return rc;
+  rc = validate_desc(d2, &P, &Q);
+  if (rc != Q8_OK) return rc;
+  if (!supported) return fail(Q8_ERR_INVALID_ARG, "q8_conv2d_then_1x1_supported: null pointer");
+  const char* why = "";
+  *supported = (d1->algo != Q8_ALGO_DIRECT && d2->algo != Q8_ALGO_DIRECT && fused_pair_eligible(*d1, *d2, &why)) ? 1 : 0;
+  return Q8_OK;
+}
+
+int q8_conv2d_then_1x1(const q8_conv_desc* d1, const q8_conv_desc* d2, const void* x, const int8_t* w1, const int32_t* bias1,
+                       const float* scale1, const int8_t* w2, const int32_t* bias2, const float* scale2,
+                       const void* residual, float residual_scale, void* y, void* stream) {
+  clear_error();
+  int P, Q;
+  int rc = validate_desc(d1, &P, &Q);
+  if (rc != Q8_OK) return rc;
+  rc = validate_desc(d2, &P, &Q);
+  if (rc != Q8_OK) return rc;
+  if (!x || !w1 || !w2 || !y || !scale1 || !scale2) return fail(Q8_ERR_INVALID_ARG, "q8_conv2d_then_1x1: null x, w1, w2, y, scale1 or scale2");
+  if (!aligned16(x) || !aligned16(w1) || !aligned16(w2) || !aligned16(y))
+    return fail(Q8_ERR_UNSUPPORTED, "q8_conv2d_then_1x1: x, w1, w2 and y must be 16-byte aligned");
+  return launch_conv_fused(*d1, *d2, x, w1, bias1, scale1, w2, bias2, scale2, residual, residual_scale, y, as_stream(stream));
+}
+
 }  // extern "C"

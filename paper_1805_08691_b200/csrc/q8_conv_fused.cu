@@ -285,10 +285,7 @@ __global__ void __launch_bounds__(kFThreads, 1)
       prev_slot = (int)slot;
       if (++slot == nslots) { slot = 0; spar ^= 1u; }
     }
-    if (lane0) {
-      bulk_wait_read<0>();  // the CTA's shared memory must outlive the reads of its last stores
-      if (ok && prev_slot >= 0 && !ld.done(m_tiles)) load_residual(ld, (uint32_t)prev_slot);  // never true: all items stored
-    }
+    if (lane0) bulk_wait_read<0>();  // the CTA's shared memory must outlive the reads of its last stores
     if (!ok && lane0) { abort_flag = 1; atomicOr(p.l1.status, kTimeoutStore); }
   } else if (warp < kFCtrlWarps + 4) {
     // ------------------------------------------------------------------ E1: layer-1 accumulator -> T[slot]

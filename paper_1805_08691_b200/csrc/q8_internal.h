@@ -63,5 +63,11 @@ int umma_plan_splits(const q8_conv_desc& d, int P, int Q, long long M);
 // Sums the split-K partial accumulators in a.workspace, adds the bias and applies the epilogue of `a`.
 int launch_splitk_reduce(const ConvArgs& a, int splits);
 int launch_conv_direct(const ConvArgs& a);
+// A stride-1 convolution followed by a 1x1 convolution over its output, in one launch (q8_conv_fused.cu).
+// Descriptors validated by the caller; `why` names the first reason a pair cannot run fused.
+bool fused_pair_eligible(const q8_conv_desc& d1, const q8_conv_desc& d2, const char** why);
+int launch_conv_fused(const q8_conv_desc& d1, const q8_conv_desc& d2, const void* x, const int8_t* w1, const int32_t* bias1,
+                      const float* scale1, const int8_t* w2, const int32_t* bias2, const float* scale2, const void* residual,
+                      float residual_scale, void* y, cudaStream_t stream);
 
 }  // namespace q8
