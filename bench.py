@@ -4,15 +4,22 @@
     python bench.py --gpus N --steps K --warmup W [--impl reference]
 
 One step = one int8 forward of the bottleneck block (1x1 256->64, 3x3 64->64, 1x1 64->256 with fused
-bias, requantisation, ReLU and residual sum) over a batch of 32 56x56x256 u8 images: three launches
-of the tcgen05 convolution kernel through the C ABI.  Prints ONE JSON line (rank 0).
+bias, requantisation, ReLU and residual sum) over a batch of 32 56x56x256 u8 images: two launches
+through the C ABI (the 1x1, then the 3x3 and the expanding 1x1 as one tcgen05 kernel whose 8-bit tensor
+between the two layers stays in shared memory).  Prints ONE JSON line (rank 0).
 
-* value      : int8 conv TOPS (2 * MACs / time), inputs resident in HBM, steps replayed as CUDA
-               graphs over rotating buffer sets whose total size exceeds L2.
+* value      : int8 conv TOPS (2 * MACs / time), inputs resident in HBM, the K steps captured as one CUDA
+               graph over rotating buffer sets whose total size exceeds L2; the graph is replayed until the
+               timed region lasts at least 0.25 s and the median time of a replay counts (timed_repeats).
 * e2e        : same metric with the u8 input of every step copied from pinned host memory and its u8 output
                copied back inside the timed region (three streams: the copies overlap the kernels).
 * roofline   : dominant kernel, algorithmic bytes / CUDA-event duration against the measured copy peak.
 * cpu_baseline: the CPU oracle timed on a bounded sample of the same workload on the host cores.
+* int8_mma_peak: issue rate of tcgen05.mma.kind::i8 128x256x32 measured on all SMs (q8_int8_mma_rate), the
+               int8 tensor peak every roofline below uses, at the SM clock sampled during the run.
+* config1    : latency of the single 14x14x64 3x3 layer (configs[0]) in microseconds.
+* resnet50_layers: every launch of ResNet-50 at batch 64 alone, cold L2: us, TOPS, bytes, bound, fraction of
+               its roofline max(2 MACs / int8 peak, bytes / copy bandwidth).
 * bandwidth_kernels: the memory-bound kernels (max-abs, quantize, dequantize, concat, pooling) against the measured
                copy bandwidth; networks: int8 forward of ResNet-50, Inception-v3 and SSD-300 (images/s), with the
                paper's Xeon figures beside them as context.  Both only at N = 1; --skip-networks leaves them out.
@@ -20,6 +27,7 @@ of the tcgen05 convolution kernel through the C ABI.  Prints ONE JSON line (rank
 With N > 1 every rank runs its own batch (weak scaling, replicated weights, no data-path collective).
 """
 import argparse
+import hashlib
 import json
 import os
 import statistics
@@ -40,11 +48,26 @@ CONFIG = {"workload": "configs[1]: ResNet-50 bottleneck, batch 32, 56x56x256 u8 
                       "1x1 64->256 + identity residual, BN folded, ReLU fused, max-abs factors from 4 seeded batches",
           "global_batch_per_gpu": BATCH, "parallelism": "replicas"}
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel from
-# the ncu capture summarised in profiles/conv_umma_bottleneck_b32.md.  Below the algorithmic bytes where the
-# output of a launch stays in the 126 MB L2 until a later launch evicts it (the write-back is charged there).
-NCU_TRAFFIC_BYTES = {"conv_umma 1x1 256->64": 25807104, "conv_umma 3x3 64->64": 6570496,
-                     "conv_umma 1x1 64->256 +res": 32237056 + 205312}
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of a kernel, from one ncu capture of
+# this workload, with the hash of the kernel sources the capture was taken with: the figure is reported only while
+# the sources still have that hash (a changed kernel has unknown traffic: null).  Traffic can lie below the
+# algorithmic bytes: the output of a launch stays in the 126 MB L2 until later launches evict it.
+NCU_TRAFFIC = {"source_sha256": "", "bytes": {}}
+KERNEL_SOURCES = ["q8_umma_common.cuh", "q8_conv_umma.cu", "q8_conv_fused.cu"]
+
+
+def kernel_source_hash():
+    h = hashlib.sha256()
+    for f in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_1805_08691_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()
+
+
+def ncu_traffic(kernel):
+    if NCU_TRAFFIC["source_sha256"] and NCU_TRAFFIC["source_sha256"] == kernel_source_hash():
+        return NCU_TRAFFIC["bytes"].get(kernel)
+    return None
 
 
 def layer_bytes(M, Cin, K, R, S, out_bytes=1, residual=False):
@@ -56,8 +79,8 @@ def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         d = json.load(open(p))
-        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"], source="measured")
-    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, source="fallback")
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"], sm_max_mhz=d.get("sm_max_mhz", 1965.0), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, sm_max_mhz=1965.0, source="fallback")
 
 
 class ClockMonitor:
@@ -300,12 +323,162 @@ def network_numbers(dev, name, reps=20):
     return out
 
 
+def int8_mma_peak(dev, sms):
+    """Issue rate of tcgen05.mma.kind::i8 (128 x 256 x 32, two alternating accumulators) on every SM: cycles per
+    instruction (slowest CTA, median of five launches) and the MACs per clock and SM that follow."""
+    import torch
+    import paper_1805_08691_b200 as q8
+    n = 8192
+    cyc = torch.zeros(sms, dtype=torch.int64, device=dev)
+    per, tops = [], []
+    for i in range(6):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        q8.q8_int8_mma_rate(256, 2, n, sms, cyc)
+        e1.record()
+        torch.cuda.synchronize()
+        if i:
+            per.append(cyc.max().item() / n)
+            tops.append(2.0 * 128 * 256 * 32 * n * sms / e0.elapsed_time(e1) / 1e9)
+    q8.q8_read_status()
+    c = statistics.median(per)
+    return {"instruction": "tcgen05.mma.cta_group::1.kind::i8 128x256x32", "instructions_per_sm": n, "sms": sms,
+            "cycles_per_instruction": c, "macs_per_clk_per_sm": 128 * 256 * 32 / c,
+            "TOPS_whole_launch": statistics.median(tops)}
+
+
+def config1_numbers(dev):
+    """configs[0]: the single 1x14x14x64 3x3 layer, launch-latency bound: microseconds per launch from a CUDA graph of
+    200 back-to-back launches, and the single-thread oracle beside it."""
+    import torch
+    import paper_1805_08691_b200 as q8
+    import oracle as o
+    g = np.random.default_rng(0)
+    x = g.integers(0, 256, (1, 14, 14, 64), dtype=np.uint8)
+    w = g.integers(-128, 128, (64, 3, 3, 64)).astype(np.int8)
+    b = g.integers(-2000, 2000, 64).astype(np.int32)
+    d = q8.make_conv_desc(1, 14, 14, 64, 64, 3, 3, (1, 1), (1, 1), (1, 1), relu=True)
+    xt, wt, bt = (torch.from_numpy(a).to(dev) for a in (x, w, b))
+    sc = torch.tensor([2e-4], device=dev)
+    y = torch.empty((1, 14, 14, 64), dtype=torch.uint8, device=dev)
+    q8.q8_conv2d(d, xt, wt, bt, sc, None, 0.0, y)
+    torch.cuda.synchronize()
+    gr = torch.cuda.CUDAGraph()
+    n = 200
+    with torch.cuda.graph(gr):
+        for _ in range(n):
+            q8.q8_conv2d(d, xt, wt, bt, sc, None, 0.0, y)
+    gr.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(5):
+        gr.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / (5 * n)
+    t0 = time.perf_counter()
+    for _ in range(5):
+        o.conv2d(x, w, b, np.float32(2e-4), pad=(1, 1), relu=True, threads=1)
+    cpu_us = (time.perf_counter() - t0) / 5 * 1e6
+    macs = 14 * 14 * 64 * 9 * 64
+    return {"workload": "configs[0]: 1x14x14x64 u8, 3x3 pad 1, 64 output channels, bias + requantize + ReLU",
+            "us_per_launch": us, "launches_in_graph": n, "TOPS": 2.0 * macs / us / 1e6,
+            "oracle_single_thread_us": cpu_us}
+
+
+def resnet50_layer_table(dev, peak_gbs, int8_peak_tops, batch=64, reps=10):
+    """Every launch of ResNet-50 at `batch`, alone: CUDA graph of reps x [evict L2, launch] minus a graph of the
+    evictions alone.  Roofline of a launch: max(2 MACs / int8 peak, algorithmic bytes / copy bandwidth)."""
+    import torch
+    import paper_1805_08691_b200 as q8
+    from paper_1805_08691_b200 import network, pipeline
+    from workloads import nets
+
+    def cuda(a):
+        return torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+
+    layers = nets.resnet50()
+    folded = {}
+    for L in layers:
+        if L.op == "conv":
+            sp = L.conv
+            folded[L.name] = (q8.q8_fold_bn(cuda(sp.w), None, cuda(sp.gamma), cuda(sp.beta), cuda(sp.mean), cuda(sp.var), 1e-5)
+                              if sp.bn else (cuda(sp.w), cuda(sp.b)))
+    folded_np = {k: (w.cpu().numpy(), b.cpu().numpy()) for k, (w, b) in folded.items()}
+    acts = nets.fp32_forward(layers, nets.images(3010, 2, 224), folded_np, device=dev)
+    cal = pipeline.Calibrator(sorted(acts), device=dev)
+    for k, v in acts.items():
+        cal.observe(k, cuda(v))
+    maxima = cal.maxima()
+    del acts
+    net = network.QuantNetwork(layers, folded, maxima, (batch, 224, 224, 3), device=dev, streams=1)
+    net.forward(cuda(nets.images(3001, batch, 224)))
+    torch.cuda.synchronize()
+    q8.q8_read_status()
+    evict = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def timed_graph(fn):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for _ in range(reps):
+                evict.zero_()
+                if fn is not None:
+                    fn()
+        g.replay()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(3):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            g.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        return statistics.median(ts) * 1e3 / reps   # us per [evict, launch]
+
+    base_us = timed_graph(None)
+    rows = []
+    ws = net.workspaces[0]
+    for L in layers:
+        if L.op != "conv" or L.name in net.fused_with or L.name in net.skip:
+            continue
+        parts = [L]
+        if L.name in net.fused_second:
+            parts = [net.by_name[L.src[0]], L]
+        macs, nbytes = 0, 0
+        for i, P in enumerate(parts):
+            d = net.convs[P.name].desc
+            pq = q8.conv_out_shape(d)
+            m = d.N * pq[0] * pq[1]
+            macs += m * P.conv.K * P.conv.R * P.conv.S * P.conv.C       # true channel counts
+            nbytes += d.K * d.R * d.S * d.C + 4 * d.K
+            if i == 0:
+                nbytes += d.N * d.H * d.W * d.C
+            if i == len(parts) - 1:
+                nbytes += m * d.K * (4 if P.f32_out else 1) + (m * d.K if P.residual else 0)
+        us = timed_graph(lambda: net._launch(L, ws)) - base_us
+        t_mma, t_hbm = 2.0 * macs / int8_peak_tops / 1e6, nbytes / peak_gbs / 1e3     # us
+        sp = parts[0].conv
+        rows.append({"layer": "+".join(P.name for P in parts),
+                     "shape": "%dx%d %d->%d %dx%d/%d" % (net.convs[parts[0].name].desc.H, net.convs[parts[0].name].desc.W,
+                                                         sp.C, parts[-1].conv.K, sp.R, sp.S, sp.stride[0]) + (" + 1x1" if len(parts) > 1 else ""),
+                     "us": us, "TOPS": 2.0 * macs / us / 1e6, "bytes": nbytes, "GB/s": nbytes / us / 1e3,
+                     "bound": "tensor" if t_mma >= t_hbm else "hbm", "roofline_us": max(t_mma, t_hbm),
+                     "frac": max(t_mma, t_hbm) / us})
+    del net
+    torch.cuda.empty_cache()
+    return {"batch": batch, "l2": "256 MB written between launches (cold inputs)", "evict_us": base_us, "layers": rows,
+            "sum_us": sum(r["us"] for r in rows), "sum_roofline_us": sum(r["roofline_us"] for r in rows)}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
     import paper_1805_08691_b200 as q8
     from paper_1805_08691_b200 import pipeline
     import workloads as wl
+    from workloads import synth
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -316,12 +489,14 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
 
     def cuda(a):
         return torch.from_numpy(np.ascontiguousarray(a)).to(dev)
 
-    # ---- preparation (untimed): fold BN, calibrate on 4 seeded batches, quantize weights/bias
-    cfg = wl.config2(seed=2000 + rank, batch=BATCH, calib_batches=4, calib_batch=8)
+    # ---- preparation (untimed): fold BN, calibrate on 4 seeded batches, quantize weights/bias.  Weights and
+    # calibration batches are the same on every rank (replicas); only the images of a rank's batch differ.
+    cfg = wl.config2(seed=2000, batch=BATCH, calib_batches=4, calib_batch=8)
     folded = []
     for sp in cfg["convs"]:
         folded.append(q8.q8_fold_bn(cuda(sp.w), None, cuda(sp.gamma), cuda(sp.beta), cuda(sp.mean), cuda(sp.var), 1e-5))
@@ -334,9 +509,11 @@ def run_ours(args):
             cal.observe(k, cuda(s[k]))
     maxima = pipeline.sync_maxima(cal.maxima(), dev if world > 1 else None)
     shape = (BATCH, H, W, C)
-    x_f32 = cuda(cfg["x"])
+    x_np = cfg["x"] if rank == 0 else synth.relu_normal(synth.rng(2001 + 100 * rank), shape)
+    x_f32 = cuda(x_np)
     n_sets = max(2, args.sets)
     blocks = [pipeline.Bottleneck(folded, maxima, shape) for _ in range(n_sets)]
+    fused = blocks[0].fused
     xs = [q8.q8_quantize(x_f32.roll(i, dims=0), blocks[0].q_x, q8.Q8_U8) for i in range(n_sets)]
     ys = [torch.empty(shape, dtype=torch.uint8, device=dev) for _ in range(n_sets)]
     del x_f32
@@ -355,34 +532,36 @@ def run_ours(args):
         with torch.cuda.graph(g):
             blocks[i](xs[i], out=ys[i])
         graphs.append(g)
-    # the timed region is ONE graph holding all K steps (step i works on buffer set i % n_sets), so that no
-    # host launch gap sits between steps
-    # (for large K: a graph of `chunk` steps, chunk the largest divisor of K up to 240 that is a multiple of the
-    # number of buffer sets when there is one, replayed K / chunk times back to back)
+    # the timed region replays ONE graph holding the K steps (step i works on buffer set i % n_sets), so that no
+    # host launch gap sits between steps (K > 240: a graph of the largest divisor of K up to 240, replayed K / chunk
+    # times per repeat)
     chunk = args.steps
     if chunk > 240:
         divs = [d for d in range(240, 0, -1) if args.steps % d == 0]
         chunk = next((d for d in divs if d % n_sets == 0), divs[0])
-    timed_reps = args.steps // chunk
+    replays_per_repeat = args.steps // chunk
     timed = torch.cuda.CUDAGraph()
     with torch.cuda.graph(timed):
         for i in range(chunk):
             blocks[i % n_sets](xs[i % n_sets], out=ys[i % n_sets])
-    # one graph per layer for the per-kernel durations: the same launch repeated over all buffer sets
+    # one graph per launch kind for the per-kernel durations: the same launch repeated over all buffer sets
     kreps = 8
+    kinds = ["a", "bc"] if fused else ["a", "b", "c"]
     kgraphs = []
-    for j in range(3):
+    for kind in kinds:
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
             for _ in range(kreps):
                 for i in range(n_sets):
                     blk = blocks[i]
-                    if j == 0:
+                    if kind == "a":
                         blk.a(xs[i], out=blk.ya)
-                    elif j == 1:
+                    elif kind == "b":
                         blk.b(blk.ya, out=blk.yb)
-                    else:
+                    elif kind == "c":
                         blk.c(blk.yb, residual=xs[i], out=ys[i])
+                    else:
+                        pipeline.fused_pair(blk.b, blk.c, blk.ya, residual=xs[i], out=ys[i])
         kgraphs.append(g)
 
     def barrier():
@@ -396,7 +575,8 @@ def run_ours(args):
     mon = ClockMonitor(local)
     if rank == 0:
         mon.start()
-    # keep the monitor sampling for a moment under load before the timed region
+    # keep the monitor sampling for a moment under load before the timed region; the step time seen here sizes
+    # the number of repeats
     t_end = time.time() + 0.3
     i = 0
     while time.time() < t_end:
@@ -404,16 +584,29 @@ def run_ours(args):
         i += 1
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    timed.replay()  # untimed: first replay of a graph uploads it
-    barrier()
     e0.record()
-    for _ in range(timed_reps):
-        timed.replay()
+    timed.replay()  # untimed: first replay of a graph uploads it
     e1.record()
     barrier()
-    ms_total = e0.elapsed_time(e1)
+    est_ms = max(e0.elapsed_time(e1) * replays_per_repeat, 1e-3)
+    repeats = int(min(2000, max(3, -(-250.0 // est_ms))))
+    if world > 1:
+        r_t = torch.tensor([repeats], dtype=torch.int64, device=dev)
+        dist.all_reduce(r_t, op=dist.ReduceOp.MAX)
+        repeats = int(r_t.item())
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(repeats + 1)]
+    barrier()
+    evs[0].record()
+    for r in range(repeats):
+        for _ in range(replays_per_repeat):
+            timed.replay()
+        evs[r + 1].record()
+    barrier()
+    rep_ms = [evs[r].elapsed_time(evs[r + 1]) for r in range(repeats)]
+    ms_total = statistics.median(rep_ms)          # K steps
+    ms_min, ms_region = min(rep_ms), evs[0].elapsed_time(evs[repeats])
 
-    # ---- per-kernel durations: CUDA events around a graph of kreps * n_sets launches of one layer
+    # ---- per-kernel durations: CUDA events around a graph of kreps * n_sets launches of one kind
     kms = []
     for g in kgraphs:
         g.replay()
@@ -423,6 +616,7 @@ def run_ours(args):
         e1.record()
         torch.cuda.synchronize()
         kms.append(e0.elapsed_time(e1) / (kreps * n_sets))
+    mma_peak = int8_mma_peak(dev, sms) if rank == 0 else None
     barrier()
     clocks = mon.stop() if rank == 0 else None
 
@@ -475,10 +669,10 @@ def run_ours(args):
     ms_e2e = e0.elapsed_time(e1) / esteps
     q8.q8_read_status()
 
-    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
+    t = torch.tensor([ms_total, ms_e2e, ms_min, ms_region], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, ms_e2e = t.tolist()
+    ms_total, ms_e2e, ms_min, ms_region = t.tolist()
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -487,34 +681,51 @@ def run_ours(args):
     ms_step = ms_total / args.steps
     ops_step = 2.0 * MACS_PER_IMAGE * BATCH * world
     peaks = measured_peaks()
+    # int8 tensor peak: the measured issue rate (MACs per clock and SM) at the SM clock sampled during this run
+    sm_mhz = (clocks or {}).get("sm_mhz") or peaks["sm_max_mhz"]
+    int8_peak = sms * mma_peak["macs_per_clk_per_sm"] * 2.0 * sm_mhz * 1e6 / 1e12
+    mma_peak.update({"sm_mhz_used": sm_mhz, "peak_TOPS_at_sampled_clock": int8_peak,
+                     "peak_TOPS_at_max_clock": sms * mma_peak["macs_per_clk_per_sm"] * 2.0 * peaks["sm_max_mhz"] * 1e6 / 1e12,
+                     "for_context_2x_bf16_burst_TOPS": 2.0 * peaks["bf16_tflops"]})
     M = BATCH * H * W
-    kinfo = [("conv_umma 1x1 256->64", layer_bytes(M, C, MID, 1, 1), 2.0 * M * C * MID),
-             ("conv_umma 3x3 64->64", layer_bytes(M, MID, MID, 3, 3), 2.0 * M * 9 * MID * MID),
-             ("conv_umma 1x1 64->256 +res", layer_bytes(M, MID, C, 1, 1, residual=True), 2.0 * M * MID * C)]
-    int8_peak = peaks["bf16_tflops"] * 2.0  # nominal int8:bf16 dense ratio 4.5 : 2.25
+    if fused:
+        kinfo = [("conv_umma 1x1 256->64", layer_bytes(M, C, MID, 1, 1), 2.0 * M * C * MID),
+                 ("conv_fused 3x3 64->64 + 1x1 64->256 +res",
+                  M * MID + 9 * MID * MID + 4 * MID + MID * C + 4 * C + 2 * M * C, 2.0 * M * (9 * MID * MID + MID * C))]
+    else:
+        kinfo = [("conv_umma 1x1 256->64", layer_bytes(M, C, MID, 1, 1), 2.0 * M * C * MID),
+                 ("conv_umma 3x3 64->64", layer_bytes(M, MID, MID, 3, 3), 2.0 * M * 9 * MID * MID),
+                 ("conv_umma 1x1 64->256 +res", layer_bytes(M, MID, C, 1, 1, residual=True), 2.0 * M * MID * C)]
     kernels = []
     for (name, nbytes, ops), ms in zip(kinfo, kms):
         kernels.append({"kernel": name, "ms": ms, "GB/s": nbytes / ms / 1e6, "TOPS": ops / ms / 1e9,
                         "roofline_ms": max(nbytes / peaks["hbm_gbs"] / 1e6, ops / int8_peak / 1e9)})
-    dom = max(range(3), key=lambda j: kms[j])
+    dom = max(range(len(kms)), key=lambda j: kms[j])
     achieved = kinfo[dom][1] / kms[dom] / 1e6
     roofline = {"bound": "hbm", "kernel": kinfo[dom][0], "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                "algorithmic_bytes_per_launch": kinfo[dom][1], "traffic": NCU_TRAFFIC_BYTES.get(kinfo[dom][0])}
+                "algorithmic_bytes_per_launch": kinfo[dom][1], "traffic": ncu_traffic(kinfo[dom][0])}
     line = {"metric": METRIC, "value": ops_step / ms_step / 1e9, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "s32", "data": "synthetic",
-            "config": dict(CONFIG, l2="rotating %d buffer sets of %.0f MB (> 126 MB L2)" % (n_sets, set_bytes / 1e6),
-                           launch="CUDA graph of %d steps replayed %d times back to back" % (chunk, timed_reps)),
+            "config": CONFIG,
+            "timing": {"l2": "rotating %d buffer sets of %.0f MB (> 126 MB L2)" % (n_sets, set_bytes / 1e6),
+                       "launch": "CUDA graph of %d steps, %d replays per repeat" % (chunk, replays_per_repeat),
+                       "timed_repeats": repeats, "statistic": "median over the repeats of the time of K steps",
+                       "ms_per_step_min": ms_min / args.steps, "timed_region_ms": ms_region},
             "clocks": clocks,
             "e2e": {"value": ops_step / ms_e2e / 1e9, "unit": UNIT, "ms_per_step": ms_e2e,
                     "h2d_bytes_per_step": BATCH * H * W * C, "d2h_bytes_per_step": BATCH * H * W * C,
                     "pipeline": "H2D, kernels and D2H of neighbouring steps overlap on three streams"},
-            "gpu_launches": 3 * args.steps,
-            "roofline": roofline, "kernels": kernels,
+            "gpu_launches": len(kinds) * args.steps * repeats,
+            "launches_per_step": len(kinds),
+            "roofline": roofline, "kernels": kernels, "int8_mma_peak": mma_peak,
             "images_per_s": BATCH * world / ms_step * 1e3}
+    if world == 1:
+        line["config1"] = config1_numbers(dev)
     if world == 1 and not args.skip_networks:
         line["bandwidth_kernels"] = bandwidth_kernel_numbers(dev, peaks["hbm_gbs"])
+        line["resnet50_layers"] = resnet50_layer_table(dev, peaks["hbm_gbs"], int8_peak)
         line["networks"] = {name: network_numbers(dev, name) for name in NETWORKS}
     if world == 1 and not args.skip_cpu_baseline:
         r = oracle_time_steps(steps=2, warmup=1)

@@ -214,6 +214,16 @@ int q8_conv2d_then_1x1(const q8_conv_desc* d1, const q8_conv_desc* d2, const voi
                        const int32_t* bias1, const float* scale1, const int8_t* w2, const int32_t* bias2,
                        const float* scale2, const void* residual, float residual_scale, void* y, void* stream);
 
+/* Measurement aid (the paper has no counterpart): issue rate of the int8 tensor-core instruction behind Eq.
+ * int8_affine's contraction, used as the measured "int8 tensor peak" of the convolution roofline.  Launches `ctas`
+ * CTAs (one per SM is the intended use); each issues `instructions` tcgen05.mma.kind::i8 of shape 128 x bn x 32 back
+ * to back on zeroed shared-memory operands, cycling over `chains` TMEM accumulators (1: each instruction depends on
+ * its predecessor), and writes the SM cycles from first issue to last completion to cycles_dev[cta] (device, `ctas`
+ * entries, caller-owned).  Asynchronous on `stream`; a bounded wait that runs out shows in q8_read_status.
+ * MACs per CTA = instructions * 128 * bn * 32.  bn: multiple of 16 in [16,256]; chains * max(bn,32) <= 512.
+ * Errors: Q8_ERR_INVALID_ARG, Q8_ERR_CUDA. */
+int q8_int8_mma_rate(int bn, int chains, int instructions, int ctas, unsigned long long* cycles_dev, void* stream);
+
 /* q8_conv2d for callers that cannot allocate device memory (the paper has no counterpart; this is a
  * property of the library, not of the method).  Meant for hosts where every byte of device memory was
  * handed out before this library is called, or where cudaMalloc is off limits because it stalls the

@@ -48,13 +48,15 @@ struct FusedParams {
 // One (m tile, chunk) item of layer 2 in this CTA's sequence, with the tile's image coordinates.
 struct ItemIter {
   TileIterT<false> ti;
-  int j;
-  __device__ __forceinline__ void init(const UmmaParams& l1) {
-    ti.init(l1, blockIdx.x, gridDim.x);
-    j = 0;
+  int j, left;
+  __device__ __forceinline__ void init(const UmmaParams& l1, int t0, int j0, int count) {
+    ti.init(l1, t0, 1);
+    j = j0;
+    left = count;
   }
-  __device__ __forceinline__ bool done(int m_tiles) const { return ti.tile >= m_tiles; }
+  __device__ __forceinline__ bool done() const { return left <= 0; }
   __device__ __forceinline__ void next(const UmmaParams& l1, int chunks) {
+    --left;
     if (++j == chunks) { j = 0; ti.next(l1); }
   }
 };
@@ -86,7 +88,23 @@ __global__ void __launch_bounds__(kFThreads, 1)
   float* const s_scale2 = reinterpret_cast<float*>(base_ptr + p.off_chan2) + p.l2.k_pad;
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   const bool lane0 = lane == 0;
-  const int m_tiles = p.l1.m_tiles, chunks = p.l2.n_tiles;
+  // Work split.  The unit is one item = (m tile, chunk of layer-2 output channels); items are numbered tile by tile
+  // and every CTA takes a contiguous range of them, so that the CTAs' loads differ by at most one item (whole tiles
+  // per CTA would leave most SMs idle for up to a tile's time at the end).  A CTA whose range starts or ends inside a
+  // tile computes layer 1 of that tile as well: the tensor pipe has time to spare, the epilogue of layer 2 has not.
+  const int chunks = p.l2.n_tiles;
+  int t0, j0, j1, my_items, my_tiles;
+  {
+    const int total = p.l1.m_tiles * chunks, per = total / (int)gridDim.x, rem = total - per * (int)gridDim.x;
+    const int c = (int)blockIdx.x;
+    my_items = per + (c < rem ? 1 : 0);
+    const int begin = c * per + (c < rem ? c : rem), last = begin + my_items - 1;
+    t0 = begin / chunks;
+    j0 = begin - t0 * chunks;
+    const int t1 = last / chunks;
+    j1 = last - t1 * chunks + 1;
+    my_tiles = my_items > 0 ? t1 - t0 + 1 : 0;
+  }
 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
@@ -159,7 +177,7 @@ __global__ void __launch_bounds__(kFThreads, 1)
   if (warp == 0) {
     // ------------------------------------------------------------------ layer-1 producer: patches and the weight ring
     TileIterT<false> ti;
-    ti.init(p.l1, blockIdx.x, gridDim.x);
+    ti.init(p.l1, t0, 1);
     const UmmaParams& q = p.l1;
     const uint32_t nstages = (uint32_t)q.stages, nbst = (uint32_t)q.b_stages;
     const uint32_t afull0 = smem_u32(&a_full[0]), aempty0 = smem_u32(&a_empty[0]);
@@ -169,7 +187,7 @@ __global__ void __launch_bounds__(kFThreads, 1)
     uint32_t bs = 0, bphase = 0, b_dst = bring0;
     const uint32_t b_tx = (uint32_t)q.b_T * q.b_tile_bytes;
     bool ok = true;
-    for (; ti.tile < m_tiles && ok; ti.next(q)) {
+    for (int k = 0; k < my_tiles && ok; ++k, ti.next(q)) {
       const int q0 = ti.qt * q.tw - q.pad_w, p0 = ti.pt * q.th - q.pad_h;
       for (int c = 0; c < q.C_pad && ok; c += q.bk) {
         if (!mbar_wait(aempty0 + stage * 8u, phase ^ 1u, abortp)) { ok = false; break; }
@@ -198,7 +216,8 @@ __global__ void __launch_bounds__(kFThreads, 1)
   } else if (warp == 1) {
     // ------------------------------------------------------------------ layer-1 MMA issue
     MmaRoleArgs ra;
-    ra.base = base; ra.tmem_base = tmem_base + (uint32_t)p.acc1_col; ra.total_tiles = m_tiles; ra.abortp = abortp;
+    ra.base = base; ra.tmem_base = tmem_base + (uint32_t)p.acc1_col; ra.total_tiles = t0 + my_tiles; ra.abortp = abortp;
+    ra.first_tile = t0; ra.tile_step = 1;
     ra.a_full = smem_u32(&a_full[0]); ra.a_empty = smem_u32(&a_empty[0]);
     ra.b_full = smem_u32(&b_full[0]); ra.b_empty = smem_u32(&b_empty[0]);
     ra.acc_full = smem_u32(&acc1_full[0]); ra.acc_empty = smem_u32(&acc1_empty[0]);
@@ -219,11 +238,12 @@ __global__ void __launch_bounds__(kFThreads, 1)
     const uint32_t ntb = (uint32_t)p.ntb;
     uint32_t slot = 0, tpar = 0, g = 0, gpar = 1;  // T slot and its parity; accumulator (= group) and the parity of its empty barrier
     bool ok = mbar_wait(smem_u32(&w2_full), 0u, abortp);
-    for (int t = blockIdx.x; t < m_tiles && ok; t += gridDim.x) {
+    for (int k = 0; k < my_tiles && ok; ++k) {
       if (!mbar_wait(tbf0 + slot * 8u, tpar, abortp)) { ok = false; break; }
       const uint64_t t_d = t_d0 + slot * tb16;
-      uint64_t w_d = w_d0;
-      for (int j = 0; j < chunks; ++j, w_d += wt16) {
+      const int jb = k == 0 ? j0 : 0, je = k == my_tiles - 1 ? j1 : chunks;  // this CTA's chunks of the tile
+      uint64_t w_d = w_d0 + (uint32_t)jb * wt16;
+      for (int j = jb; j < je; ++j, w_d += wt16) {
         if (!mbar_wait(a2e0 + g * 8u, gpar, abortp)) { ok = false; break; }
         tcgen05_fence_after();
         if (lane0) {
@@ -262,16 +282,16 @@ __global__ void __launch_bounds__(kFThreads, 1)
       }
     };
     ItemIter ld, st;
-    ld.init(h);
-    st.init(h);
+    ld.init(h, t0, j0, my_items);
+    st.init(h, t0, j0, my_items);
     if (lane0)
-      for (uint32_t s = 0; s < nslots && !ld.done(m_tiles); ++s, ld.next(h, chunks)) load_residual(ld, s);
+      for (uint32_t s = 0; s < nslots && !ld.done(); ++s, ld.next(h, chunks)) load_residual(ld, s);
     else
-      for (uint32_t s = 0; s < nslots && !ld.done(m_tiles); ++s) ld.next(h, chunks);
+      for (uint32_t s = 0; s < nslots && !ld.done(); ++s) ld.next(h, chunks);
     uint32_t slot = 0, spar = 0;
     int prev_slot = -1;
     bool ok = true;
-    for (; !st.done(m_tiles); st.next(h, chunks)) {
+    for (; !st.done(); st.next(h, chunks)) {
       if (!mbar_wait(ready0 + slot * 8u, spar, abortp)) { ok = false; break; }
       if (lane0) {
         uint32_t src = base + q.off_bufs + slot * q.tile8_bytes;
@@ -279,9 +299,9 @@ __global__ void __launch_bounds__(kFThreads, 1)
           tma_store_4d(&tmY, src, c, st.ti.qt * h.tw, st.ti.pt * h.th, st.ti.img);
         bulk_commit();
         bulk_wait_read<1>();  // the store before this one has read its buffer: that buffer takes the next residual
-        if (prev_slot >= 0 && !ld.done(m_tiles)) load_residual(ld, (uint32_t)prev_slot);
+        if (prev_slot >= 0 && !ld.done()) load_residual(ld, (uint32_t)prev_slot);
       }
-      if (prev_slot >= 0 && !ld.done(m_tiles)) ld.next(h, chunks);
+      if (prev_slot >= 0 && !ld.done()) ld.next(h, chunks);
       prev_slot = (int)slot;
       if (++slot == nslots) { slot = 0; spar ^= 1u; }
     }
@@ -303,7 +323,7 @@ __global__ void __launch_bounds__(kFThreads, 1)
     const uint32_t nacc = (uint32_t)q.nacc, ntb = (uint32_t)p.ntb;
     uint32_t ab = 0, apar = 0, slot = 0, tpar = 1;
     const int nchunk = q.bn >> 4;
-    for (int tl = blockIdx.x; tl < m_tiles; tl += gridDim.x) {
+    for (int k = 0; k < my_tiles; ++k) {
       bool ok = mbar_wait(accf0 + ab * 8u, apar, abortp);
       if (ok) ok = mbar_wait(tbe0 + slot * 8u, tpar, abortp);
       if (!ok) {
@@ -333,10 +353,9 @@ __global__ void __launch_bounds__(kFThreads, 1)
     const uint32_t accf = smem_u32(&acc2_full[g]), acce = smem_u32(&acc2_empty[g]);
     const uint32_t bfull0 = smem_u32(&buf_full[0]), ready0 = smem_u32(&store_ready[0]);
     const uint32_t nslots = (uint32_t)p.nslots;
-    const int my_tiles = m_tiles > (int)blockIdx.x ? (m_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
-    const int items = my_tiles * chunks;
+    const int items = my_items;
     uint32_t apar = 0, slot = (uint32_t)g % nslots, spar = ((uint32_t)g / nslots) & 1u;
-    int j = g % chunks;
+    int j = (j0 + g) % chunks;
     const int nchunk = q.bn >> 4;
     const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)g * (uint32_t)kFAcc2Cols;
     for (int i = g; i < items; i += kFE2Groups) {
@@ -631,7 +650,8 @@ int launch_conv_fused(const q8_conv_desc& d1, const q8_conv_desc& d2, const void
   cr = encode_rows(&tmY, y, p.l2.c_off + d2.K, p.l2.ldc, CU_TENSOR_MAP_L2_PROMOTION_NONE);
   if (cr != CUDA_SUCCESS) return fail(Q8_ERR_CUDA, "conv_fused: output tensor map rejected (CUresult %d)", (int)cr);
 
-  const int grid = p.l1.m_tiles < sm_count() ? p.l1.m_tiles : sm_count();
+  const long long items = (long long)p.l1.m_tiles * p.l2.n_tiles;
+  const int grid = (int)(items < sm_count() ? items : sm_count());
   if (d1.y_type == Q8_U8) {
     if (d2.y_type == Q8_U8) return launch_fused_variant<Q8_U8, Q8_U8>(tmA, tmB1, tmB2, tmRes, tmY, p, pl.dyn, grid, stream);
     return launch_fused_variant<Q8_U8, Q8_S8>(tmA, tmB1, tmB2, tmRes, tmY, p, pl.dyn, grid, stream);

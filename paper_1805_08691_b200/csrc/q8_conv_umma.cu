@@ -379,6 +379,7 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
     const int who = warp == 1 ? 0 : warp - 3;
     MmaRoleArgs ra;
     ra.base = base; ra.tmem_base = tmem_base; ra.total_tiles = total_tiles; ra.abortp = abortp;
+    ra.first_tile = (int)blockIdx.x; ra.tile_step = (int)gridDim.x;
     ra.a_full = smem_u32(&a_full[0]); ra.a_empty = smem_u32(&a_empty[0]);
     ra.b_full = smem_u32(&b_full[0]); ra.b_empty = smem_u32(&b_empty[0]);
     ra.acc_full = smem_u32(&acc_full[0]); ra.acc_empty = smem_u32(&acc_empty[0]);

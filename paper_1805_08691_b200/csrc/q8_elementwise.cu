@@ -569,6 +569,126 @@ void launch_pool16_window(const void* x, int N, int H, int W, int cg, int st_h, 
       static_cast<const uint4*>(x), H, W, cg, st_h, st_w, pad_h, pad_w, P, Q, inv, total, static_cast<uint4*>(y));
 }
 
+// 3x3 windows with stride 1 or 2, 16 channels per thread, as vertical strips: a thread owns one output column and
+// kRows consecutive output rows and slides down the image, reducing each input row of its three columns once
+// (three 16-byte loads) and keeping the last rows' partial results in registers.  The one-thread-per-output form
+// above issues nine loads per output and is bound by the load/store unit (measured 29 % of the copy bandwidth for
+// stride 1, 50 % for stride 2); here an output costs three (stride 1) or six (stride 2) loads.
+// Average: bytes are summed as 16-bit lanes (signed input biased by +128 per in-image cell), the sum becomes a
+// float exactly through the 2^23 trick, then clamp(Round(float(sum) * inv)) as defined: one fp32 multiply, round
+// half even by adding 1.5 * 2^23 (|v| <= 255, and a full-window divisor keeps the result inside the 8-bit range).
+struct PoolRow {
+  unsigned int a[4], b[4];  // max: a = byte-wise maximum.  average: a = lanes of bytes 0,2; b = lanes of bytes 1,3
+  int cells;                // average, signed input: in-image cells that went into the sums
+};
+
+template <bool kSigned, bool kAvg>
+__device__ __forceinline__ PoolRow pool_row3(const uint4* __restrict__ img, int h, int H, int W, int cg, int w0) {
+  PoolRow r;
+  const unsigned int init = (!kAvg && kSigned) ? 0x80808080u : 0u;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) { r.a[j] = init; r.b[j] = 0u; }
+  r.cells = 0;
+  if (h < 0 || h >= H) return r;
+  const uint4* row = img + (size_t)h * W * cg;
+  uint4 v[3];
+  bool ok[3];
+#pragma unroll
+  for (int s = 0; s < 3; ++s) {
+    ok[s] = w0 + s >= 0 && w0 + s < W;
+    v[s] = ok[s] ? __ldg(row + (size_t)(w0 + s) * cg) : make_uint4(init, init, init, init);
+  }
+#pragma unroll
+  for (int s = 0; s < 3; ++s) {
+    const unsigned int word[4] = {v[s].x, v[s].y, v[s].z, v[s].w};
+    if (!kAvg) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) r.a[j] = kSigned ? __vmaxs4(r.a[j], word[j]) : __vmaxu4(r.a[j], word[j]);
+    } else if (ok[s]) {
+      const unsigned int flip = kSigned ? 0x80808080u : 0u;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const unsigned int wj = word[j] ^ flip;
+        r.a[j] += wj & 0x00ff00ffu;
+        r.b[j] += __byte_perm(wj, 0u, 0x4341u);  // bytes 1 and 3 as 16-bit lanes
+      }
+      ++r.cells;
+    }
+  }
+  return r;
+}
+
+template <bool kSigned, bool kAvg>
+__device__ __forceinline__ uint4 pool_combine3(const PoolRow& r0, const PoolRow& r1, const PoolRow& r2, float inv) {
+  unsigned int out[4];
+  if (!kAvg) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      out[j] = kSigned ? __vmaxs4(__vmaxs4(r0.a[j], r1.a[j]), r2.a[j]) : __vmaxu4(__vmaxu4(r0.a[j], r1.a[j]), r2.a[j]);
+  } else {
+    // float(lane) = bits(0x4B00LLLL) - 2^23 exactly; the +128 per cell of signed input comes off in the same subtraction
+    const float off = 8388608.0f + (kSigned ? 128.0f * (float)(r0.cells + r1.cells + r2.cells) : 0.0f);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const unsigned int e = r0.a[j] + r1.a[j] + r2.a[j], o = r0.b[j] + r1.b[j] + r2.b[j];
+      const float f0 = __fsub_rn(__uint_as_float(__byte_perm(e, 0x4B000000u, 0x7610u)), off);
+      const float f1 = __fsub_rn(__uint_as_float(__byte_perm(o, 0x4B000000u, 0x7610u)), off);
+      const float f2 = __fsub_rn(__uint_as_float(__byte_perm(e, 0x4B000000u, 0x7632u)), off);
+      const float f3 = __fsub_rn(__uint_as_float(__byte_perm(o, 0x4B000000u, 0x7632u)), off);
+      // Round half even: adding 1.5 * 2^23 leaves the rounded integer in the low mantissa bits (two's complement)
+      const unsigned int z0 = __float_as_uint(__fadd_rn(__fmul_rn(f0, inv), 12582912.0f));
+      const unsigned int z1 = __float_as_uint(__fadd_rn(__fmul_rn(f1, inv), 12582912.0f));
+      const unsigned int z2 = __float_as_uint(__fadd_rn(__fmul_rn(f2, inv), 12582912.0f));
+      const unsigned int z3 = __float_as_uint(__fadd_rn(__fmul_rn(f3, inv), 12582912.0f));
+      out[j] = __byte_perm(__byte_perm(z0, z1, 0x0040u), __byte_perm(z2, z3, 0x0040u), 0x5410u);
+    }
+  }
+  return make_uint4(out[0], out[1], out[2], out[3]);
+}
+
+template <bool kSigned, bool kAvg, int kStride, int kRows>
+__global__ void __launch_bounds__(256) pool3_strip_kernel(const uint4* __restrict__ x, int H, int W, int cg, int pad_h,
+                                                          int pad_w, int P, int Q, int strips, float inv, unsigned int total,
+                                                          uint4* __restrict__ y) {
+  const unsigned int nthreads = gridDim.x * blockDim.x;
+  for (unsigned int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += nthreads) {
+    const unsigned int c = i % (unsigned)cg;
+    unsigned int t = i / (unsigned)cg;
+    const int q = (int)(t % (unsigned)Q);
+    t /= (unsigned)Q;
+    const int strip = (int)(t % (unsigned)strips);
+    const unsigned int n = t / (unsigned)strips;
+    const int p0 = strip * kRows, p1 = min(P, p0 + kRows);
+    const int w0 = q * kStride - pad_w;
+    const uint4* img = x + (size_t)n * H * W * cg + c;
+    uint4* out = y + ((size_t)n * P * Q + (size_t)p0 * Q + q) * cg + c;
+    int h = p0 * kStride - pad_h;
+    PoolRow r0 = pool_row3<kSigned, kAvg>(img, h, H, W, cg, w0);
+    PoolRow r1 = pool_row3<kSigned, kAvg>(img, h + 1, H, W, cg, w0);
+    for (int p = p0; p < p1; ++p, h += kStride, out += (size_t)Q * cg) {
+      const PoolRow r2 = pool_row3<kSigned, kAvg>(img, h + 2, H, W, cg, w0);
+      *out = pool_combine3<kSigned, kAvg>(r0, r1, r2, inv);
+      if (kStride == 1) {
+        r0 = r1;
+        r1 = r2;
+      } else {
+        r0 = r2;
+        if (p + 1 < p1) r1 = pool_row3<kSigned, kAvg>(img, h + 3, H, W, cg, w0);
+      }
+    }
+  }
+}
+
+template <bool kSigned, bool kAvg, int kStride>
+void launch_pool3_strip(const void* x, int N, int H, int W, int cg, int pad_h, int pad_w, int P, int Q, float inv, void* y,
+                        cudaStream_t s) {
+  constexpr int kRows = 8;
+  const int strips = (P + kRows - 1) / kRows;
+  const unsigned int total = (unsigned int)((size_t)N * strips * Q * cg);
+  pool3_strip_kernel<kSigned, kAvg, kStride, kRows><<<grid_for(total, 256, 8), 256, 0, s>>>(
+      static_cast<const uint4*>(x), H, W, cg, pad_h, pad_w, P, Q, strips, inv, total, static_cast<uint4*>(y));
+}
+
 // Global average pooling (the window is the whole image, one output pixel): a block takes one image and 64
 // channels; thread (g, c) sums every 16th pixel of channel word c, the 16 partial sums meet in shared memory.
 template <bool kSigned>
@@ -638,6 +758,17 @@ int launch_pool(const void* x, int t, int N, int H, int W, int C, int kh, int kw
   if (C % 16 == 0 && aligned16(x) && aligned16(y) && kh == kw && (kh == 3 || kh == 2) &&
       (size_t)N * P * Q * (C / 16) < (1ull << 31) && (size_t)N * H * W * (C / 16) < (1ull << 31)) {
     const int cg = C / 16;
+    // strips of eight output rows once that still gives every SM several hundred threads
+    if (kh == 3 && st_h == st_w && (st_h == 1 || st_h == 2) && (size_t)N * ((P + 7) / 8) * Q * cg >= (size_t)sm_count() * 512) {
+      if (st_h == 1) {
+        if (t == Q8_S8) launch_pool3_strip<true, kAvg, 1>(x, N, H, W, cg, pad_h, pad_w, P, Q, inv, y, s);
+        else launch_pool3_strip<false, kAvg, 1>(x, N, H, W, cg, pad_h, pad_w, P, Q, inv, y, s);
+      } else {
+        if (t == Q8_S8) launch_pool3_strip<true, kAvg, 2>(x, N, H, W, cg, pad_h, pad_w, P, Q, inv, y, s);
+        else launch_pool3_strip<false, kAvg, 2>(x, N, H, W, cg, pad_h, pad_w, P, Q, inv, y, s);
+      }
+      return check_launch("pool3_strip_kernel");
+    }
     if (kh == 3) {
       if (t == Q8_S8) launch_pool16_window<true, kAvg, 3, 3>(x, N, H, W, cg, st_h, st_w, pad_h, pad_w, P, Q, inv, y, s);
       else launch_pool16_window<false, kAvg, 3, 3>(x, N, H, W, cg, st_h, st_w, pad_h, pad_w, P, Q, inv, y, s);

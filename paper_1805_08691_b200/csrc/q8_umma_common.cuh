@@ -649,7 +649,7 @@ struct MmaRoleArgs {
   uint32_t base, tmem_base;
   uint32_t a_full, a_empty, b_full, b_empty, acc_full, acc_empty, bres_full, turn;
   const uint32_t* tap_shift16;
-  int total_tiles;
+  int first_tile, tile_step, total_tiles;  // this CTA's work items: first_tile, first_tile + tile_step, ... below total_tiles
   volatile int* abortp;
 };
 
@@ -665,7 +665,7 @@ __device__ __forceinline__ bool mma_role(const UmmaParams& p, const MmaRoleArgs&
   TileIterT<false> ti;
   const int L = p.mma_lanes;
   const bool lane0 = (threadIdx.x & 31u) == 0;  // the whole warp walks the schedule, this lane issues
-  ti.init(p, blockIdx.x + who * (int)gridDim.x, L * (int)gridDim.x);
+  ti.init(p, r.first_tile + who * r.tile_step, L * r.tile_step);
   const uint32_t nstages = (uint32_t)p.stages, nbst = (uint32_t)p.b_stages;
   // descriptors: high word constant; low word = start address >> 4 (shared memory ends below 256 KiB,
   // the 14-bit field never wraps) plus the leading-byte-offset field (bits 16-29), unused for swizzled

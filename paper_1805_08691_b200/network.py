@@ -40,13 +40,15 @@ from . import pipeline
 
 class QuantNetwork:
     def __init__(self, layers, folded: Dict[str, tuple], maxima: Dict[str, float], in_shape, device="cuda",
-                 per_channel=False, streams=1):
+                 per_channel=False, streams=1, fuse=True):
         """folded[name] = (w KRSC, b K) FP32 device tensors; maxima: calibrated max-abs of "input", every layer
         output and "<name>:pre" of residual convolutions; in_shape = (N, H, W, 3); per_channel: one weight
         factor per output channel instead of one per tensor; streams: independent branches (the
         branches of an Inception module, a projection shortcut beside its residual branch, detection heads beside
         the trunk) are enqueued on up to this many CUDA streams, so that one branch's kernels start on SMs that
-        another branch's kernel has already left."""
+        another branch's kernel has already left.  fuse: a convolution whose only reader is a 1x1 convolution runs
+        with it in one launch where the library supports the pair (q8_conv2d_then_1x1: same bytes, the tensor between
+        them is not written, so it is absent from the returned tensors)."""
         self.layers = layers
         self.maxima = maxima
         self.by_name = {L.name: L for L in layers}
@@ -112,6 +114,7 @@ class QuantNetwork:
             if name in self.in_place or (self.by_name[name].op == "concat" and root != name):
                 self.bufs[name] = self.bufs[root][..., off:off + self.shape[name][3]]
         ws_bytes = max(ws_bytes, self._merge_sibling_heads(device))
+        self._pair_layers(bool(fuse))
         self._assign_streams(max(1, int(streams)))
         # split-K scratch: one per stream, layers on different streams may run at the same time
         self.workspaces = [torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device=device) if ws_bytes else None
@@ -122,6 +125,8 @@ class QuantNetwork:
         for L in layers:
             if L.op == "conv" and L.name in self.bufs and self.bufs[L.name].shape[-1] != L.conv.K and L.name not in self.slot:
                 self.outputs[L.name] = self.bufs[L.name][..., :L.conv.K]
+        for first in self.fused_with:   # the tensor between two layers of one launch is never written
+            self.outputs.pop(first, None)
 
     # ---- host bookkeeping ---------------------------------------------------------------------------
     def _shapes(self, in_shape):
@@ -234,6 +239,28 @@ class QuantNetwork:
             ws_bytes = max(ws_bytes, q8.q8_conv2d_workspace_bytes(desc))
         return ws_bytes
 
+    def _pair_layers(self, fuse):
+        """fused_with[first] = second for every convolution pair that runs as one launch: `second` is a 1x1
+        convolution, the only reader of `first`, neither writes a concat slice or a padded tensor, `second` does not
+        take `first` as its residual, and the library accepts the pair."""
+        self.fused_with, self.fused_second = {}, set()
+        if not fuse:
+            return
+        for L in self.layers:
+            if L.op != "conv" or L.name in self.skip or L.name in self.merged or L.name in self.in_place or L.f32_out:
+                continue
+            readers = self.uses.get(L.name, [])
+            if len(readers) != 1 or L.residual is not None or self.shape[L.name][3] != L.conv.K:
+                continue
+            R = readers[0]
+            if (R.op != "conv" or R.src != [L.name] or R.residual == L.name or R.name in self.skip or R.name in self.merged
+                    or R.name in self.in_place or R.f32_out or self.shape[R.name][3] != R.conv.K
+                    or L.name in self.fused_second):
+                continue
+            if q8.q8_conv2d_then_1x1_supported(self.convs[L.name].desc, self.convs[R.name].desc):
+                self.fused_with[L.name] = R.name
+                self.fused_second.add(R.name)
+
     def _assign_streams(self, limit):
         """stream_of[layer]: a layer continues on the stream of its first input if it is that tensor's first
         reader, otherwise it opens the least recently used other stream.  deps[layer]: the tensors it must wait
@@ -316,6 +343,12 @@ class QuantNetwork:
             res = b[L.residual] if L.residual is not None else None
             if L.name in self.skip:
                 return  # computed by the merged launch of its first sibling
+            if L.name in self.fused_with:
+                return  # runs together with its reader, below
+            if L.name in self.fused_second:
+                first = self.by_name[L.src[0]]
+                pipeline.fused_pair(self.convs[first.name], qc, b[first.src[0]], res, b[L.name])
+                return
             y = b[self.slot[L.name][0]] if L.name in self.in_place else b[L.name]
             if L.name in self.merged:
                 y = b[L.name + ":merged"]

@@ -88,6 +88,12 @@ def prepare_conv(w, b, in_shape, q_x, q_y, x_type=q8.Q8_U8, y_type=q8.Q8_U8, rel
     return QuantConv(desc, w_q, b_q, scale, q_w, q_x, q_y, res_scale)
 
 
+def fused_pair(first: QuantConv, second: QuantConv, x_q, residual=None, out=None):
+    """`first` followed by the 1x1 layer `second` in one launch; the tensor between them is never written."""
+    return q8.q8_conv2d_then_1x1(first.desc, second.desc, x_q, first.w_q, first.b_q, first.scale, second.w_q, second.b_q,
+                                 second.scale, residual, second.res_scale, out)
+
+
 class Bottleneck:
     """ResNet bottleneck (1x1 -> 3x3 -> 1x1 + identity residual, ReLU fused everywhere) in int8.
 
@@ -96,7 +102,9 @@ class Bottleneck:
     q_y = max(max|c|, max|x|) / 255.
     """
 
-    def __init__(self, folded, maxima, in_shape, algo=q8.Q8_ALGO_AUTO):
+    def __init__(self, folded, maxima, in_shape, algo=q8.Q8_ALGO_AUTO, fuse=True):
+        """fuse: run the 3x3 and the expanding 1x1 as one launch (q8_conv2d_then_1x1) when the library supports the
+        pair; the result is the same bit for bit, the 3x3 output is then never written (self.yb stays unused)."""
         N, H, W, C = in_shape
         (wa, ba), (wb, bb), (wc, bc) = folded
         mid = wa.shape[0]
@@ -109,9 +117,12 @@ class Bottleneck:
         self.c = prepare_conv(wc, bc, (N, H, W, mid), self.q_b, self.q_y, relu=True, q_res=self.q_x, algo=algo)
         self.ya = torch.empty((N, H, W, mid), dtype=torch.uint8, device=wa.device)
         self.yb = torch.empty((N, H, W, mid), dtype=torch.uint8, device=wa.device)
+        self.fused = bool(fuse) and algo == q8.Q8_ALGO_AUTO and q8.q8_conv2d_then_1x1_supported(self.b.desc, self.c.desc)
 
     def __call__(self, x_q, out=None):
         self.a(x_q, out=self.ya)
+        if self.fused:
+            return fused_pair(self.b, self.c, self.ya, residual=x_q, out=out)
         self.b(self.ya, out=self.yb)
         return self.c(self.yb, residual=x_q, out=out)
 

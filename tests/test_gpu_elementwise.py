@@ -116,6 +116,20 @@ def test_pools_bit_exact(q8, k, st, pad, ceil, C):
     assert np.array_equal(got, o.pool(xs, "avg", (k, k), (st, st), (pad, pad), ceil))
 
 
+@pytest.mark.parametrize("st,pad,ceil", [(1, 1, False), (2, 1, False), (2, 0, True), (1, 0, False), (2, 2, False)])
+def test_3x3_pools_in_row_strips_bit_exact(q8, st, pad, ceil):
+    """Tensors large enough for the strip kernel (eight output rows per thread): ragged last strip, both strides,
+    padding 0 to 2, extreme codes in the corners, u8 and s8."""
+    g = np.random.default_rng(31 * st + pad)
+    x = g.integers(0, 256, (6, 45, 39, 96), dtype=np.uint8)
+    x[:, :2, :2, :] = 255
+    x[:, -2:, -2:, :] = 0
+    for arr in (x, x.view(np.int8)):
+        for kind, fn in (("max", q8.q8_maxpool2d), ("avg", q8.q8_avgpool2d)):
+            got = fn(_cuda(arr), (3, 3), (st, st), (pad, pad), ceil).cpu().numpy()
+            assert np.array_equal(got, o.pool(arr, kind, (3, 3), (st, st), (pad, pad), ceil)), (kind, arr.dtype)
+
+
 @pytest.mark.parametrize("value,dt", [(255, np.uint8), (-128, np.int8), (127, np.int8)])
 def test_avgpool_extreme_codes_largest_window(q8, value, dt):
     """A 16 x 16 window of one extreme code: the packed 16-bit lane sums may not carry into their neighbours."""

@@ -19,7 +19,27 @@ def _cuda(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
-def _run_both(q8, layers, hw, batch, calib_batches, seed, check_layers=None, per_channel=False, streams=1):
+def _compare(layers, got, want, net, info, rows=None, check_layers=None):
+    """Every tensor the network exposes against the oracle's, bit for bit (rows: the images of the batch the oracle
+    ran).  A tensor is absent only if its layer runs in one launch with its reader."""
+    for L in layers:
+        if check_layers is not None and L.name not in check_layers:
+            continue
+        if L.name not in got:
+            assert L.name in net.fused_with, L.name
+            continue
+        a, e = got[L.name].cpu().numpy(), want[L.name]
+        if rows is not None:
+            a = a[rows]
+        if a.dtype == np.float32:
+            a, e = a.view(np.uint32), e.view(np.uint32)
+        assert a.shape == e.shape and np.array_equal(a, e), L.name
+        assert net.info[L.name][1] == info[L.name][1], L.name
+
+
+def _run_both(q8, layers, hw, batch, calib_batches, seed, check_layers=None, per_channel=False, streams=1, fuse=False,
+              calib_batch=None, rows=None):
+    """rows: run the library on the whole batch but the oracle only on these images of it (images are independent)."""
     from paper_1805_08691_b200 import network, pipeline
     # fold BN on both sides, must agree bit for bit
     folded_o, folded_g = {}, {}
@@ -41,7 +61,7 @@ def _run_both(q8, layers, hw, batch, calib_batches, seed, check_layers=None, per
     cal = None
     max_o = {}
     for i in range(calib_batches):
-        acts = nets.fp32_forward(layers, nets.images(seed + 10 + i, batch, hw), folded_o, device="cuda")
+        acts = nets.fp32_forward(layers, nets.images(seed + 10 + i, calib_batch or batch, hw), folded_o, device="cuda")
         if cal is None:
             names = sorted(acts)
             cal = pipeline.Calibrator(names)
@@ -53,19 +73,13 @@ def _run_both(q8, layers, hw, batch, calib_batches, seed, check_layers=None, per
     # prepare and run
     x = nets.images(seed + 1, batch, hw)
     prep, info = oracle_net.network_prepare(layers, folded_o, max_o, per_channel)
-    want = oracle_net.network_forward(layers, prep, info, x, threads=batch)
-    net = network.QuantNetwork(layers, folded_g, max_g, x.shape, per_channel=per_channel, streams=streams)
+    xo = x if rows is None else np.ascontiguousarray(x[rows])
+    want = oracle_net.network_forward(layers, prep, info, xo, threads=min(len(xo), o.hw_threads()))
+    net = network.QuantNetwork(layers, folded_g, max_g, x.shape, per_channel=per_channel, streams=streams, fuse=fuse)
     got = net.forward(_cuda(x))
     q8.q8_read_status()
-    for L in layers:
-        if check_layers is not None and L.name not in check_layers:
-            continue
-        a, e = got[L.name].cpu().numpy(), want[L.name]
-        if a.dtype == np.float32:
-            a, e = a.view(np.uint32), e.view(np.uint32)
-        assert a.shape == e.shape and np.array_equal(a, e), L.name
-        assert net.info[L.name][1] == info[L.name][1], L.name
-    ref = nets.fp32_forward(layers, x, folded_o, device="cuda")
+    _compare(layers, got, want, net, info, rows, check_layers)
+    ref = nets.fp32_forward(layers, xo, folded_o, device="cuda")
     return got, want, ref, net
 
 
@@ -73,6 +87,30 @@ def test_bottleneck_stack_every_layer(q8):
     layers = nets.bottleneck_stack(C=64, blocks=2)
     _run_both(q8, layers, hw=32, batch=3, calib_batches=2, seed=3100)
     _run_both(q8, layers, hw=32, batch=3, calib_batches=2, seed=3100, streams=2)
+    got, want, ref, net = _run_both(q8, layers, hw=32, batch=3, calib_batches=2, seed=3100, streams=2, fuse=True)
+    assert len(net.fused_with) == 2     # the 3x3 of each block runs in one launch with the 1x1 after it
+
+
+# ---- the benchmarked launch configurations: whole batch on the GPU (pair mode, tile widths and reduction splits
+# depend on the batch), every layer of three sampled images against the oracle run on just those images
+FULL = [("resnet50", 224, 64, 3000, False), ("resnet50", 224, 1, 3000, False), ("resnet50_sparsity_removed", 224, 64, 3000, False),
+        ("resnet50", 224, 64, 3000, True), ("inception_v3", 299, 64, 4000, True), ("ssd300", 300, 32, 5000, True)]
+
+
+@pytest.mark.parametrize("name,hw,batch,seed,fuse", FULL, ids=[f"{n}_b{b}{'_fused' if f else ''}" for n, _, b, _, f in FULL])
+def test_full_batch_sampled_images_bit_exact(q8, name, hw, batch, seed, fuse):
+    """Configs 3-5 at the batch sizes bench.py times (64 / 64 / 32, ResNet-50 also at 1), four streams, with and
+    without layer pairs in one launch: every tensor of the first, middle and last image equals the oracle's."""
+    if name == "resnet50_sparsity_removed":
+        from paper_1805_08691_b200 import graph
+        layers = graph.remove_sparsity(nets.resnet50())
+    else:
+        layers = getattr(nets, name)()
+    rows = sorted({0, batch // 2, batch - 1})
+    got, want, ref, net = _run_both(q8, layers, hw=hw, batch=batch, calib_batches=1, seed=seed, streams=4, fuse=fuse,
+                                    calib_batch=2, rows=rows)
+    if fuse and name == "resnet50":
+        assert len(net.fused_with) >= 7
 
 
 def test_per_channel_weight_factors_every_layer(q8):
