@@ -283,6 +283,25 @@ def network_numbers(dev, name, reps=20):
     maxima = cal.maxima()
     del acts
     out = {"macs_per_image": nets.macs(layers, hw), "paper_xeon": cfg["paper_xeon"]}
+    # int8 against FP32 on two seeded images (the stand-in for the paper's accuracy table, which needs trained
+    # weights and data sets): relative L2 error of the dequantized outputs (logits / all detection heads) for one
+    # weight factor per tensor (the paper) or per output channel, and for the factor of a fused residual sum from
+    # the "+" rule on its summands or calibrated on the sum itself
+    xt = nets.images(cfg["seed"] + 2, 2, hw)
+    ref = nets.fp32_forward(layers, xt, folded_np, device=dev)
+    heads = [L.name for L in layers if L.f32_out]
+    rel = {}
+    for per_channel in (False, True):
+        for policy in ("max", "post_sum"):
+            net = network.QuantNetwork(layers, folded, maxima, (2, hw, hw, 3), device=dev, per_channel=per_channel,
+                                       sum_policy=policy)
+            got = net.forward(cuda(xt))
+            num = sum(float(((got[h].cpu().numpy().astype(np.float64) - ref[h]) ** 2).sum()) for h in heads)
+            den = sum(float((ref[h].astype(np.float64) ** 2).sum()) for h in heads)
+            rel[("per_channel" if per_channel else "per_tensor") + "/" + policy] = (num / den) ** 0.5
+            del net, got
+    out["rel_l2_int8_vs_fp32"] = rel
+    del ref
     variants = [("batch%d" % cfg["batch"], cfg["batch"], layers), ("batch1", 1, layers)]
     if name == "resnet50":
         # the paper's "remove sparsity" graph rewrite: same FP32 function, 3 % fewer MACs (throughput is still

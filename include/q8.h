@@ -224,6 +224,15 @@ int q8_conv2d_then_1x1(const q8_conv_desc* d1, const q8_conv_desc* d2, const voi
  * Errors: Q8_ERR_INVALID_ARG, Q8_ERR_CUDA. */
 int q8_int8_mma_rate(int bn, int chains, int instructions, int ctas, unsigned long long* cycles_dev, void* stream);
 
+/* Test aid (the paper has no counterpart): every wait inside the tensor-core kernels is bounded; when one runs
+ * out, the kernel sets a bit of the device status word, all roles of the CTA drain and the kernel returns, and the
+ * next q8_read_status reports Q8_ERR_TIMEOUT and clears the word.  This call makes that happen without any fault:
+ * it launches one small CTA whose first warp waits `limit_us` microseconds (1 .. 1 000 000) on a barrier nothing
+ * signals, and whose second warp waits with the library's normal limit (2 s) and must leave early because the first
+ * gave up.  Asynchronous on `stream`; afterwards q8_read_status(stream) returns Q8_ERR_TIMEOUT (site mask 0x5)
+ * once, then Q8_OK.  Errors: Q8_ERR_INVALID_ARG, Q8_ERR_CUDA. */
+int q8_selftest_bounded_wait(unsigned int limit_us, void* stream);
+
 /* q8_conv2d for callers that cannot allocate device memory (the paper has no counterpart; this is a
  * property of the library, not of the method).  Meant for hosts where every byte of device memory was
  * handed out before this library is called, or where cudaMalloc is off limits because it stalls the

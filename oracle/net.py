@@ -103,10 +103,14 @@ def _concat_groups(layers):
     return root, shared, leaves
 
 
-def network_prepare(layers, folded, maxima, per_channel=False):
+def network_prepare(layers, folded, maxima, per_channel=False, sum_policy="max"):
     """Returns {layer name: dict} with the quantized parameters and the (type, factor) of every tensor.
     per_channel: one weight factor per output channel, max|w[k]| / 127 (the paper takes one per tensor); bias
-    and requantisation multiplier of channel k then use q_w[k]."""
+    and requantisation multiplier of channel k then use q_w[k].
+    sum_policy: factor of a fused residual sum.  "max": the "+" rule of Eq. arithmetics on the two summands,
+    max(max|conv|, max|residual|) / 255.  "post_sum": the calibration rule applied to the tensor the layer
+    actually emits, max|ReLU(conv + residual)| / 255 (never larger than twice the first, often smaller)."""
+    assert sum_policy in ("max", "post_sum")
     root, shared, leaves = _concat_groups(layers)
     by_name = {L.name: L for L in layers}
     own = {}
@@ -121,6 +125,8 @@ def network_prepare(layers, folded, maxima, per_channel=False):
                 own[name] = final_factor(L.src[0])
             elif L.op == "concat":
                 own[name] = group_factor(root[name])
+            elif L.residual is not None and sum_policy == "post_sum":
+                own[name] = o.factor(maxima[name], 8)
             elif L.residual is not None:
                 own[name] = o.factor(max(maxima[name + ":pre"], maxima[L.residual]), 8)
             else:

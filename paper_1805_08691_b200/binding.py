@@ -21,7 +21,7 @@ TORCH_DTYPES = {Q8_U8: torch.uint8, Q8_S8: torch.int8, Q8_S32: torch.int32, Q8_F
 EXPORTS = ["q8_version", "q8_last_error", "q8_read_status", "q8_calibrate_maxabs", "q8_factor", "q8_requant_scale",
            "q8_bias_factor", "q8_quantize", "q8_quantize_pad_channels", "q8_dequantize", "q8_fold_bn",
            "q8_conv2d_workspace_bytes", "q8_conv2d_query_algo", "q8_conv2d", "q8_static_workspace_bytes",
-           "q8_conv2d_static_workspace", "q8_conv2d_then_1x1_supported", "q8_conv2d_then_1x1", "q8_int8_mma_rate", "q8_concat", "q8_concat_branch", "q8_calibrate_maxabs_rows", "q8_quantize_rows", "q8_quantize_pad_image", "q8_pool_out_extent",
+           "q8_conv2d_static_workspace", "q8_conv2d_then_1x1_supported", "q8_conv2d_then_1x1", "q8_int8_mma_rate", "q8_selftest_bounded_wait", "q8_concat", "q8_concat_branch", "q8_calibrate_maxabs_rows", "q8_quantize_rows", "q8_quantize_pad_image", "q8_pool_out_extent",
            "q8_maxpool2d", "q8_avgpool2d"]
 
 
@@ -66,6 +66,7 @@ lib.q8_conv2d_workspace_bytes.argtypes = [C.POINTER(q8_conv_desc), C.POINTER(_sz
 lib.q8_conv2d_query_algo.argtypes = [C.POINTER(q8_conv_desc), _ip]
 lib.q8_conv2d.argtypes = [C.POINTER(q8_conv_desc), _vp, _vp, _vp, _vp, _vp, _f, _vp, _vp, _sz, _vp]
 lib.q8_static_workspace_bytes.argtypes = []
+lib.q8_selftest_bounded_wait.argtypes = [C.c_uint, _vp]
 lib.q8_int8_mma_rate.argtypes = [_i, _i, _i, _i, _vp, _vp]
 lib.q8_conv2d_then_1x1_supported.argtypes = [C.POINTER(q8_conv_desc), C.POINTER(q8_conv_desc), _ip]
 lib.q8_conv2d_then_1x1.argtypes = [C.POINTER(q8_conv_desc), C.POINTER(q8_conv_desc), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _f, _vp, _vp]
@@ -238,6 +239,10 @@ def q8_int8_mma_rate(bn, chains, instructions, ctas, cycles):
     """cycles: int64 CUDA tensor of `ctas` entries, filled with the SM cycles each CTA needed."""
     _check(lib.q8_int8_mma_rate(bn, chains, instructions, ctas, _dev(cycles, "cycles"), _stream()))
     return cycles
+
+
+def q8_selftest_bounded_wait(limit_us):
+    _check(lib.q8_selftest_bounded_wait(int(limit_us), _stream()))
 
 
 def q8_static_workspace_bytes():

@@ -209,17 +209,42 @@ __global__ void __launch_bounds__(kThreads) quantize_pad_image_kernel(const floa
   }
 }
 
-// Images: 3 channels -> 16.  Four pixels per thread: three 16-byte loads (12 floats), four 16-byte stores.
-__global__ void __launch_bounds__(kThreads) quantize_pad3_kernel(const float4* __restrict__ x, size_t quads, float q, int lo,
-                                                                 int hi, uint4* __restrict__ z) {
-  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < quads; i += nthreads) {
-    const float4 a = __ldcs(x + 3 * i), b = __ldcs(x + 3 * i + 1), c = __ldcs(x + 3 * i + 2);
-    uint4* out = z + 4 * i;
-    __stcs(out, make_uint4(pack4(quant1(a.x, q, lo, hi), quant1(a.y, q, lo, hi), quant1(a.z, q, lo, hi), 0), 0u, 0u, 0u));
-    __stcs(out + 1, make_uint4(pack4(quant1(a.w, q, lo, hi), quant1(b.x, q, lo, hi), quant1(b.y, q, lo, hi), 0), 0u, 0u, 0u));
-    __stcs(out + 2, make_uint4(pack4(quant1(b.z, q, lo, hi), quant1(b.w, q, lo, hi), quant1(c.x, q, lo, hi), 0), 0u, 0u, 0u));
-    __stcs(out + 3, make_uint4(pack4(quant1(c.y, q, lo, hi), quant1(c.z, q, lo, hi), quant1(c.w, q, lo, hi), 0), 0u, 0u, 0u));
+// Images: 3 channels -> 16, rows of W pixels padded to W_pad output pixels.  A warp takes 128 output pixels of one
+// row: it reads their 384 floats with fully coalesced 4-byte loads into shared memory, then every lane quantizes
+// four pixels (three conflict-free shared-memory reads each) and the warp writes 512 contiguous bytes per store.
+// (One thread per pixel reads 12-byte and writes 16-byte pieces 48 / 64 bytes apart: a third / a quarter of every
+// sector per instruction, measured 61 % of the copy bandwidth.)
+__global__ void __launch_bounds__(kThreads) quantize_pad3_rows_kernel(const float* __restrict__ x, size_t rows, size_t W,
+                                                                      size_t W_pad, float q, int lo, int hi,
+                                                                      uint4* __restrict__ z) {
+  __shared__ float stage[kThreads / 32][384];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float* st = stage[warp];
+  const size_t chunks_per_row = (W_pad + 127) / 128, chunks = rows * chunks_per_row;
+  const size_t nwarps = (size_t)gridDim.x * (kThreads / 32);
+  for (size_t ch = (size_t)blockIdx.x * (kThreads / 32) + warp; ch < chunks; ch += nwarps) {
+    const size_t r = ch / chunks_per_row, w0 = (ch - r * chunks_per_row) * 128;
+    const size_t in_px = w0 < W ? (W - w0 < 128 ? W - w0 : 128) : 0;      // real pixels of this chunk
+    const size_t out_px = W_pad - w0 < 128 ? W_pad - w0 : 128;
+    const float* src = x + (r * W + w0) * 3;
+    const int nf = (int)in_px * 3;
+#pragma unroll
+    for (int k = 0; k < 12; ++k) {
+      const int f = k * 32 + lane;
+      if (f < nf) st[f] = __ldcs(src + f);
+    }
+    __syncwarp();
+    uint4* out = z + r * W_pad + w0;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int px = k * 32 + lane;
+      if ((size_t)px < out_px) {
+        unsigned int w = 0u;
+        if ((size_t)px < in_px) w = pack4(quant1(st[3 * px], q, lo, hi), quant1(st[3 * px + 1], q, lo, hi), quant1(st[3 * px + 2], q, lo, hi), 0);
+        __stcs(out + px, make_uint4(w, 0u, 0u, 0u));
+      }
+    }
+    __syncwarp();
   }
 }
 
@@ -302,6 +327,45 @@ __device__ __forceinline__ unsigned int requant_word(unsigned int w, float s) {
                requant_byte<kSigned>((w >> 16) & 0xff, s), requant_byte<kSigned>(w >> 24, s));
 }
 
+// Packed fp32 pairs: two independent IEEE operations (round to nearest even) per instruction.
+__device__ __forceinline__ unsigned long long pack_f2(float a, float b) {
+  unsigned long long d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(a), "f"(b));
+  return d;
+}
+__device__ __forceinline__ void unpack_f2(unsigned long long d, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(d));
+}
+__device__ __forceinline__ unsigned long long fmul2(unsigned long long a, unsigned long long b) {
+  unsigned long long d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ unsigned long long fsub2(unsigned long long a, unsigned long long b) {
+  unsigned long long d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
+// The same re-expression for multipliers in (0, 1] (the shared factor is the largest branch factor, so this is the
+// case in practice): |z * s| <= |z| needs no clamp, the byte becomes a float exactly through the 2^23 trick (signed
+// bytes biased by 128), one fp32 multiply, and round-half-even by adding 1.5 * 2^23, whose low mantissa byte is the
+// result in two's complement.  Less than half the instructions of the general form, which bounds this kernel.
+template <bool kSigned>
+__device__ __forceinline__ unsigned int requant_word_small(unsigned int w, float s) {
+  const unsigned int u = kSigned ? (w ^ 0x80808080u) : w;
+  const float off = kSigned ? 8388736.0f : 8388608.0f;
+  const unsigned long long off2 = pack_f2(off, off), s2 = pack_f2(s, s);
+  float v0, v1, v2, v3;
+  unpack_f2(fmul2(fsub2(pack_f2(__uint_as_float(__byte_perm(u, 0x4B000000u, 0x7540u)),
+                                __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7541u))), off2), s2), v0, v1);
+  unpack_f2(fmul2(fsub2(pack_f2(__uint_as_float(__byte_perm(u, 0x4B000000u, 0x7542u)),
+                                __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7543u))), off2), s2), v2, v3);
+  const unsigned int z0 = __float_as_uint(__fadd_rn(v0, 12582912.0f)), z1 = __float_as_uint(__fadd_rn(v1, 12582912.0f));
+  const unsigned int z2 = __float_as_uint(__fadd_rn(v2, 12582912.0f)), z3 = __float_as_uint(__fadd_rn(v3, 12582912.0f));
+  return __byte_perm(__byte_perm(z0, z1, 0x0040u), __byte_perm(z2, z3, 0x0040u), 0x5410u);
+}
+
 // vec path: channels, c_total and c_off multiples of 16, pointers 16-byte aligned
 template <bool kSigned>
 __global__ void __launch_bounds__(kThreads) concat_vec_kernel(const uint4* __restrict__ x, size_t pixels, int cvec,
@@ -318,7 +382,12 @@ __global__ void __launch_bounds__(kThreads) concat_vec_kernel(const uint4* __res
 #pragma unroll 4
   for (; i < total; i += nthreads) {
     uint4 v = __ldcs(x + i);
-    if (!copy_only) {
+    if (copy_only == 2) {  // multiplier in (0, 1]
+      v.x = requant_word_small<kSigned>(v.x, s);
+      v.y = requant_word_small<kSigned>(v.y, s);
+      v.z = requant_word_small<kSigned>(v.z, s);
+      v.w = requant_word_small<kSigned>(v.w, s);
+    } else if (!copy_only) {
       v.x = requant_word<kSigned>(v.x, s);
       v.y = requant_word<kSigned>(v.y, s);
       v.z = requant_word<kSigned>(v.z, s);
@@ -341,7 +410,7 @@ __global__ void __launch_bounds__(kThreads) concat_scalar_kernel(const unsigned 
     size_t px = i / ch;
     int c = (int)(i - px * ch);
     unsigned int b = x[i];
-    y[px * ctot + coff + c] = copy_only ? (unsigned char)b : (unsigned char)requant_byte<kSigned>(b, s);
+    y[px * ctot + coff + c] = copy_only == 1 ? (unsigned char)b : (unsigned char)requant_byte<kSigned>(b, s);
   }
 }
 
@@ -572,8 +641,8 @@ void launch_pool16_window(const void* x, int N, int H, int W, int cg, int st_h, 
 // 3x3 windows with stride 1 or 2, 16 channels per thread, as vertical strips: a thread owns one output column and
 // kRows consecutive output rows and slides down the image, reducing each input row of its three columns once
 // (three 16-byte loads) and keeping the last rows' partial results in registers.  The one-thread-per-output form
-// above issues nine loads per output and is bound by the load/store unit (measured 29 % of the copy bandwidth for
-// stride 1, 50 % for stride 2); here an output costs three (stride 1) or six (stride 2) loads.
+// above issues nine loads per output (measured 29 % of the copy bandwidth for stride 1, 50 % for stride 2); here an
+// output costs two (stride 1, two columns per thread) or six (stride 2) loads.
 // Average: bytes are summed as 16-bit lanes (signed input biased by +128 per in-image cell), the sum becomes a
 // float exactly through the 2^23 trick, then clamp(Round(float(sum) * inv)) as defined: one fp32 multiply, round
 // half even by adding 1.5 * 2^23 (|v| <= 255, and a full-window divisor keeps the result inside the 8-bit range).
@@ -631,6 +700,7 @@ __device__ __forceinline__ uint4 pool_combine3(const PoolRow& r0, const PoolRow&
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const unsigned int e = r0.a[j] + r1.a[j] + r2.a[j], o = r0.b[j] + r1.b[j] + r2.b[j];
+      // (scalar on purpose: the packed f32x2 forms of these operations made this kernel slower, measured)
       const float f0 = __fsub_rn(__uint_as_float(__byte_perm(e, 0x4B000000u, 0x7610u)), off);
       const float f1 = __fsub_rn(__uint_as_float(__byte_perm(o, 0x4B000000u, 0x7610u)), off);
       const float f2 = __fsub_rn(__uint_as_float(__byte_perm(e, 0x4B000000u, 0x7632u)), off);
@@ -644,6 +714,85 @@ __device__ __forceinline__ uint4 pool_combine3(const PoolRow& r0, const PoolRow&
     }
   }
   return make_uint4(out[0], out[1], out[2], out[3]);
+}
+
+// Lanes of one input pixel (average) or the pixel itself (max); outside the image: the identity of the reduction.
+template <bool kSigned, bool kAvg>
+__device__ __forceinline__ PoolRow pool_pixel(const uint4* __restrict__ row, int w, int W, int cg, bool row_ok) {
+  PoolRow r;
+  const unsigned int init = (!kAvg && kSigned) ? 0x80808080u : 0u;
+  const bool ok = row_ok && w >= 0 && w < W;
+  const uint4 v = ok ? __ldg(row + (size_t)w * cg) : make_uint4(init, init, init, init);
+  const unsigned int word[4] = {v.x, v.y, v.z, v.w};
+  r.cells = ok ? 1 : 0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    if (!kAvg) { r.a[j] = word[j]; r.b[j] = 0u; }
+    else {
+      const unsigned int wj = ok ? (word[j] ^ (kSigned ? 0x80808080u : 0u)) : 0u;
+      r.a[j] = wj & 0x00ff00ffu;
+      r.b[j] = __byte_perm(wj, 0u, 0x4341u);
+    }
+  }
+  return r;
+}
+
+template <bool kSigned, bool kAvg>
+__device__ __forceinline__ PoolRow pool_join(const PoolRow& x, const PoolRow& y) {
+  PoolRow r;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    if (!kAvg) { r.a[j] = kSigned ? __vmaxs4(x.a[j], y.a[j]) : __vmaxu4(x.a[j], y.a[j]); r.b[j] = 0u; }
+    else { r.a[j] = x.a[j] + y.a[j]; r.b[j] = x.b[j] + y.b[j]; }
+  }
+  r.cells = x.cells + y.cells;
+  return r;
+}
+
+// Stride 1: a thread owns TWO adjacent output columns and kRows output rows: four loads per input row serve two
+// outputs (the two middle pixels are reduced once for both).
+template <bool kSigned, bool kAvg, int kRows>
+__global__ void __launch_bounds__(256) pool3_strip2_kernel(const uint4* __restrict__ x, int H, int W, int cg, int pad_h,
+                                                           int pad_w, int P, int Q, int strips, float inv, unsigned int total,
+                                                           uint4* __restrict__ y) {
+  const int Q2 = (Q + 1) >> 1;
+  const unsigned int nthreads = gridDim.x * blockDim.x;
+  for (unsigned int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += nthreads) {
+    const unsigned int c = i % (unsigned)cg;
+    unsigned int t = i / (unsigned)cg;
+    const int q = (int)(t % (unsigned)Q2) * 2;
+    t /= (unsigned)Q2;
+    const int strip = (int)(t % (unsigned)strips);
+    const unsigned int n = t / (unsigned)strips;
+    const int p0 = strip * kRows, p1 = min(P, p0 + kRows);
+    const int w0 = q - pad_w;
+    const bool two = q + 1 < Q;
+    const uint4* img = x + (size_t)n * H * W * cg + c;
+    uint4* out = y + ((size_t)n * P * Q + (size_t)p0 * Q + q) * cg + c;
+    PoolRow ra[3], rb[3];  // the last three input rows, reduced over the columns of output q and of output q + 1
+    auto load_row = [&](int h, PoolRow& oa, PoolRow& ob) {
+      const bool row_ok = h >= 0 && h < H;
+      const uint4* row = img + (size_t)(row_ok ? h : 0) * W * cg;
+      const PoolRow x0 = pool_pixel<kSigned, kAvg>(row, w0, W, cg, row_ok);
+      const PoolRow x1 = pool_pixel<kSigned, kAvg>(row, w0 + 1, W, cg, row_ok);
+      const PoolRow x2 = pool_pixel<kSigned, kAvg>(row, w0 + 2, W, cg, row_ok);
+      const PoolRow x3 = pool_pixel<kSigned, kAvg>(row, w0 + 3, W, cg, row_ok && two);
+      const PoolRow mid = pool_join<kSigned, kAvg>(x1, x2);
+      oa = pool_join<kSigned, kAvg>(x0, mid);
+      ob = pool_join<kSigned, kAvg>(mid, x3);
+    };
+    int h = p0 - pad_h;
+    load_row(h, ra[0], rb[0]);
+    load_row(h + 1, ra[1], rb[1]);
+#pragma unroll 1
+    for (int p = p0; p < p1; ++p, ++h, out += (size_t)Q * cg) {
+      load_row(h + 2, ra[2], rb[2]);
+      out[0] = pool_combine3<kSigned, kAvg>(ra[0], ra[1], ra[2], inv);
+      if (two) out[cg] = pool_combine3<kSigned, kAvg>(rb[0], rb[1], rb[2], inv);
+      ra[0] = ra[1]; ra[1] = ra[2];
+      rb[0] = rb[1]; rb[1] = rb[2];
+    }
+  }
 }
 
 template <bool kSigned, bool kAvg, int kStride, int kRows>
@@ -682,8 +831,14 @@ __global__ void __launch_bounds__(256) pool3_strip_kernel(const uint4* __restric
 template <bool kSigned, bool kAvg, int kStride>
 void launch_pool3_strip(const void* x, int N, int H, int W, int cg, int pad_h, int pad_w, int P, int Q, float inv, void* y,
                         cudaStream_t s) {
-  constexpr int kRows = 8;
+  constexpr int kRows = 4;
   const int strips = (P + kRows - 1) / kRows;
+  if (kStride == 1) {
+    const unsigned int total = (unsigned int)((size_t)N * strips * ((Q + 1) / 2) * cg);
+    pool3_strip2_kernel<kSigned, kAvg, kRows><<<grid_for(total, 256, 8), 256, 0, s>>>(
+        static_cast<const uint4*>(x), H, W, cg, pad_h, pad_w, P, Q, strips, inv, total, static_cast<uint4*>(y));
+    return;
+  }
   const unsigned int total = (unsigned int)((size_t)N * strips * Q * cg);
   pool3_strip_kernel<kSigned, kAvg, kStride, kRows><<<grid_for(total, 256, 8), 256, 0, s>>>(
       static_cast<const uint4*>(x), H, W, cg, pad_h, pad_w, P, Q, strips, inv, total, static_cast<uint4*>(y));
@@ -758,8 +913,8 @@ int launch_pool(const void* x, int t, int N, int H, int W, int C, int kh, int kw
   if (C % 16 == 0 && aligned16(x) && aligned16(y) && kh == kw && (kh == 3 || kh == 2) &&
       (size_t)N * P * Q * (C / 16) < (1ull << 31) && (size_t)N * H * W * (C / 16) < (1ull << 31)) {
     const int cg = C / 16;
-    // strips of eight output rows once that still gives every SM several hundred threads
-    if (kh == 3 && st_h == st_w && (st_h == 1 || st_h == 2) && (size_t)N * ((P + 7) / 8) * Q * cg >= (size_t)sm_count() * 512) {
+    // strips of four output rows once that still gives every SM a few warps
+    if (kh == 3 && st_h == st_w && (st_h == 1 || st_h == 2) && (size_t)N * ((P + 3) / 4) * Q * cg >= (size_t)sm_count() * 256) {
       if (st_h == 1) {
         if (t == Q8_S8) launch_pool3_strip<true, kAvg, 1>(x, N, H, W, cg, pad_h, pad_w, P, Q, inv, y, s);
         else launch_pool3_strip<false, kAvg, 1>(x, N, H, W, cg, pad_h, pad_w, P, Q, inv, y, s);
@@ -910,13 +1065,10 @@ int q8_quantize_pad_channels(const float* x, size_t pixels, int C, int C_pad, fl
   if (out_type != Q8_U8 && out_type != Q8_S8) return fail(Q8_ERR_INVALID_ARG, "q8_quantize_pad_channels: bad out_type");
   if (pixels == 0) return Q8_OK;
   const int lo = out_type == Q8_U8 ? 0 : -128, hi = out_type == Q8_U8 ? 255 : 127;
-  if (C == 3 && C_pad == 16 && aligned16(z) && aligned16(x)) {
-    const size_t quads = pixels / 4;
-    if (quads) quantize_pad3_kernel<<<grid_for(quads, kThreads, 8), kThreads, 0, as_stream(stream)>>>(
-        reinterpret_cast<const float4*>(x), quads, q, lo, hi, static_cast<uint4*>(z));
-    if (quads * 4 < pixels)  // the last one to three pixels
-      quantize_pad16_kernel<<<1, 32, 0, as_stream(stream)>>>(x + quads * 12, pixels - quads * 4, 3, 1, q, lo, hi, static_cast<uint4*>(z) + quads * 4);
-    return check_launch("quantize_pad3_kernel");
+  if (C == 3 && C_pad == 16 && aligned16(z)) {
+    quantize_pad3_rows_kernel<<<grid_for((pixels + 127) / 128, kThreads / 32, 4), kThreads, 0, as_stream(stream)>>>(
+        x, 1, pixels, pixels, q, lo, hi, static_cast<uint4*>(z));
+    return check_launch("quantize_pad3_rows_kernel");
   }
   if (C_pad % 16 == 0 && aligned16(z)) {
     const int groups = C_pad / 16;
@@ -943,6 +1095,12 @@ int q8_quantize_pad_image(const float* x, int N, int H, int W, int C, int W_pad,
   if (rows == 0 || W_pad == 0) return Q8_OK;
   const int lo = out_type == Q8_U8 ? 0 : -128, hi = out_type == Q8_U8 ? 255 : 127;
   const int groups = C_pad / 16;
+  if (C == 3 && C_pad == 16) {
+    const size_t chunks = rows * (((size_t)W_pad + 127) / 128);
+    quantize_pad3_rows_kernel<<<grid_for(chunks, kThreads / 32, 4), kThreads, 0, as_stream(stream)>>>(
+        x, rows, (size_t)W, (size_t)W_pad, q, lo, hi, static_cast<uint4*>(z));
+    return check_launch("quantize_pad3_rows_kernel");
+  }
   quantize_pad_image_kernel<<<grid_for(rows * W_pad * groups, kThreads, 8), kThreads, 0, as_stream(stream)>>>(
       x, rows, W, C, W_pad, groups, q, lo, hi, static_cast<uint4*>(z));
   return check_launch("quantize_pad_image_kernel");
@@ -1001,7 +1159,7 @@ int q8_concat_branch(const void* x, int channels, float in_factor, float out_fac
   cudaStream_t s = as_stream(stream);
   volatile double ratio = (double)in_factor / (double)out_factor;
   float sc = (float)ratio;
-  int copy_only = sc == 1.0f;
+  int copy_only = sc == 1.0f ? 1 : ((sc > 0.0f && sc < 1.0f) ? 2 : 0);  // 2: the clamp-free form (vector kernel)
   const int ch = channels, ctot = y_ldc, off = y_c_offset;
   bool vec = (ch % 16 == 0) && (ctot % 16 == 0) && (off % 16 == 0) && aligned16(x) && aligned16(y);
   if (vec) {

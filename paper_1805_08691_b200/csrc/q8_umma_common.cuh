@@ -210,7 +210,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Slow path of a wait, out of line to keep the role loops small.  Gives up after about
 // kWaitLimitNs or when another role of this CTA has already given up; the caller then records the
 // site and leaves its loop.  The wall clock is only read once the wait has lasted a while.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                            unsigned long long limit_ns = kWaitLimitNs) {
   unsigned long long t0 = 0;
   uint32_t spins = 0;
   for (;;) {
@@ -219,7 +220,7 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
       int give_up = *abort_flag;
       const unsigned long long now = global_timer_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) give_up = 1;
+      else if (now - t0 > limit_ns) give_up = 1;
       if (__any_sync(0xffffffffu, give_up)) return false;
     }
   }

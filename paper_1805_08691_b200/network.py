@@ -9,7 +9,8 @@ for the fused residual sum; all tensor arithmetic runs in the library's kernels.
                                       adds no output (the kernel reads stride-2 inputs as pixel pairs)
   conv + ReLU                       : u8, q = max / 255
   conv without ReLU                 : s8, q = max|y| / 127
-  conv + residual sum + ReLU        : u8, q = max(max|conv|, max|residual|) / 255
+  conv + residual sum + ReLU        : u8, q = max(max|conv|, max|residual|) / 255 (the paper's "+" rule), or with
+                                      sum_policy="post_sum" the calibrated maximum of the sum itself / 255
   dequantized output (logits, heads): fp32
   sibling heads                     : dequantized convolutions that read the same tensor with the same filter
                                       geometry (the localisation and confidence heads of an SSD source map) run as
@@ -40,7 +41,7 @@ from . import pipeline
 
 class QuantNetwork:
     def __init__(self, layers, folded: Dict[str, tuple], maxima: Dict[str, float], in_shape, device="cuda",
-                 per_channel=False, streams=1, fuse=True):
+                 per_channel=False, streams=1, fuse=True, sum_policy="max"):
         """folded[name] = (w KRSC, b K) FP32 device tensors; maxima: calibrated max-abs of "input", every layer
         output and "<name>:pre" of residual convolutions; in_shape = (N, H, W, 3); per_channel: one weight
         factor per output channel instead of one per tensor; streams: independent branches (the
@@ -49,6 +50,8 @@ class QuantNetwork:
         another branch's kernel has already left.  fuse: a convolution whose only reader is a 1x1 convolution runs
         with it in one launch where the library supports the pair (q8_conv2d_then_1x1: same bytes, the tensor between
         them is not written, so it is absent from the returned tensors)."""
+        assert sum_policy in ("max", "post_sum")
+        self.sum_policy = sum_policy
         self.layers = layers
         self.maxima = maxima
         self.by_name = {L.name: L for L in layers}
@@ -197,6 +200,8 @@ class QuantNetwork:
             return self._factor(L.src[0])
         if L.op == "concat":
             return self._factor(name)
+        if L.residual is not None and self.sum_policy == "post_sum":
+            return q8.q8_factor(m[name], 8)       # calibrated on the tensor the layer emits
         if L.residual is not None:
             return q8.q8_factor(max(m[name + ":pre"], m[L.residual]), 8)
         return q8.q8_factor(m[name], 8 if L.conv.relu else 7)

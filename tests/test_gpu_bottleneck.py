@@ -57,9 +57,14 @@ def _run_both(q8, cfg, check_images):
     xq_o = o.quantize(x, fo["q_x"], o.U8)
     xq_g = q8.q8_quantize(_cuda(x), block.q_x, q8.Q8_U8)
     assert np.array_equal(xq_g.cpu().numpy(), xq_o)
+    assert block.fused          # the 3x3 and the expanding 1x1 run as one launch; its 3x3 output is never written
     y = block(xq_g)
     q8.q8_read_status()
-    ya_g, yb_g, y_g = block.ya.cpu().numpy(), block.yb.cpu().numpy(), y.cpu().numpy()
+    plain = pipeline.Bottleneck(folded_g, max_g, x.shape, fuse=False)   # three launches, every tensor written
+    y3 = plain(xq_g)
+    q8.q8_read_status()
+    ya_g, yb_g, y_g = plain.ya.cpu().numpy(), plain.yb.cpu().numpy(), y.cpu().numpy()
+    assert torch.equal(y, y3) and torch.equal(block.ya, plain.ya)
     for n in check_images:
         ya, yb, yo = oracle_net.bottleneck_forward(fo, xq_o[n:n + 1])
         assert np.array_equal(ya_g[n:n + 1], ya)

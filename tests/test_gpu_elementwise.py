@@ -95,9 +95,11 @@ def test_concat_bit_exact(q8, chans, signed):
     lo, hi = (-128, 128) if signed else (0, 256)
     xs = [g.integers(lo, hi, (2, 5, 6, c)).astype(dt) for c in chans]
     fac = [float(np.float32(0.01 * (i + 1))) for i in range(len(chans))]
-    out_f = max(fac)
-    got = q8.q8_concat([_cuda(a) for a in xs], fac, out_f).cpu().numpy()
-    assert np.array_equal(got, o.concat(xs, fac, out_f))
+    # the shared factor as the rule gives it (multipliers <= 1, no clamp can act), and a smaller one (multipliers
+    # > 1: codes saturate)
+    for out_f in (max(fac), min(fac) * 0.75):
+        got = q8.q8_concat([_cuda(a) for a in xs], fac, out_f).cpu().numpy()
+        assert np.array_equal(got, o.concat(xs, fac, out_f))
 
 
 @pytest.mark.parametrize("k,st,pad,ceil", [(3, 2, 1, False), (2, 2, 0, True), (3, 1, 1, False), (3, 2, 0, False), (7, 1, 0, False)])
@@ -121,7 +123,7 @@ def test_3x3_pools_in_row_strips_bit_exact(q8, st, pad, ceil):
     """Tensors large enough for the strip kernel (eight output rows per thread): ragged last strip, both strides,
     padding 0 to 2, extreme codes in the corners, u8 and s8."""
     g = np.random.default_rng(31 * st + pad)
-    x = g.integers(0, 256, (6, 45, 39, 96), dtype=np.uint8)
+    x = g.integers(0, 256, (16, 61, 52, 128), dtype=np.uint8)
     x[:, :2, :2, :] = 255
     x[:, -2:, -2:, :] = 0
     for arr in (x, x.view(np.int8)):

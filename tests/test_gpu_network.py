@@ -38,7 +38,7 @@ def _compare(layers, got, want, net, info, rows=None, check_layers=None):
 
 
 def _run_both(q8, layers, hw, batch, calib_batches, seed, check_layers=None, per_channel=False, streams=1, fuse=False,
-              calib_batch=None, rows=None):
+              calib_batch=None, rows=None, sum_policy="max"):
     """rows: run the library on the whole batch but the oracle only on these images of it (images are independent)."""
     from paper_1805_08691_b200 import network, pipeline
     # fold BN on both sides, must agree bit for bit
@@ -72,10 +72,11 @@ def _run_both(q8, layers, hw, batch, calib_batches, seed, check_layers=None, per
     assert max_g == max_o
     # prepare and run
     x = nets.images(seed + 1, batch, hw)
-    prep, info = oracle_net.network_prepare(layers, folded_o, max_o, per_channel)
+    prep, info = oracle_net.network_prepare(layers, folded_o, max_o, per_channel, sum_policy)
     xo = x if rows is None else np.ascontiguousarray(x[rows])
     want = oracle_net.network_forward(layers, prep, info, xo, threads=min(len(xo), o.hw_threads()))
-    net = network.QuantNetwork(layers, folded_g, max_g, x.shape, per_channel=per_channel, streams=streams, fuse=fuse)
+    net = network.QuantNetwork(layers, folded_g, max_g, x.shape, per_channel=per_channel, streams=streams, fuse=fuse,
+                               sum_policy=sum_policy)
     got = net.forward(_cuda(x))
     q8.q8_read_status()
     _compare(layers, got, want, net, info, rows, check_layers)
@@ -89,6 +90,8 @@ def test_bottleneck_stack_every_layer(q8):
     _run_both(q8, layers, hw=32, batch=3, calib_batches=2, seed=3100, streams=2)
     got, want, ref, net = _run_both(q8, layers, hw=32, batch=3, calib_batches=2, seed=3100, streams=2, fuse=True)
     assert len(net.fused_with) == 2     # the 3x3 of each block runs in one launch with the 1x1 after it
+    # factor of a fused sum calibrated on the sum itself instead of the "+" rule on its summands
+    _run_both(q8, layers, hw=32, batch=3, calib_batches=2, seed=3100, fuse=True, sum_policy="post_sum")
 
 
 # ---- the benchmarked launch configurations: whole batch on the GPU (pair mode, tile widths and reduction splits

@@ -110,6 +110,34 @@ def test_residual_stack_follows_fp32_and_uses_the_plus_rule():
     assert np.array_equal(out["blk1_branch2c"], want.astype(np.uint8))
 
 
+def test_post_sum_policy_calibrates_the_emitted_tensor():
+    """sum_policy="post_sum": the factor of a fused residual sum is the calibrated maximum of the sum itself; every
+    other factor is untouched; on a calibration batch the sum then reaches the top code, which the "+" rule on the
+    two summands only does when the maxima of conv and residual do not add up."""
+    layers = nets.bottleneck_stack(C=16, blocks=2)
+    folded = _fold(layers)
+    x = nets.images(41, 2, 16)
+    acts = nets.fp32_forward(layers, x, folded)
+    maxima = {k: o.maxabs(v) for k, v in acts.items()}
+    prep_m, info_m = oracle_net.network_prepare(layers, folded, maxima)
+    prep_s, info_s = oracle_net.network_prepare(layers, folded, maxima, sum_policy="post_sum")
+    sums = [L.name for L in layers if L.residual is not None]
+    assert sums == ["blk0_branch2c", "blk1_branch2c"]
+    for L in layers:
+        if L.name in sums:
+            assert info_s[L.name][1] == o.factor(maxima[L.name], 8)
+            # |a + b| <= |a| + |b| <= 2 max(|a|, |b|): the post-sum factor is at most twice the "+" rule's
+            assert info_s[L.name][1] <= 2 * info_m[L.name][1]
+    assert info_s["conv1"] == info_m["conv1"] and info_s["blk0_branch2a"] == info_m["blk0_branch2a"]
+    out_s = oracle_net.network_forward(layers, prep_s, info_s, x)
+    # calibrated on this very batch: the largest FP32 value of the sum maps to 255 (quantization noise of the
+    # layers before it moves the largest code by a few steps at most)
+    assert out_s["blk0_branch2c"].max() >= 250
+    ref = acts
+    for name in sums:
+        assert _rel(o.dequantize(out_s[name], info_s[name][1]), ref[name]) < 0.12, name
+
+
 def test_layer_lists_match_the_published_architectures():
     r50, inc, ssd = nets.resnet50(), nets.inception_v3(), nets.ssd300()
     assert sum(L.op == "conv" for L in r50) == 54 and nets.macs(r50, 224) == 3857973248
