@@ -111,8 +111,28 @@ __global__ void __launch_bounds__(kFThreads, 1)
   // Prologue.  Weights, biases and multipliers are constants of the layer pair: they are fetched BEFORE the kernel
   // orders itself behind the previous kernel of the stream (griddepcontrol.wait), so that under a programmatic
   // dependent launch they arrive while that kernel drains.  Only activations (input patches, residual tiles)
-  // wait for it.
-  if (warp == 0) {
+  // wait for it.  The control warps meet on barrier 1 among themselves and start; the epilogue warps touch every line
+  // of the kernel parameters (warming the constant cache for the control warps), stage bias and multipliers, and
+  // join on barrier 3, which the control warps only signal.
+  if (warp >= kFCtrlWarps) {
+    const unsigned int* words = reinterpret_cast<const unsigned int*>(&p);
+    unsigned int touched = 0;
+    const int et = (int)threadIdx.x - kFCtrlWarps * 32, en = kFThreads - kFCtrlWarps * 32;
+    for (int i = et * 16; i < (int)(sizeof(FusedParams) / 4); i += en * 16) touched ^= words[i];
+    asm volatile("" ::"r"(touched));
+    // bias and multiplier of every channel of both layers (zero beyond Cout; one multiplier replicated if per tensor)
+    for (int i = et; i < p.l1.k_pad; i += en) {
+      s_bias1[i] = (p.l1.bias && i < p.l1.K) ? p.l1.bias[i] : 0;
+      s_scale1[i] = p.l1.scale_count == 1 ? p.l1.scale[0] : (i < p.l1.K ? p.l1.scale[i] : 0.f);
+    }
+    for (int i = et; i < p.l2.k_pad; i += en) {
+      s_bias2[i] = (p.l2.bias && i < p.l2.K) ? p.l2.bias[i] : 0;
+      s_scale2[i] = p.l2.scale_count == 1 ? p.l2.scale[0] : (i < p.l2.K ? p.l2.scale[i] : 0.f);
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("bar.sync 3, %0;" ::"r"(kFThreads) : "memory");
+    tcgen05_fence_after();
+  } else if (warp == 0) {
     if (lane < p.l1.stages) { mbar_init(smem_u32(&a_full[lane]), 1); mbar_init(smem_u32(&a_empty[lane]), 1); }
     else if (lane >= 8 && lane - 8 < p.l1.b_stages) { mbar_init(smem_u32(&b_full[lane - 8]), 1); mbar_init(smem_u32(&b_empty[lane - 8]), 1); }
     else if (lane == 16) { mbar_init(smem_u32(&w1_full), 1); mbar_init(smem_u32(&w2_full), 1); abort_flag = 0; }
@@ -137,7 +157,8 @@ __global__ void __launch_bounds__(kFThreads, 1)
     }
     __syncwarp();
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("bar.arrive 1, %0;" ::"r"(kFThreads) : "memory");
+    asm volatile("bar.arrive 1, %0;" ::"r"(kFCtrlWarps * 32) : "memory");
+    asm volatile("bar.arrive 3, %0;" ::"r"(kFThreads) : "memory");
   } else {
     if (warp == 1) {
       if (lane < p.l1.nacc) { mbar_init(smem_u32(&acc1_full[lane]), 1); mbar_init(smem_u32(&acc1_empty[lane]), 4); }
@@ -157,18 +178,10 @@ __global__ void __launch_bounds__(kFThreads, 1)
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (threadIdx.x >= 32 && (int)threadIdx.x - 32 < p.l1.taps) tap_shift16[threadIdx.x - 32] = p.l1.tap_shift16[threadIdx.x - 32];
-    // bias and multiplier of every channel of both layers (zero beyond Cout; one multiplier replicated if per tensor)
-    for (int i = threadIdx.x - 32; i < p.l1.k_pad; i += kFThreads - 32) {
-      s_bias1[i] = (p.l1.bias && i < p.l1.K) ? p.l1.bias[i] : 0;
-      s_scale1[i] = p.l1.scale_count == 1 ? p.l1.scale[0] : (i < p.l1.K ? p.l1.scale[i] : 0.f);
-    }
-    for (int i = threadIdx.x - 32; i < p.l2.k_pad; i += kFThreads - 32) {
-      s_bias2[i] = (p.l2.bias && i < p.l2.K) ? p.l2.bias[i] : 0;
-      s_scale2[i] = p.l2.scale_count == 1 ? p.l2.scale[0] : (i < p.l2.K ? p.l2.scale[i] : 0.f);
-    }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     tcgen05_fence_before();
-    asm volatile("bar.sync 1, %0;" ::"r"(kFThreads) : "memory");
+    asm volatile("bar.arrive 3, %0;" ::"r"(kFThreads) : "memory");
+    asm volatile("bar.sync 1, %0;" ::"r"(kFCtrlWarps * 32) : "memory");
     tcgen05_fence_after();
   }
   const uint32_t tmem_base = warp == 0 ? 0u : tmem_holder;

@@ -195,10 +195,25 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   // Prologue.  Each control lane initialises the barriers it owns.  Warp 0 only signals the
-  // start-up barrier (bar.arrive) and goes straight to its loads, so that the first bytes are on
-  // their way while the others allocate TMEM and fetch bias and scale; everybody else waits on it.
+  // start-up barriers (bar.arrive) and goes straight to its loads, so that the first bytes are on
+  // their way while the others allocate TMEM.  Single CTAs keep the epilogue warps off the critical path: the
+  // control warps meet on barrier 1 among themselves and start; the epilogue warps first touch every line of the
+  // kernel parameters (the control warps' first reads of them would otherwise miss the constant cache one after
+  // the other), fetch bias and scale, and join on barrier 3, which the control warps only signal.
   const int nthreads = kCtrlThreads + G * kGroupThreads;
-  if (warp == 0) {
+  if (!kCta2 && warp >= kCtrlWarps) {
+    const unsigned int* words = reinterpret_cast<const unsigned int*>(&p);
+    unsigned int touched = 0;
+    for (int i = ((int)threadIdx.x - kCtrlThreads) * 16; i < (int)(sizeof(UmmaParams) / 4); i += G * kGroupThreads * 16) touched ^= words[i];
+    asm volatile("" ::"r"(touched));
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    for (int i = (int)threadIdx.x - kCtrlThreads; i < p.k_pad; i += G * kGroupThreads) {
+      s_bias[i] = (p.bias && i < p.K) ? p.bias[i] : 0;
+      s_scale[i] = p.scale ? (p.scale_count == 1 ? p.scale[0] : (i < p.K ? p.scale[i] : 0.f)) : 0.f;
+    }
+    asm volatile("bar.sync 3, %0;" ::"r"(nthreads) : "memory");
+    tcgen05_fence_after();
+  } else if (warp == 0) {
     // one barrier per lane: a lone lane would spend ~50 cycles on each
     if (lane < p.stages) { mbar_init(smem_u32(&a_full[lane]), 1); mbar_init(smem_u32(&a_empty[lane]), 1); }
     else if (lane >= 8 && lane - 8 < p.b_stages) { mbar_init(smem_u32(&b_full[lane - 8]), 1); mbar_init(smem_u32(&b_empty[lane - 8]), 1); }
@@ -208,8 +223,13 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncwarp();
     asm volatile("griddepcontrol.wait;" ::: "memory");  // everything the previous kernel wrote is visible from here
-    if constexpr (kCta2) cluster_sync_all();  // the peer's barriers exist before anything signals them
-    asm volatile("bar.arrive 1, %0;" ::"r"(nthreads) : "memory");
+    if constexpr (kCta2) {
+      cluster_sync_all();  // the peer's barriers exist before anything signals them
+      asm volatile("bar.arrive 1, %0;" ::"r"(nthreads) : "memory");
+    } else {
+      asm volatile("bar.arrive 1, %0;" ::"r"(kCtrlThreads) : "memory");
+      asm volatile("bar.arrive 3, %0;" ::"r"(nthreads) : "memory");
+    }
   } else {
     if (warp == 1) {
       // one arrival per epilogue warp that reads the accumulator: a group's four, or all of them in split mode
@@ -237,17 +257,21 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
     }
     if (p.a_mode == kAHalo && threadIdx.x >= 32 && threadIdx.x - 32 < p.taps) tap_shift16[threadIdx.x - 32] = p.tap_shift16[threadIdx.x - 32];
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    // bias and scale of every channel, once per CTA (zero beyond Cout; one scale replicated if per tensor)
-    for (int i = threadIdx.x - 32; i < p.k_pad; i += nthreads - 32) {
-      s_bias[i] = (p.bias && i < p.K) ? p.bias[i] : 0;
-      s_scale[i] = p.scale ? (p.scale_count == 1 ? p.scale[0] : (i < p.K ? p.scale[i] : 0.f)) : 0.f;
-    }
-    tcgen05_fence_before();
     if constexpr (kCta2) {
+      // bias and scale of every channel, once per CTA (zero beyond Cout; one scale replicated if per tensor)
+      for (int i = threadIdx.x - 32; i < p.k_pad; i += nthreads - 32) {
+        s_bias[i] = (p.bias && i < p.K) ? p.bias[i] : 0;
+        s_scale[i] = p.scale ? (p.scale_count == 1 ? p.scale[0] : (i < p.K ? p.scale[i] : 0.f)) : 0.f;
+      }
+      tcgen05_fence_before();
       __syncwarp();
       cluster_sync_all();
+      asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
+    } else {
+      tcgen05_fence_before();
+      asm volatile("bar.arrive 3, %0;" ::"r"(nthreads) : "memory");      // the epilogue warps wait for this set-up
+      asm volatile("bar.sync 1, %0;" ::"r"(kCtrlThreads) : "memory");    // the control warps only for each other
     }
-    asm volatile("bar.sync 1, %0;" ::"r"(nthreads) : "memory");
     tcgen05_fence_after();
   }
   const uint32_t tmem_base = warp == 0 ? 0u : tmem_holder;  // warp 0 never touches TMEM
