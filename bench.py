@@ -763,11 +763,19 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sets", type=int, default=6, help="rotating buffer sets (working set must exceed L2)")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--bandwidth-only", type=int, default=0, metavar="REPS",
+                    help="run only the memory-bound kernels, REPS timed launches each, print their JSON and exit "
+                         "(the command the ncu summary of these kernels is taken with)")
     ap.add_argument("--skip-networks", "--skip-resnet50", dest="skip_networks", action="store_true",
                     help="leave out the whole-network numbers (ResNet-50, Inception-v3, SSD-300)")
     args = ap.parse_args()
     if args.steps is None:
         args.steps = 3 if args.impl == "reference" else 12000
+    if args.bandwidth_only:
+        import torch
+        print(json.dumps({"bandwidth_kernels": bandwidth_kernel_numbers(torch.device("cuda", 0), measured_peaks()["hbm_gbs"],
+                                                                        reps=args.bandwidth_only)}), flush=True)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:

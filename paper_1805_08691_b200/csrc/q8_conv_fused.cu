@@ -411,6 +411,9 @@ int launch_fused_variant(const CUtensorMap& tmA, const CUtensorMap& tmB1, const 
     int rc = check_cuda(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit - kStaticSmemReserve),
                         "conv_fused: set shared memory size");
     if (rc != Q8_OK) return rc;
+    rc = check_cuda(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared),
+                    "conv_fused: set shared memory carve-out");
+    if (rc != Q8_OK) return rc;
     if (dev >= 0) configured[dev].store(true, std::memory_order_release);
   }
   cudaLaunchConfig_t cfg;

@@ -589,6 +589,11 @@ int launch_variant(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtenso
     int rc = check_cuda(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit - kStaticSmemReserve),
                         "conv_umma: set shared memory size");
     if (rc != Q8_OK) return rc;
+    // every tensor-core kernel of the library asks for the largest shared-memory carve-out, so that consecutive
+    // launches of different kernels or shapes never make the SMs switch their L1 / shared-memory split
+    rc = check_cuda(cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared),
+                    "conv_umma: set shared memory carve-out");
+    if (rc != Q8_OK) return rc;
     if (dev >= 0) configured[dev].store(true, std::memory_order_release);
   }
   cudaLaunchConfig_t cfg;

@@ -344,8 +344,55 @@ def test_pools_against_library(k, st, pad, ceil):
         sums = F.avg_pool2d(xt, k, st, pad, count_include_pad=True, divisor_override=1).permute(0, 2, 3, 1).numpy()
         want = np.rint(sums.astype(np.float32) * (np.float32(1) / np.float32(k * k))).astype(np.uint8)
         assert np.array_equal(o.pool(x, "avg", (k, k), (st, st), (pad, pad), ceil), want)
+    # average pooling in both modes, signed input too, against window sums taken by slicing a zero-embedded copy
+    # (cells outside the image count as zeros, the divisor is the full window; ceil mode only adds windows)
+    for arr in (x, x.view(np.int8)):
+        N, H, W, C = arr.shape
+        P, Q = o.pool_out(H, k, st, pad, ceil), o.pool_out(W, k, st, pad, ceil)
+        big = np.zeros((N, pad + (P - 1) * st + k + pad, pad + (Q - 1) * st + k + pad, C), dtype=np.int64)
+        big[:, pad:pad + H, pad:pad + W, :] = arr
+        want = np.empty((N, P, Q, C), dtype=arr.dtype)
+        for pi in range(P):
+            for qi in range(Q):
+                sums = big[:, pi * st:pi * st + k, qi * st:qi * st + k, :].sum(axis=(1, 2))
+                want[:, pi, qi, :] = np.rint(sums.astype(np.float32) * (np.float32(1) / np.float32(k * k))).astype(arr.dtype)
+        assert np.array_equal(o.pool(arr, "avg", (k, k), (st, st), (pad, pad), ceil), want)
 
 
 def test_pool_ceil_mode_extent():
     assert o.pool_out(75, 2, 2, 0, True) == 38 and o.pool_out(75, 2, 2, 0, False) == 37
     assert o.pool_out(112, 3, 2, 1, False) == 56 and o.pool_out(147, 3, 2, 0, False) == 73
+
+
+# ----------------------------------------------------------------------------- multiplier and dequantizer, by properties
+def test_requant_scale_exact_on_powers_of_two_and_single_rounding():
+    """s = q_x q_w / q_y: with powers of two every step is exact, so the value is known without any formula of the
+    test's own; for general factors the result is the fp32 nearest to the exact rational (one rounding), which the
+    rational arithmetic of Python's fractions decides."""
+    from fractions import Fraction
+    assert o.requant_scale(0.5, 0.25, 0.125) == 1.0
+    assert o.requant_scale(2.0 ** -7, 2.0 ** -9, 2.0 ** -3) == 2.0 ** -13
+    assert o.requant_scale(0.5, 0.25, 0.25) == 2 * o.requant_scale(0.5, 0.25, 0.5)
+    g = np.random.default_rng(12)
+    for _ in range(200):
+        qx, qw, qy = (float(np.float32(v)) for v in g.uniform(1e-4, 2.0, 3))
+        exact = Fraction(qx) * Fraction(qw) / Fraction(qy)
+        s = float(o.requant_scale(qx, qw, qy))
+        lo, hi = float(np.nextafter(np.float32(s), np.float32(-np.inf))), float(np.nextafter(np.float32(s), np.float32(np.inf)))
+        assert abs(Fraction(s) - exact) <= abs(Fraction(lo) - exact) and abs(Fraction(s) - exact) <= abs(Fraction(hi) - exact)
+
+
+def test_dequantize_is_one_fp32_product():
+    """r' = q z: exact for power-of-two factors, odd in z, and the fp32 nearest to the exact product otherwise."""
+    from fractions import Fraction
+    z = np.arange(-128, 128, dtype=np.int8)
+    assert np.array_equal(o.dequantize(z, 0.25), z.astype(np.float32) / 4)
+    assert np.array_equal(o.dequantize(z[1:], 0.3), -o.dequantize((-z[1:].astype(np.int16)).astype(np.int8), 0.3))
+    q = float(np.float32(0.0123))
+    got = o.dequantize(np.array([77, 255], dtype=np.uint8), q)
+    for v, zz in zip(got, (77, 255)):
+        exact = Fraction(q) * zz
+        near = [float(v), float(np.nextafter(v, np.float32(-np.inf))), float(np.nextafter(v, np.float32(np.inf)))]
+        assert min(near, key=lambda c: abs(Fraction(c) - exact)) == float(v)
+    big = o.dequantize(np.array([2 ** 30 + 12345, -(2 ** 31)], dtype=np.int32), 0.5)    # int32 -> fp32 rounds first
+    assert big[0] == np.float32(2 ** 30 + 12345) * np.float32(0.5) and big[1] == -(2.0 ** 30)
