@@ -330,6 +330,7 @@ __global__ void __launch_bounds__(kFThreads, 1)
     const int pp = row / q.twb, qq = row - pp * q.twb;  // accumulator row -> pixel of the patch grid
     t.smem_ok = pp < q.th && qq < q.tw;
     t.srow = t.smem_ok ? pp * q.tw + qq : 0;
+    epi_row_setup(q, t);
     t.n0 = 0; t.y_off = 0; t.m = 0; t.row_ok = false;
     const uint32_t accf0 = smem_u32(&acc1_full[0]), acce0 = smem_u32(&acc1_empty[0]);
     const uint32_t tbf0 = smem_u32(&tb_full[0]), tbe0 = smem_u32(&tb_empty[0]);
@@ -362,6 +363,7 @@ __global__ void __launch_bounds__(kFThreads, 1)
     t.s_scale = s_scale2;
     t.srow = row;                               // T rows are the tile's pixels in dense order
     t.smem_ok = row < p.l1.th * p.l1.tw;
+    epi_row_setup(q, t);
     t.y_off = 0; t.m = 0; t.row_ok = false;
     const uint32_t accf = smem_u32(&acc2_full[g]), acce = smem_u32(&acc2_empty[g]);
     const uint32_t bfull0 = smem_u32(&buf_full[0]), ready0 = smem_u32(&store_ready[0]);

@@ -514,6 +514,7 @@ __global__ void __launch_bounds__(kCtrlThreads + G * kGroupThreads, 1)
       t.smem_ok = pp < p.th && qq < p.tw;
       t.srow = t.smem_ok ? pp * p.tw + qq : 0;
     }
+    epi_row_setup(p, t);
     // this group's tiles are lt = g, g + G, ... of the CTA's sequence; ring positions advance by additions
     // pair mode: the accumulators of both CTAs are handed back on the leader's barriers
     const uint32_t accf0 = smem_u32(&acc_full[0]);

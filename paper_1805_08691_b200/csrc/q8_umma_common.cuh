@@ -469,10 +469,19 @@ struct EpiTile {
   long long m;             // output pixel (row of the [M][Cout] result) of this thread
   long long y_off;         // element offset of this work item's output (split-K partial results), else 0
   int srow;                // row of this thread's pixel inside the 8-bit tile buffer
+  uint32_t row_base, swz;  // byte offset of that row inside a panel, and the row's swizzle term (set by epi_row_setup)
   int n0;                  // first channel of the tile
   bool row_ok;             // the pixel exists (inside the image and below M)
   bool smem_ok;            // this accumulator row maps to a pixel of the tile (always, except halo tiles)
 };
+
+// Position of a thread's row in the swizzled 8-bit tile buffers: constant for the thread's lifetime.  A panel is
+// 128 rows of 2^pw_shift bytes; the 16-byte chunk index of a row is XORed with address bits 7.. (the swizzle the
+// TMA and the tensor core use), which for rows of one swizzle span depend on the row alone.
+__device__ __forceinline__ void epi_row_setup(const UmmaParams& p, EpiTile& t) {
+  t.row_base = (uint32_t)t.srow << p.pw_shift;
+  t.swz = ((t.row_base >> 7) & (uint32_t)p.pmask) << 4;
+}
 
 // One 16-column chunk of one accumulator row.  kOut: Q8_U8, Q8_S8, Q8_S32 or Q8_F32.  kRes: kResNone, kResTma
 // (a residual from the tile buffer if p.res_mode says so, else none: decided at run time) or kResGlobal.  Fewer
@@ -515,9 +524,7 @@ __device__ __forceinline__ void epilogue_chunk(const UmmaParams& p, const EpiTil
   uint32_t off = 0;
   if (kOut == Q8_U8 || kOut == Q8_S8 || (kRes == kResTma && p.res_mode == kResTma)) {
     const int pn = c16 >> p.pw_shift;
-    off = ((uint32_t)t.srow << p.pw_shift) + (uint32_t)(c16 & ((1 << p.pw_shift) - 1));
-    off ^= ((off >> 7) & (uint32_t)p.pmask) << 4;
-    off += (uint32_t)pn * ((uint32_t)kBM << p.pw_shift);
+    off = t.row_base + (((uint32_t)(c16 & ((1 << p.pw_shift) - 1))) ^ t.swz) + (uint32_t)pn * ((uint32_t)kBM << p.pw_shift);
   }
   unsigned long long v2[8];  // v[2i], v[2i + 1]
   float v[16];
