@@ -210,30 +210,59 @@ __global__ void __launch_bounds__(kThreads) quantize_pad_image_kernel(const floa
 }
 
 // Images: 3 channels -> 16, rows of W pixels padded to W_pad output pixels.  A warp takes 128 output pixels of one
-// row: it reads their 384 floats with fully coalesced 4-byte loads into shared memory, then every lane quantizes
-// four pixels (three conflict-free shared-memory reads each) and the warp writes 512 contiguous bytes per store.
-// (One thread per pixel reads 12-byte and writes 16-byte pieces 48 / 64 bytes apart: a third / a quarter of every
-// sector per instruction, measured 61 % of the copy bandwidth.)
-__global__ void __launch_bounds__(kThreads) quantize_pad3_rows_kernel(const float* __restrict__ x, size_t rows, size_t W,
-                                                                      size_t W_pad, float q, int lo, int hi,
-                                                                      uint4* __restrict__ z) {
-  __shared__ float stage[kThreads / 32][384];
+// row: their 384 floats travel to shared memory as asynchronous copies (16 bytes each where the chunk starts on a
+// 16-byte boundary, else 4), the copies of the warp's next chunk are in flight while every lane quantizes four pixels
+// of the present one (three conflict-free shared-memory reads each), and the warp writes 512 contiguous bytes per
+// store.  (One thread per pixel reads 12-byte and writes 16-byte pieces 48 / 64 bytes apart: a third / a quarter
+// of every sector per instruction, measured 61 % of the copy bandwidth; without the second buffer the loads and
+// the arithmetic of a warp alternate, 66 %.)
+constexpr int kPadThreads = 256;
+
+__device__ __forceinline__ void cp_async4(float* dst, const float* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((unsigned)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async16(float* dst, const float* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((unsigned)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+}
+
+__global__ void __launch_bounds__(kPadThreads, 8) quantize_pad3_rows_kernel(const float* __restrict__ x, size_t rows, size_t W,
+                                                                            size_t W_pad, float q, int lo, int hi,
+                                                                            uint4* __restrict__ z) {
+  __shared__ __align__(16) float stage[2][kPadThreads / 32][384];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  float* st = stage[warp];
   const size_t chunks_per_row = (W_pad + 127) / 128, chunks = rows * chunks_per_row;
-  const size_t nwarps = (size_t)gridDim.x * (kThreads / 32);
-  for (size_t ch = (size_t)blockIdx.x * (kThreads / 32) + warp; ch < chunks; ch += nwarps) {
-    const size_t r = ch / chunks_per_row, w0 = (ch - r * chunks_per_row) * 128;
-    const size_t in_px = w0 < W ? (W - w0 < 128 ? W - w0 : 128) : 0;      // real pixels of this chunk
-    const size_t out_px = W_pad - w0 < 128 ? W_pad - w0 : 128;
-    const float* src = x + (r * W + w0) * 3;
-    const int nf = (int)in_px * 3;
+  const size_t nwarps = (size_t)gridDim.x * (kPadThreads / 32);
+  auto fetch = [&](size_t ch, int buf) {
+    if (ch < chunks) {
+      const size_t r = ch / chunks_per_row, w0 = (ch - r * chunks_per_row) * 128;
+      const size_t in_px = w0 < W ? (W - w0 < 128 ? W - w0 : 128) : 0;      // real pixels of this chunk
+      const float* src = x + (r * W + w0) * 3;
+      float* st = stage[buf][warp];
+      if (in_px == 128 && (reinterpret_cast<uintptr_t>(src) & 15) == 0) {
 #pragma unroll
-    for (int k = 0; k < 12; ++k) {
-      const int f = k * 32 + lane;
-      if (f < nf) st[f] = __ldcs(src + f);
+        for (int k = 0; k < 3; ++k) cp_async16(st + (k * 32 + lane) * 4, src + (k * 32 + lane) * 4);
+      } else {
+        const int nf = (int)in_px * 3;
+#pragma unroll
+        for (int k = 0; k < 12; ++k) {
+          const int f = k * 32 + lane;
+          if (f < nf) cp_async4(st + f, src + f);
+        }
+      }
     }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  size_t ch = (size_t)blockIdx.x * (kPadThreads / 32) + warp;
+  int buf = 0;
+  fetch(ch, 0);
+  for (; ch < chunks; ch += nwarps, buf ^= 1) {
+    fetch(ch + nwarps, buf ^ 1);
+    asm volatile("cp.async.wait_group 1;" ::: "memory");
     __syncwarp();
+    const size_t r = ch / chunks_per_row, w0 = (ch - r * chunks_per_row) * 128;
+    const size_t in_px = w0 < W ? (W - w0 < 128 ? W - w0 : 128) : 0;
+    const size_t out_px = W_pad - w0 < 128 ? W_pad - w0 : 128;
+    const float* st = stage[buf][warp];
     uint4* out = z + r * W_pad + w0;
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
@@ -246,6 +275,7 @@ __global__ void __launch_bounds__(kThreads) quantize_pad3_rows_kernel(const floa
     }
     __syncwarp();
   }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -366,38 +396,99 @@ __device__ __forceinline__ unsigned int requant_word_small(unsigned int w, float
   return __byte_perm(__byte_perm(z0, z1, 0x0040u), __byte_perm(z2, z3, 0x0040u), 0x5410u);
 }
 
-// vec path: channels, c_total and c_off multiples of 16, pointers 16-byte aligned
-template <bool kSigned>
-__global__ void __launch_bounds__(kThreads) concat_vec_kernel(const uint4* __restrict__ x, size_t pixels, int cvec,
-                                                              int ctot_vec, int coff_vec, float s, int copy_only,
-                                                              uint4* __restrict__ y) {
-  const size_t total = pixels * (size_t)cvec;
-  const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+// vec path: channels, c_total and c_off multiples of 16, pointers 16-byte aligned.
+// One thread moves 16-byte groups i0, i0 + nthreads, ... of a branch; two loads are issued before the first of
+// them is used, with all 2048 threads of an SM resident (a loop whose body branches on the kind of multiplier kept one load in flight per thread and ran at
+// 0.67 of the copy bandwidth).  kMode 0: general multiplier, 1: copy, 2: multiplier in (0, 1).
+template <bool kSigned, int kMode>
+__device__ __forceinline__ uint4 concat_word(uint4 v, float s) {
+  if (kMode == 2) {
+    v.x = requant_word_small<kSigned>(v.x, s);
+    v.y = requant_word_small<kSigned>(v.y, s);
+    v.z = requant_word_small<kSigned>(v.z, s);
+    v.w = requant_word_small<kSigned>(v.w, s);
+  } else if (kMode == 0) {
+    v.x = requant_word<kSigned>(v.x, s);
+    v.y = requant_word<kSigned>(v.y, s);
+    v.z = requant_word<kSigned>(v.z, s);
+    v.w = requant_word<kSigned>(v.w, s);
+  }
+  return v;
+}
+
+template <bool kSigned, int kMode>
+__device__ __forceinline__ void concat_span(const uint4* __restrict__ x, size_t total, int cvec, int ctot_vec,
+                                            int coff_vec, float s, size_t i, size_t nthreads, uint4* __restrict__ y) {
   // (pixel, 16-byte group) of this thread's element, advanced by additions: one division per thread
-  size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   size_t px = i / cvec;
   int c = (int)(i - px * cvec);
   const size_t dpx = nthreads / cvec;
   const int dc = (int)(nthreads - dpx * cvec);
-#pragma unroll 4
-  for (; i < total; i += nthreads) {
-    uint4 v = __ldcs(x + i);
-    if (copy_only == 2) {  // multiplier in (0, 1]
-      v.x = requant_word_small<kSigned>(v.x, s);
-      v.y = requant_word_small<kSigned>(v.y, s);
-      v.z = requant_word_small<kSigned>(v.z, s);
-      v.w = requant_word_small<kSigned>(v.w, s);
-    } else if (!copy_only) {
-      v.x = requant_word<kSigned>(v.x, s);
-      v.y = requant_word<kSigned>(v.y, s);
-      v.z = requant_word<kSigned>(v.z, s);
-      v.w = requant_word<kSigned>(v.w, s);
+  constexpr int kBatch = 2;
+  for (; i + (kBatch - 1) * nthreads < total; i += kBatch * nthreads) {
+    uint4 v[kBatch];
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) v[u] = __ldcs(x + i + u * nthreads);
+#pragma unroll
+    for (int u = 0; u < kBatch; ++u) {
+      y[px * ctot_vec + coff_vec + c] = concat_word<kSigned, kMode>(v[u], s);
+      px += dpx;
+      c += dc;
+      if (c >= cvec) { c -= cvec; ++px; }
     }
-    y[px * ctot_vec + coff_vec + c] = v;
+  }
+  for (; i < total; i += nthreads) {
+    y[px * ctot_vec + coff_vec + c] = concat_word<kSigned, kMode>(__ldcs(x + i), s);
     px += dpx;
     c += dc;
     if (c >= cvec) { c -= cvec; ++px; }
   }
+}
+
+template <bool kSigned>
+__device__ __forceinline__ void concat_span_mode(int mode, const uint4* __restrict__ x, size_t total, int cvec,
+                                                 int ctot_vec, int coff_vec, float s, size_t i, size_t nthreads,
+                                                 uint4* __restrict__ y) {
+  if (mode == 1) concat_span<kSigned, 1>(x, total, cvec, ctot_vec, coff_vec, s, i, nthreads, y);
+  else if (mode == 2) concat_span<kSigned, 2>(x, total, cvec, ctot_vec, coff_vec, s, i, nthreads, y);
+  else concat_span<kSigned, 0>(x, total, cvec, ctot_vec, coff_vec, s, i, nthreads, y);
+}
+
+template <bool kSigned>
+__global__ void __launch_bounds__(kThreads, 4) concat_vec_kernel(const uint4* __restrict__ x, size_t pixels, int cvec,
+                                                              int ctot_vec, int coff_vec, float s, int copy_only,
+                                                              uint4* __restrict__ y) {
+  concat_span_mode<kSigned>(copy_only, x, pixels * (size_t)cvec, cvec, ctot_vec, coff_vec, s,
+                            (size_t)blockIdx.x * blockDim.x + threadIdx.x, (size_t)gridDim.x * blockDim.x, y);
+}
+
+// All branches in one launch: a block belongs to one branch (its range of block indices is proportional to the
+// branch's bytes) and moves that branch with the blocks of its range.
+struct ConcatBranch {
+  const uint4* x;
+  int cvec, coff_vec;
+  float s;
+  int mode;            // 0: general multiplier, 1: copy, 2: multiplier in (0, 1)
+  unsigned int block0; // first block of this branch
+};
+struct ConcatBranches {
+  ConcatBranch b[8];
+  int n;
+  unsigned int blocks;  // all branches
+};
+
+template <bool kSigned>
+__global__ void __launch_bounds__(kThreads, 4) concat_multi_kernel(const __grid_constant__ ConcatBranches br, size_t pixels,
+                                                                int ctot_vec, uint4* __restrict__ y) {
+  int k = 0;
+#pragma unroll
+  for (int j = 1; j < 8; ++j)
+    if (j < br.n && blockIdx.x >= br.b[j].block0) k = j;
+  const ConcatBranch& me = br.b[k];
+  const unsigned int nblocks = (k + 1 < br.n ? br.b[k + 1].block0 : br.blocks) - me.block0;
+  concat_span_mode<kSigned>(me.mode, me.x, pixels * (size_t)me.cvec, me.cvec, ctot_vec, me.coff_vec, me.s,
+                            (size_t)(blockIdx.x - me.block0) * blockDim.x + threadIdx.x,
+                            (size_t)nblocks * blockDim.x, y);
 }
 
 template <bool kSigned>
@@ -1066,7 +1157,7 @@ int q8_quantize_pad_channels(const float* x, size_t pixels, int C, int C_pad, fl
   if (pixels == 0) return Q8_OK;
   const int lo = out_type == Q8_U8 ? 0 : -128, hi = out_type == Q8_U8 ? 255 : 127;
   if (C == 3 && C_pad == 16 && aligned16(z)) {
-    quantize_pad3_rows_kernel<<<grid_for((pixels + 127) / 128, kThreads / 32, 4), kThreads, 0, as_stream(stream)>>>(
+    quantize_pad3_rows_kernel<<<grid_for((pixels + 127) / 128, kPadThreads / 32, 8), kPadThreads, 0, as_stream(stream)>>>(
         x, 1, pixels, pixels, q, lo, hi, static_cast<uint4*>(z));
     return check_launch("quantize_pad3_rows_kernel");
   }
@@ -1097,7 +1188,7 @@ int q8_quantize_pad_image(const float* x, int N, int H, int W, int C, int W_pad,
   const int groups = C_pad / 16;
   if (C == 3 && C_pad == 16) {
     const size_t chunks = rows * (((size_t)W_pad + 127) / 128);
-    quantize_pad3_rows_kernel<<<grid_for(chunks, kThreads / 32, 4), kThreads, 0, as_stream(stream)>>>(
+    quantize_pad3_rows_kernel<<<grid_for(chunks, kPadThreads / 32, 8), kPadThreads, 0, as_stream(stream)>>>(
         x, rows, (size_t)W, (size_t)W_pad, q, lo, hi, static_cast<uint4*>(z));
     return check_launch("quantize_pad3_rows_kernel");
   }
@@ -1187,6 +1278,36 @@ int q8_concat(int n_in, const void* const* xs, const int* channels, const float*
     ctot += channels[i];
   }
   if (ctot > 0x7fffffffLL) return fail(Q8_ERR_INVALID_ARG, "q8_concat: too many channels");
+  if (pixels == 0) return Q8_OK;
+  // one launch for all branches when every branch takes the 16-byte path
+  bool vec = n_in > 1 && ctot % 16 == 0 && aligned16(y);
+  for (int i = 0; i < n_in && vec; ++i) vec = channels[i] % 16 == 0 && aligned16(xs[i]);
+  if (vec) {
+    ConcatBranches br{};
+    br.n = n_in;
+    size_t items = pixels * (size_t)(ctot / 16);
+    const unsigned int grid = (unsigned int)grid_for(items, kThreads, 4);
+    unsigned int next = 0;
+    int coff = 0;
+    for (int i = 0; i < n_in; ++i) {
+      volatile double ratio = (double)in_factors[i] / (double)out_factor;
+      float sc = (float)ratio;
+      br.b[i].x = static_cast<const uint4*>(xs[i]);
+      br.b[i].cvec = channels[i] / 16;
+      br.b[i].coff_vec = coff / 16;
+      br.b[i].s = sc;
+      br.b[i].mode = sc == 1.0f ? 1 : ((sc > 0.0f && sc < 1.0f) ? 2 : 0);
+      br.b[i].block0 = next;
+      unsigned long long share = ((unsigned long long)grid * (unsigned long long)channels[i] + ctot - 1) / ctot;
+      next += (unsigned int)(share < 1 ? 1 : share);
+      coff += channels[i];
+    }
+    br.blocks = next;
+    cudaStream_t s = as_stream(stream);
+    if (t == Q8_S8) concat_multi_kernel<true><<<next, kThreads, 0, s>>>(br, pixels, (int)(ctot / 16), static_cast<uint4*>(y));
+    else concat_multi_kernel<false><<<next, kThreads, 0, s>>>(br, pixels, (int)(ctot / 16), static_cast<uint4*>(y));
+    return check_launch("concat_multi_kernel");
+  }
   int off = 0;
   for (int i = 0; i < n_in; ++i) {
     int rc = q8_concat_branch(xs[i], channels[i], in_factors[i], out_factor, t, pixels, y, (int)ctot, off, stream);

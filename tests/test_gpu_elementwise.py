@@ -102,6 +102,20 @@ def test_concat_bit_exact(q8, chans, signed):
         assert np.array_equal(got, o.concat(xs, fac, out_f))
 
 
+@pytest.mark.parametrize("signed", [False, True])
+def test_concat_one_launch_many_blocks_per_branch(q8, signed):
+    """All branches 16-byte aligned: one launch whose blocks are split between the branches; a copied branch, one
+    with a multiplier below one, one above one, and a single-group branch, over enough pixels for many blocks each."""
+    g = np.random.default_rng(77)
+    dt = np.int8 if signed else np.uint8
+    lo, hi = (-128, 128) if signed else (0, 256)
+    chans = (192, 16, 64, 128)
+    fac = [0.02, 0.013, 0.031, 0.0071]
+    xs = [g.integers(lo, hi, (3, 71, 53, c)).astype(dt) for c in chans]
+    got = q8.q8_concat([_cuda(a) for a in xs], fac, 0.02).cpu().numpy()
+    assert np.array_equal(got, o.concat(xs, fac, 0.02))
+
+
 @pytest.mark.parametrize("k,st,pad,ceil", [(3, 2, 1, False), (2, 2, 0, True), (3, 1, 1, False), (3, 2, 0, False), (7, 1, 0, False)])
 @pytest.mark.parametrize("C", [64, 48, 12, 5])
 def test_pools_bit_exact(q8, k, st, pad, ceil, C):
