@@ -734,96 +734,106 @@ void launch_pool16_window(const void* x, int N, int H, int W, int cg, int st_h, 
 // (three 16-byte loads) and keeping the last rows' partial results in registers.  The one-thread-per-output form
 // above issues nine loads per output (measured 29 % of the copy bandwidth for stride 1, 50 % for stride 2); here an
 // output costs two (stride 1, two columns per thread) or six (stride 2) loads.
-// Average: bytes are summed as 16-bit lanes (signed input biased by +128 per in-image cell), the sum becomes a
-// float exactly through the 2^23 trick, then clamp(Round(float(sum) * inv)) as defined: one fp32 multiply, round
-// half even by adding 1.5 * 2^23 (|v| <= 255, and a full-window divisor keeps the result inside the 8-bit range).
+// Average: bytes are summed as 16-bit lanes (signed input biased by +128 per in-image cell); the rounding of
+// clamp(Round(float(sum) * fp32(1/9))) is taken by one fused multiply-add per value (see pool_combine3; a
+// full-window divisor keeps the result inside the 8-bit range, so the clamp never acts).
+// Maximum: the same 16-bit lanes (signed input made unsigned by flipping the sign bits), reduced with the native
+// two-lane maximum of two or three operands; the byte-wise SIMD maximum is emulated by about ten instructions per
+// word (measured: 415 warp instructions per 512 output bytes, ALU pipe 72 % busy, 0.56 of the copy bandwidth).
 struct PoolRow {
-  unsigned int a[4], b[4];  // max: a = byte-wise maximum.  average: a = lanes of bytes 0,2; b = lanes of bytes 1,3
+  unsigned int a[4], b[4];  // a = lanes of bytes 0,2; b = lanes of bytes 1,3 (sums, or maxima of sign-flipped bytes)
   int cells;                // average, signed input: in-image cells that went into the sums
 };
+
+__device__ __forceinline__ unsigned int max_u16x2(unsigned int a, unsigned int b) {
+  unsigned int d;
+  asm("max.u16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
 
 template <bool kSigned, bool kAvg>
 __device__ __forceinline__ PoolRow pool_row3(const uint4* __restrict__ img, int h, int H, int W, int cg, int w0) {
   PoolRow r;
-  const unsigned int init = (!kAvg && kSigned) ? 0x80808080u : 0u;
 #pragma unroll
-  for (int j = 0; j < 4; ++j) { r.a[j] = init; r.b[j] = 0u; }
+  for (int j = 0; j < 4; ++j) { r.a[j] = 0u; r.b[j] = 0u; }
   r.cells = 0;
   if (h < 0 || h >= H) return r;
   const uint4* row = img + (size_t)h * W * cg;
+  const unsigned int flip = kSigned ? 0x80808080u : 0u;
   uint4 v[3];
   bool ok[3];
 #pragma unroll
   for (int s = 0; s < 3; ++s) {
     ok[s] = w0 + s >= 0 && w0 + s < W;
-    v[s] = ok[s] ? __ldg(row + (size_t)(w0 + s) * cg) : make_uint4(init, init, init, init);
+    v[s] = ok[s] ? __ldg(row + (size_t)(w0 + s) * cg) : make_uint4(flip, flip, flip, flip);
   }
+  unsigned int e[3][4], o[3][4];
 #pragma unroll
   for (int s = 0; s < 3; ++s) {
     const unsigned int word[4] = {v[s].x, v[s].y, v[s].z, v[s].w};
-    if (!kAvg) {
 #pragma unroll
-      for (int j = 0; j < 4; ++j) r.a[j] = kSigned ? __vmaxs4(r.a[j], word[j]) : __vmaxu4(r.a[j], word[j]);
-    } else if (ok[s]) {
-      const unsigned int flip = kSigned ? 0x80808080u : 0u;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const unsigned int wj = word[j] ^ flip;
-        r.a[j] += wj & 0x00ff00ffu;
-        r.b[j] += __byte_perm(wj, 0u, 0x4341u);  // bytes 1 and 3 as 16-bit lanes
-      }
-      ++r.cells;
+    for (int j = 0; j < 4; ++j) {
+      const unsigned int wj = word[j] ^ flip;  // outside the image: 0, the identity of both reductions
+      e[s][j] = wj & 0x00ff00ffu;
+      o[s][j] = __byte_perm(wj, 0u, 0x4341u);  // bytes 1 and 3 as 16-bit lanes
     }
+    if (ok[s]) ++r.cells;
+  }
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    if (kAvg) { r.a[j] = e[0][j] + e[1][j] + e[2][j]; r.b[j] = o[0][j] + o[1][j] + o[2][j]; }
+    else { r.a[j] = __vimax3_u16x2(e[0][j], e[1][j], e[2][j]); r.b[j] = __vimax3_u16x2(o[0][j], o[1][j], o[2][j]); }
   }
   return r;
 }
 
 template <bool kSigned, bool kAvg>
-__device__ __forceinline__ uint4 pool_combine3(const PoolRow& r0, const PoolRow& r1, const PoolRow& r2, float inv) {
+__device__ __forceinline__ uint4 pool_combine3(const PoolRow& r0, const PoolRow& r1, const PoolRow& r2) {
   unsigned int out[4];
   if (!kAvg) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j)
-      out[j] = kSigned ? __vmaxs4(__vmaxs4(r0.a[j], r1.a[j]), r2.a[j]) : __vmaxu4(__vmaxu4(r0.a[j], r1.a[j]), r2.a[j]);
+    for (int j = 0; j < 4; ++j) {
+      const unsigned int e = __vimax3_u16x2(r0.a[j], r1.a[j], r2.a[j]);
+      const unsigned int o = __vimax3_u16x2(r0.b[j], r1.b[j], r2.b[j]);
+      out[j] = __byte_perm(e, o, 0x6240u) ^ (kSigned ? 0x80808080u : 0u);
+    }
   } else {
-    // float(lane) = bits(0x4B00LLLL) - 2^23 exactly; the +128 per cell of signed input comes off in the same subtraction
-    const float off = 8388608.0f + (kSigned ? 128.0f * (float)(r0.cells + r1.cells + r2.cells) : 0.0f);
+    // One fused multiply-add per value.  bits(0x4B10LLLL) is the float 9 * 2^20 + n exactly (n = the lane, for signed
+    // input raised to sum + 128 * 9 first); times fp32(1/9) that is 2^20 + n/9 + d with 0 < d < 0.01, and adding the
+    // integer 1.5 * 2^23 - 2^20 (- 128 for signed input) rounds once, half to even at unit spacing, leaving
+    // Round(n/9) in the low mantissa bits.  n/9 lies at least 1/18 from a tie, so d changes nothing, and neither does
+    // the rounding of the definition's own fp32 product: the same integer as clamp(Round(float(sum) * fp32(1/9)))
+    // for every possible window sum (checked exhaustively on the host in the tests).
+    const unsigned int adj = kSigned ? (unsigned int)(128 * (9 - (r0.cells + r1.cells + r2.cells))) * 0x00010001u : 0u;
+    const float c = kSigned ? (12582912.0f - 1048576.0f - 128.0f) : (12582912.0f - 1048576.0f);
+    constexpr float kInv9 = 1.0f / 9.0f;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const unsigned int e = r0.a[j] + r1.a[j] + r2.a[j], o = r0.b[j] + r1.b[j] + r2.b[j];
-      // (scalar on purpose: the packed f32x2 forms of these operations made this kernel slower, measured)
-      const float f0 = __fsub_rn(__uint_as_float(__byte_perm(e, 0x4B000000u, 0x7610u)), off);
-      const float f1 = __fsub_rn(__uint_as_float(__byte_perm(o, 0x4B000000u, 0x7610u)), off);
-      const float f2 = __fsub_rn(__uint_as_float(__byte_perm(e, 0x4B000000u, 0x7632u)), off);
-      const float f3 = __fsub_rn(__uint_as_float(__byte_perm(o, 0x4B000000u, 0x7632u)), off);
-      // Round half even: adding 1.5 * 2^23 leaves the rounded integer in the low mantissa bits (two's complement)
-      const unsigned int z0 = __float_as_uint(__fadd_rn(__fmul_rn(f0, inv), 12582912.0f));
-      const unsigned int z1 = __float_as_uint(__fadd_rn(__fmul_rn(f1, inv), 12582912.0f));
-      const unsigned int z2 = __float_as_uint(__fadd_rn(__fmul_rn(f2, inv), 12582912.0f));
-      const unsigned int z3 = __float_as_uint(__fadd_rn(__fmul_rn(f3, inv), 12582912.0f));
+      const unsigned int e = r0.a[j] + r1.a[j] + r2.a[j] + adj, o = r0.b[j] + r1.b[j] + r2.b[j] + adj;
+      const unsigned int z0 = __float_as_uint(__fmaf_rn(__uint_as_float(__byte_perm(e, 0x4B100000u, 0x7610u)), kInv9, c));
+      const unsigned int z1 = __float_as_uint(__fmaf_rn(__uint_as_float(__byte_perm(o, 0x4B100000u, 0x7610u)), kInv9, c));
+      const unsigned int z2 = __float_as_uint(__fmaf_rn(__uint_as_float(__byte_perm(e, 0x4B100000u, 0x7632u)), kInv9, c));
+      const unsigned int z3 = __float_as_uint(__fmaf_rn(__uint_as_float(__byte_perm(o, 0x4B100000u, 0x7632u)), kInv9, c));
       out[j] = __byte_perm(__byte_perm(z0, z1, 0x0040u), __byte_perm(z2, z3, 0x0040u), 0x5410u);
     }
   }
   return make_uint4(out[0], out[1], out[2], out[3]);
 }
 
-// Lanes of one input pixel (average) or the pixel itself (max); outside the image: the identity of the reduction.
+// Lanes of one input pixel; outside the image: zero, the identity of both reductions.
 template <bool kSigned, bool kAvg>
 __device__ __forceinline__ PoolRow pool_pixel(const uint4* __restrict__ row, int w, int W, int cg, bool row_ok) {
   PoolRow r;
-  const unsigned int init = (!kAvg && kSigned) ? 0x80808080u : 0u;
+  const unsigned int flip = kSigned ? 0x80808080u : 0u;
   const bool ok = row_ok && w >= 0 && w < W;
-  const uint4 v = ok ? __ldg(row + (size_t)w * cg) : make_uint4(init, init, init, init);
+  const uint4 v = ok ? __ldg(row + (size_t)w * cg) : make_uint4(flip, flip, flip, flip);
   const unsigned int word[4] = {v.x, v.y, v.z, v.w};
   r.cells = ok ? 1 : 0;
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    if (!kAvg) { r.a[j] = word[j]; r.b[j] = 0u; }
-    else {
-      const unsigned int wj = ok ? (word[j] ^ (kSigned ? 0x80808080u : 0u)) : 0u;
-      r.a[j] = wj & 0x00ff00ffu;
-      r.b[j] = __byte_perm(wj, 0u, 0x4341u);
-    }
+    const unsigned int wj = word[j] ^ flip;
+    r.a[j] = wj & 0x00ff00ffu;
+    r.b[j] = __byte_perm(wj, 0u, 0x4341u);
   }
   return r;
 }
@@ -833,7 +843,7 @@ __device__ __forceinline__ PoolRow pool_join(const PoolRow& x, const PoolRow& y)
   PoolRow r;
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    if (!kAvg) { r.a[j] = kSigned ? __vmaxs4(x.a[j], y.a[j]) : __vmaxu4(x.a[j], y.a[j]); r.b[j] = 0u; }
+    if (!kAvg) { r.a[j] = max_u16x2(x.a[j], y.a[j]); r.b[j] = max_u16x2(x.b[j], y.b[j]); }
     else { r.a[j] = x.a[j] + y.a[j]; r.b[j] = x.b[j] + y.b[j]; }
   }
   r.cells = x.cells + y.cells;
@@ -878,8 +888,8 @@ __global__ void __launch_bounds__(256) pool3_strip2_kernel(const uint4* __restri
 #pragma unroll 1
     for (int p = p0; p < p1; ++p, ++h, out += (size_t)Q * cg) {
       load_row(h + 2, ra[2], rb[2]);
-      out[0] = pool_combine3<kSigned, kAvg>(ra[0], ra[1], ra[2], inv);
-      if (two) out[cg] = pool_combine3<kSigned, kAvg>(rb[0], rb[1], rb[2], inv);
+      out[0] = pool_combine3<kSigned, kAvg>(ra[0], ra[1], ra[2]);
+      if (two) out[cg] = pool_combine3<kSigned, kAvg>(rb[0], rb[1], rb[2]);
       ra[0] = ra[1]; ra[1] = ra[2];
       rb[0] = rb[1]; rb[1] = rb[2];
     }
@@ -907,7 +917,7 @@ __global__ void __launch_bounds__(256) pool3_strip_kernel(const uint4* __restric
     PoolRow r1 = pool_row3<kSigned, kAvg>(img, h + 1, H, W, cg, w0);
     for (int p = p0; p < p1; ++p, h += kStride, out += (size_t)Q * cg) {
       const PoolRow r2 = pool_row3<kSigned, kAvg>(img, h + 2, H, W, cg, w0);
-      *out = pool_combine3<kSigned, kAvg>(r0, r1, r2, inv);
+      *out = pool_combine3<kSigned, kAvg>(r0, r1, r2);
       if (kStride == 1) {
         r0 = r1;
         r1 = r2;

@@ -396,3 +396,34 @@ def test_dequantize_is_one_fp32_product():
         assert min(near, key=lambda c: abs(Fraction(c) - exact)) == float(v)
     big = o.dequantize(np.array([2 ** 30 + 12345, -(2 ** 31)], dtype=np.int32), 0.5)    # int32 -> fp32 rounds first
     assert big[0] == np.float32(2 ** 30 + 12345) * np.float32(0.5) and big[1] == -(2.0 ** 30)
+
+
+def test_avgpool_3x3_is_nearest_integer_division_for_every_window_sum():
+    """A 3x3 window sum n is never half-way between multiples of 9, so clamp(Round(float(n) * fp32(1/9))) must be
+    the integer nearest to n / 9 (Python integers decide) for every sum a window of u8 or s8 codes can have.  The
+    images hold one window each, chosen so that all sums 0..2295 and -1152..1143 occur."""
+    for dt, lo, hi in ((np.uint8, 0, 255), (np.int8, -128, 127)):
+        sums = np.arange(9 * lo, 9 * hi + 1)
+        base, extra = np.divmod(sums - 9 * lo, 9)                     # nine cells: base each, `extra` of them one more
+        cells = lo + base[:, None] + (np.arange(9)[None, :] < extra[:, None])
+        assert np.array_equal(cells.sum(1), sums) and cells.min() >= lo and cells.max() <= hi
+        x = cells.astype(dt).reshape(-1, 3, 3, 1)
+        got = o.pool(x, "avg", (3, 3), (1, 1), (0, 0)).reshape(-1).astype(np.int64)
+        want = np.array([(2 * int(n) + 9) // 18 for n in sums])       # floor(n/9 + 1/2); no ties exist
+        assert np.array_equal(got, want)
+
+
+def test_single_fused_multiply_add_form_of_the_3x3_average():
+    """Host check of the arithmetic the strip pooling kernels use: with B = 9 * 2^20, fma(float(B + n), fp32(1/9),
+    1.5 * 2^23 - 2^20) rounds once at unit spacing and leaves Round(n / 9) in the low mantissa bits.  The fused
+    operation is evaluated exactly here (a 24 x 24 bit product fits a double; the sum with an integer below 2^24 is
+    then rounded half to even to an integer), for every n a window can produce (signed sums shifted by 9 * 128)."""
+    inv = np.float32(1.0) / np.float32(9.0)
+    B = 9 * 2 ** 20
+    for n in range(0, 9 * 255 + 1):
+        x = np.float32(B + n)
+        assert int(x) == B + n                                        # representable: below 2^24
+        exact = float(np.float64(x) * np.float64(inv))                # exact product
+        assert 2 ** 23 <= exact + (1.5 * 2 ** 23 - 2 ** 20) < 2 ** 24 # the sum lands where fp32 spacing is 1
+        z = int(np.rint(exact)) - 2 ** 20                             # the integer constant only shifts the result
+        assert z == (2 * n + 9) // 18
