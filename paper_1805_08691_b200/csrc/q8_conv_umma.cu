@@ -749,6 +749,13 @@ int launch_conv_umma_plan(const ConvArgs& a, int splits, int bk_cap, bool allow_
   const int BK = pick_bk(c_eff) < bk_cap ? pick_bk(c_eff) : bk_cap;
   int BN = pick_bn(d.K, d.R * d.S * d.C);
   {
+    // Few output tiles (small images with many channels): 128-wide tiles run the tensor pipe at the same rate
+    // per column as 256-wide ones, and twice as many CTAs get work.
+    const long long m_tiles = p.a_mode == kAHalo ? (long long)d.N * ((a.P + ht.th - 1) / ht.th) * ((a.Q + ht.tw - 1) / ht.tw)
+                                                 : (a.M + kBM - 1) / kBM;
+    if (splits == 1 && BN == 256 && d.K % 256 == 0 && m_tiles * (d.K / 256) * 2 <= sm_count()) BN = 128;
+  }
+  {
     const int want = tune_env("Q8_BN", BN, 16, 256);
     if (want % 16 == 0) BN = want;
   }
