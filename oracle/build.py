@@ -7,15 +7,15 @@ import os
 import subprocess
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-SRC = os.path.join(HERE, "q8_oracle.cpp")
+SRCS = [os.path.join(HERE, "q8_oracle.cpp"), os.path.join(HERE, "q8_oracle_detect.cpp")]
 LIB = os.path.join(HERE, "libq8_oracle.so")
 
 
 def build(force: bool = False) -> str:
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= os.path.getmtime(SRC):
+    if not force and os.path.exists(LIB) and all(os.path.getmtime(LIB) >= os.path.getmtime(s) for s in SRCS):
         return LIB
     cmd = ["g++", "-std=c++17", "-O2", "-ffp-contract=off", "-fno-fast-math", "-shared", "-fPIC",
-           "-pthread", SRC, "-o", LIB]
+           "-pthread", *SRCS, "-o", LIB]
     subprocess.run(cmd, check=True)
     return LIB
 

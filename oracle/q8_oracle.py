@@ -226,3 +226,86 @@ def pool(x, kind, k, stride, pad=(0, 0), ceil_mode=False):
                   k[0], k[1], stride[0], stride[1], pad[0], pad[1], int(ceil_mode),
                   _ptr(y.view(np.uint8), _u8p))
     return y
+
+
+# ------------------------------------------------------------------ SSD tail (oracle/q8_oracle_detect.cpp)
+_lib.q8o_l2norm_mult.restype = C.c_float
+_lib.q8o_l2norm_mult.argtypes = [C.c_float] * 3
+_lib.q8o_l2norm.restype = None
+_lib.q8o_l2norm.argtypes = [_u8p, C.c_size_t, C.c_int, C.c_float, C.c_float, _f32p, _u8p]
+_lib.q8o_exp.restype = C.c_float
+_lib.q8o_exp.argtypes = [C.c_float]
+_lib.q8o_softmax.restype = None
+_lib.q8o_softmax.argtypes = [_f32p, C.c_size_t, C.c_int, _f32p]
+_lib.q8o_decode_boxes.restype = None
+_lib.q8o_decode_boxes.argtypes = [_f32p, _f32p, _f32p, C.c_int, C.c_int, _f32p]
+_lib.q8o_iou.restype = C.c_float
+_lib.q8o_iou.argtypes = [_f32p, _f32p]
+_lib.q8o_detection_output.restype = None
+_lib.q8o_detection_output.argtypes = [_f32p, _f32p, _f32p, _f32p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_float,
+                                      C.c_float, C.c_int, C.c_int, _f32p, _i32p]
+_lib.q8o_add_relu_quantize.restype = None
+_lib.q8o_add_relu_quantize.argtypes = [_f32p, _f32p, C.c_size_t, C.c_float, _u8p]
+
+
+def l2norm_mult(gamma, qx, qy):
+    """Per-channel multipliers gamma_c q_x / q_y of the L2 normalisation layer."""
+    return np.array([_lib.q8o_l2norm_mult(np.float32(g), np.float32(qx), np.float32(qy)) for g in np.ravel(gamma)],
+                    dtype=np.float32)
+
+
+def l2norm(x, qx, eps, mult):
+    """x: [..., C] uint8 codes with factor qx; mult: [C] from l2norm_mult.  Returns uint8 codes with factor qy."""
+    x = np.ascontiguousarray(x, dtype=np.uint8)
+    m = _f32(mult)
+    y = np.empty_like(x)
+    _lib.q8o_l2norm(_ptr(x, _u8p), x.size // x.shape[-1], x.shape[-1], np.float32(qx), np.float32(eps), _ptr(m, _f32p),
+                    _ptr(y, _u8p))
+    return y
+
+
+def exp(x):
+    x = _f32(x)
+    return np.array([_lib.q8o_exp(v) for v in x.ravel()], dtype=np.float32).reshape(x.shape)
+
+
+def softmax(conf):
+    """conf: [..., classes] fp32 logits."""
+    conf = _f32(conf)
+    p = np.empty_like(conf)
+    _lib.q8o_softmax(_ptr(conf, _f32p), conf.size // conf.shape[-1], conf.shape[-1], _ptr(p, _f32p))
+    return p
+
+
+def decode_boxes(loc, priors, var):
+    """loc [N, P, 4], priors [P, 4] (cx, cy, w, h), var [4] -> corner boxes [N, P, 4]."""
+    loc, priors, var = _f32(loc), _f32(priors), _f32(var)
+    b = np.empty_like(loc)
+    _lib.q8o_decode_boxes(_ptr(loc, _f32p), _ptr(priors, _f32p), _ptr(var, _f32p), loc.shape[0], loc.shape[1], _ptr(b, _f32p))
+    return b
+
+
+def iou(a, b):
+    a, b = _f32(a), _f32(b)
+    return float(_lib.q8o_iou(_ptr(a, _f32p), _ptr(b, _f32p)))
+
+
+def detection_output(loc, conf, priors, var, background=0, conf_thresh=0.01, nms_thresh=0.45, nms_top_k=400,
+                     keep_top_k=200):
+    """loc [N, P, 4], conf [N, P, classes] logits.  Returns (rows [N, keep_top_k, 6], counts [N])."""
+    loc, conf, priors, var = _f32(loc), _f32(conf), _f32(priors), _f32(var)
+    N, P, classes = conf.shape
+    out = np.empty((N, keep_top_k, 6), dtype=np.float32)
+    counts = np.empty(N, dtype=np.int32)
+    _lib.q8o_detection_output(_ptr(loc, _f32p), _ptr(conf, _f32p), _ptr(priors, _f32p), _ptr(var, _f32p), N, P, classes,
+                              background, np.float32(conf_thresh), np.float32(nms_thresh), nms_top_k, keep_top_k,
+                              _ptr(out, _f32p), _ptr(counts, _i32p))
+    return out, counts
+
+
+def add_relu_quantize(a, b, qy):
+    """The FP32 route for a residual sum with a signed summand: Q_8(max(a + b, 0), q_y) as uint8."""
+    a, b = _f32(a), _f32(b)
+    y = np.empty(a.shape, dtype=np.uint8)
+    _lib.q8o_add_relu_quantize(_ptr(a, _f32p), _ptr(b, _f32p), a.size, np.float32(qy), _ptr(y, _u8p))
+    return y

@@ -285,3 +285,45 @@ def macs(layers: List[Layer], hw: int) -> int:
             P, Q = H, W
         size[L.name] = (P, Q)
     return total
+
+
+# SSD-300 prior boxes (inputs of the detection output step, fixed by the detector's published configuration, not by
+# the quantization method): six source maps, per cell one box of the minimum size, one of sqrt(min * max), and two
+# per extra aspect ratio; centres at (cell + 0.5) * step / 300.
+SSD300_MAPS = (38, 19, 10, 5, 3, 1)
+SSD300_STEPS = (8, 16, 32, 64, 100, 300)
+SSD300_MIN = (30, 60, 111, 162, 213, 264)
+SSD300_MAX = (60, 111, 162, 213, 264, 315)
+SSD300_RATIOS = ((2,), (2, 3), (2, 3), (2, 3), (2,), (2,))
+SSD300_VARIANCES = (0.1, 0.1, 0.2, 0.2)
+
+
+def ssd300_priors() -> np.ndarray:
+    """[8732, 4] fp32 (cx, cy, w, h) in units of the image side, in the order of the head outputs: source map,
+    row, column, box."""
+    rows = []
+    for fm, step, smin, smax, ratios in zip(SSD300_MAPS, SSD300_STEPS, SSD300_MIN, SSD300_MAX, SSD300_RATIOS):
+        sizes = [(smin / 300.0, smin / 300.0), ((smin * smax) ** 0.5 / 300.0,) * 2]
+        for r in ratios:
+            sizes.append((smin / 300.0 * r ** 0.5, smin / 300.0 / r ** 0.5))
+            sizes.append((smin / 300.0 / r ** 0.5, smin / 300.0 * r ** 0.5))
+        for i in range(fm):
+            for j in range(fm):
+                cx, cy = (j + 0.5) * step / 300.0, (i + 0.5) * step / 300.0
+                rows.extend((cx, cy, w, h) for w, h in sizes)
+    return np.asarray(rows, dtype=np.float32)
+
+
+def detection_inputs(seed: int, batch: int, priors: int = 8732, classes: int = 21, peaked: float = 0.02):
+    """Seeded stand-ins for the head outputs of a detector: localisation offsets N(0, 1) and class logits N(0, 1)
+    with a fraction `peaked` of the boxes given one strongly preferred class (confident detections), the rest
+    mostly background.  Returns (loc [N, P, 4], conf [N, P, classes])."""
+    g = rng(seed)
+    loc = normal(g, (batch, priors, 4))
+    conf = normal(g, (batch, priors, classes))
+    conf[..., 0] += 4.0                                         # background dominates, as in a trained detector
+    hot = g.random((batch, priors)) < peaked
+    cls = g.integers(1, classes, (batch, priors))
+    n_idx, p_idx = np.nonzero(hot)
+    conf[n_idx, p_idx, cls[n_idx, p_idx]] += g.uniform(4.0, 9.0, n_idx.size).astype(np.float32)
+    return loc.astype(np.float32), conf.astype(np.float32)
