@@ -297,6 +297,57 @@ int q8_maxpool2d(const void* x, int t, int N, int H, int W, int C, int kh, int k
 int q8_avgpool2d(const void* x, int t, int N, int H, int W, int C, int kh, int kw, int stride_h,
                  int stride_w, int pad_h, int pad_w, int ceil_mode, void* y, void* stream);
 
+/* ------------------------------------------------------------------------
+ * The SSD tail and the FP32 route for signed sums.  The paper runs SSD with a detection-output layer
+ * (artifact appendix) and sends potentially negative activations through FP32 (Sec. "8-bit Low Precision
+ * Inference", calibration paragraph) but prints no arithmetic for them; these calls follow the detector's
+ * published definition with every floating-point step one IEEE fp32 operation in a fixed order.
+ * ---------------------------------------------------------------------- */
+
+/* L2 normalisation across the channels of each pixel, on unsigned 8-bit codes:
+ *   S = sum_c z_c^2 (integer),  d = sqrt(float(S) * (qx * qx) + eps),
+ *   y_c = clamp(Round((float(z_c) * mult[c]) / d), 0, 255),   mult[c] = gamma_c qx / qy (formed by the caller).
+ * x, y: device [pixels][C] u8 (may not overlap); d_mult: device [C] fp32.  The fast path needs C % 4 == 0,
+ * x and y 4-byte aligned and d_mult 16-byte aligned; anything else takes a scalar kernel.  0 / 0 (an all-zero
+ * pixel with eps == 0) gives code 0.  Asynchronous on `stream`.
+ * Errors: Q8_ERR_INVALID_ARG (null pointer, C outside 1..65536), Q8_ERR_NONFINITE (qx not finite positive, eps
+ * negative or not finite), Q8_ERR_CUDA. */
+int q8_l2norm(const void* x, size_t pixels, int C, float qx, float eps, const float* d_mult, void* y, void* stream);
+
+/* The FP32 route of a residual sum whose summands may be negative: a and b are dequantized (fp32) convolution
+ * outputs, y = clamp(Round(max(a + b, 0) / q), 0, 255) as u8 (one fp32 add, one IEEE division, Round half to even).
+ * a, b: device fp32 [n]; y: device u8 [n].  Vector path when a, b are 16-byte and y 4-byte aligned.
+ * Errors: Q8_ERR_INVALID_ARG, Q8_ERR_NONFINITE (q not finite positive), Q8_ERR_CUDA. */
+int q8_add_relu_quantize(const float* a, const float* b, size_t n, float q, void* y, void* stream);
+
+/* Detection output for a batch of N images.
+ * Inputs: n_sources (<= 8) head tensors.  Source i has cells[i] cells per image and boxes_per_cell[i] boxes per
+ * cell; its localisation values for image n, cell k, box b are the four floats at
+ * loc[i] + (n * cells[i] + k) * loc_stride[i] + 4 b, its class logits the `classes` floats at
+ * conf[i] + (n * cells[i] + k) * conf_stride[i] + classes * b (strides in floats; device pointers in HOST arrays;
+ * a merged head passes the same base twice with an offset).  Boxes are numbered source by source, cell by cell, box
+ * by box: P = sum cells * boxes_per_cell in all.  d_priors: device [P][4] fp32 (centre x, centre y, width, height),
+ * 16-byte aligned.  variances: HOST [4].
+ * Steps: corners = decode(loc, prior, variances) (centre-size code, exp by a fixed fp32 recipe, no clipping);
+ * probabilities = softmax(logits); per image and class other than `background` (-1: none): boxes with probability
+ * > conf_thresh, best nms_top_k by probability (ties: lower box index), greedy suppression of boxes whose overlap
+ * (intersection over union) with a kept box exceeds nms_thresh; per image the best keep_top_k of all kept (ties:
+ * lower class, lower box index).
+ * Outputs: d_out device [N][keep_top_k][6] fp32 rows (class, probability, xmin, ymin, xmax, ymax), best first, rows
+ * beyond the count zero; d_counts device [N] int32.
+ * workspace: device, 256-byte aligned, q8_detection_output_workspace_bytes(...) bytes, caller-owned; three kernels
+ * are enqueued on `stream`, nothing is allocated.
+ * Limits: P <= 16384, nms_top_k <= 512, (foreground classes) * nms_top_k <= 16384, N <= 65535.
+ * Errors: Q8_ERR_INVALID_ARG, Q8_ERR_UNSUPPORTED (a limit), Q8_ERR_NONFINITE (thresholds), Q8_ERR_ALIGNMENT,
+ * Q8_ERR_WORKSPACE, Q8_ERR_CUDA.  Nothing is launched on error. */
+int q8_detection_output_workspace_bytes(int N, int P, int classes, int background, int nms_top_k, int keep_top_k,
+                                        size_t* bytes);
+int q8_detection_output(int n_sources, const float* const* loc, const int* loc_stride, const float* const* conf,
+                        const int* conf_stride, const int* cells, const int* boxes_per_cell, const float* d_priors,
+                        const float* variances, int N, int classes, int background, float conf_thresh,
+                        float nms_thresh, int nms_top_k, int keep_top_k, void* workspace, size_t workspace_bytes,
+                        float* d_out, int* d_counts, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

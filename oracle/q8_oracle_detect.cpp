@@ -43,8 +43,8 @@ void q8o_l2norm(const uint8_t* x, size_t pixels, int C, float qx, float eps, con
     const float d = std::sqrt(t + eps);
     for (int c = 0; c < C; ++c) {
       const float num = (float)xp[c] * mult[c];
-      const float r = std::nearbyintf(num / d);
-      y[p * (size_t)C + c] = (uint8_t)(r < 0.0f ? 0.0f : (r > 255.0f ? 255.0f : r));
+      const float r = std::nearbyintf(num / d);   // 0 / 0 (an all-zero pixel with eps = 0) gives NaN, which maps to 0
+      y[p * (size_t)C + c] = (uint8_t)(!(r > 0.0f) ? 0.0f : (r > 255.0f ? 255.0f : r));
     }
   }
 }

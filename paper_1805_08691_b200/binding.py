@@ -22,7 +22,8 @@ EXPORTS = ["q8_version", "q8_last_error", "q8_read_status", "q8_calibrate_maxabs
            "q8_bias_factor", "q8_quantize", "q8_quantize_pad_channels", "q8_dequantize", "q8_fold_bn",
            "q8_conv2d_workspace_bytes", "q8_conv2d_query_algo", "q8_conv2d", "q8_static_workspace_bytes",
            "q8_conv2d_static_workspace", "q8_conv2d_then_1x1_supported", "q8_conv2d_then_1x1", "q8_int8_mma_rate", "q8_selftest_bounded_wait", "q8_concat", "q8_concat_branch", "q8_calibrate_maxabs_rows", "q8_quantize_rows", "q8_quantize_pad_image", "q8_pool_out_extent",
-           "q8_maxpool2d", "q8_avgpool2d"]
+           "q8_maxpool2d", "q8_avgpool2d", "q8_l2norm", "q8_add_relu_quantize", "q8_detection_output_workspace_bytes",
+           "q8_detection_output"]
 
 
 class Q8Error(RuntimeError):
@@ -79,6 +80,11 @@ lib.q8_concat_branch.argtypes = [_vp, _i, _f, _f, _i, _sz, _vp, _i, _i, _vp]
 lib.q8_pool_out_extent.argtypes = [_i] * 5 + [_ip]
 lib.q8_maxpool2d.argtypes = [_vp, _i] + [_i] * 11 + [_vp, _vp]
 lib.q8_avgpool2d.argtypes = [_vp, _i] + [_i] * 11 + [_vp, _vp]
+lib.q8_l2norm.argtypes = [_vp, _sz, _i, _f, _f, _vp, _vp, _vp]
+lib.q8_add_relu_quantize.argtypes = [_vp, _vp, _sz, _f, _vp, _vp]
+lib.q8_detection_output_workspace_bytes.argtypes = [_i] * 6 + [C.POINTER(_sz)]
+lib.q8_detection_output.argtypes = [_i, C.POINTER(_vp), _ip, C.POINTER(_vp), _ip, _ip, _ip, _vp, _fp, _i, _i, _i, _f, _f, _i, _i,
+                                    _vp, _sz, _vp, _vp, _vp]
 for _n in EXPORTS[2:]:
     getattr(lib, _n).restype = C.c_int
 lib.q8_static_workspace_bytes.restype = C.c_size_t
@@ -323,3 +329,61 @@ def q8_maxpool2d(x, k, stride, pad=(0, 0), ceil_mode=False, out=None):
 
 def q8_avgpool2d(x, k, stride, pad=(0, 0), ceil_mode=False, out=None):
     return _pool(lib.q8_avgpool2d, x, k, stride, pad, ceil_mode, out)
+
+
+def q8_l2norm(x, qx, eps, mult, out=None):
+    """L2 normalisation across the last dimension of a u8 tensor; mult: CUDA fp32 [C] = gamma qx / qy."""
+    Cc = int(x.shape[-1])
+    if out is None:
+        out = torch.empty_like(x)
+    _check(lib.q8_l2norm(_dev(x, "x"), x.numel() // Cc, Cc, qx, eps, _dev(mult, "mult"), _dev(out, "out"), _stream()))
+    return out
+
+
+def q8_add_relu_quantize(a, b, q, out=None):
+    """Q_8(max(a + b, 0), q) of two fp32 tensors as u8 (the FP32 route of a residual sum)."""
+    if out is None:
+        out = torch.empty(a.shape, dtype=torch.uint8, device=a.device)
+    _check(lib.q8_add_relu_quantize(_dev(a, "a"), _dev(b, "b"), a.numel(), q, _dev(out, "out"), _stream()))
+    return out
+
+
+def q8_detection_output_workspace_bytes(N, P, classes, background, nms_top_k, keep_top_k):
+    n = C.c_size_t()
+    _check(lib.q8_detection_output_workspace_bytes(N, P, classes, background, nms_top_k, keep_top_k, C.byref(n)))
+    return n.value
+
+
+def q8_detection_output(sources, priors, variances, classes, background=0, conf_thresh=0.01, nms_thresh=0.45,
+                        nms_top_k=400, keep_top_k=200, workspace=None, out=None, counts=None):
+    """sources: list of (loc, conf, boxes_per_cell) with loc [N, cells..., >= boxes*4] and conf [N, cells...,
+    >= boxes*classes] contiguous CUDA fp32 tensors (the last dimension is the cell stride), or of
+    (loc, conf, boxes_per_cell, loc_offset, conf_offset) where both views start that many floats into a cell of a
+    shared tensor.  priors: CUDA fp32 [P, 4].  Returns (rows [N, keep_top_k, 6], counts [N])."""
+    N = int(sources[0][0].shape[0])
+    n = len(sources)
+    locp, confp = (C.c_void_p * n)(), (C.c_void_p * n)()
+    lstr, cstr, cells, boxes = (C.c_int * n)(), (C.c_int * n)(), (C.c_int * n)(), (C.c_int * n)()
+    P = 0
+    for i, src in enumerate(sources):
+        loc, conf, b = src[0], src[1], int(src[2])
+        lo, co = (int(src[3]), int(src[4])) if len(src) > 3 else (0, 0)
+        _dev(loc, "loc"), _dev(conf, "conf")
+        locp[i], confp[i] = loc.data_ptr() + 4 * lo, conf.data_ptr() + 4 * co
+        lstr[i], cstr[i] = int(loc.shape[-1]), int(conf.shape[-1])
+        cells[i] = loc.numel() // (N * int(loc.shape[-1]))
+        boxes[i] = b
+        P += cells[i] * b
+    dev = sources[0][0].device
+    nbytes = q8_detection_output_workspace_bytes(N, P, classes, background, nms_top_k, keep_top_k)
+    if workspace is None:
+        workspace = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    if out is None:
+        out = torch.empty((N, keep_top_k, 6), dtype=torch.float32, device=dev)
+    if counts is None:
+        counts = torch.empty(N, dtype=torch.int32, device=dev)
+    var = (C.c_float * 4)(*[float(v) for v in variances])
+    _check(lib.q8_detection_output(n, locp, lstr, confp, cstr, cells, boxes, _dev(priors, "priors"), var, N, classes, background,
+                                   conf_thresh, nms_thresh, nms_top_k, keep_top_k, _dev(workspace, "workspace"), workspace.numel(),
+                                   _dev(out, "out"), _dev(counts, "counts"), _stream()))
+    return out, counts

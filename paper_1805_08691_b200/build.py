@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libq8.so")
-SOURCES = ["q8_api.cu", "q8_elementwise.cu", "q8_conv_direct.cu", "q8_conv_splitk.cu", "q8_conv_static.cu", "q8_conv_umma.cu", "q8_conv_fused.cu", "q8_mma_rate.cu", "q8_selftest.cu"]
+SOURCES = ["q8_api.cu", "q8_elementwise.cu", "q8_conv_direct.cu", "q8_conv_splitk.cu", "q8_conv_static.cu", "q8_conv_umma.cu", "q8_conv_fused.cu", "q8_mma_rate.cu", "q8_selftest.cu", "q8_detect.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-fmad=false",
          "-Xcompiler", "-fPIC,-ffp-contract=off,-fno-fast-math", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 
