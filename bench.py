@@ -22,7 +22,9 @@ between the two layers stays in shared memory).  Prints ONE JSON line (rank 0).
                its roofline max(2 MACs / int8 peak, bytes / copy bandwidth).
 * bandwidth_kernels: the memory-bound kernels (max-abs, quantize, dequantize, concat, pooling) against the measured
                copy bandwidth; networks: int8 forward of ResNet-50, Inception-v3 and SSD-300 (images/s), with the
-               paper's Xeon figures beside them as context.  Both only at N = 1; --skip-networks leaves them out.
+               paper's Xeon figures beside them as context.  ssd_tail: L2 normalisation, detection output, and the
+               projection blocks of ResNet-50 through the int8 route and through the paper's FP32 route for signed
+               tensors.  All only at N = 1; --skip-networks leaves them out.
 * --impl reference: the oracle alone (there is no reference implementation to install for this paper).
 With N > 1 every rank runs its own batch (weak scaling, replicated weights, no data-path collective).
 """
@@ -746,6 +748,7 @@ def run_ours(args):
     if world == 1 and not args.skip_networks:
         line["bandwidth_kernels"] = bandwidth_kernel_numbers(dev, peaks["hbm_gbs"])
         line["resnet50_layers"] = resnet50_layer_table(dev, peaks["hbm_gbs"], int8_peak)
+        line["ssd_tail"] = ssd_tail_numbers(dev, peaks["hbm_gbs"])
         line["networks"] = {name: network_numbers(dev, name) for name in NETWORKS}
     if world == 1 and not args.skip_cpu_baseline:
         r = oracle_time_steps(steps=2, warmup=1)
@@ -754,6 +757,101 @@ def run_ours(args):
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def ssd_tail_numbers(dev, peak_gbs, reps=20):
+    """The SSD tail and the FP32 route (all at N = 1, CUDA-event times of back-to-back launches):
+    * l2norm: L2 normalisation of a conv4_3-shaped tensor (128 x 38 x 38 x 512 u8, in + out larger than L2) against
+      the measured copy bandwidth;
+    * detection_output: 8732 boxes x 21 classes per image at batch 32, seeded head outputs (2 % confident boxes);
+    * fp32_route: the four projection blocks of ResNet-50 at batch 64, the shortcut convolution (no ReLU, signed
+      output) and the block's last 1x1 convolution, (a) as the library runs them: s8 shortcut, residual sum fused
+      into the last convolution's epilogue; (b) the paper's FP32 route for signed tensors: both convolutions write
+      fp32, one more kernel adds, applies the ReLU and quantizes."""
+    import torch
+    import paper_1805_08691_b200 as q8
+    from workloads import nets
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps * 1e-3
+
+    g = torch.Generator(device=dev).manual_seed(0)
+
+    def rnd(shape, lo=0, hi=256, dt=torch.uint8):
+        return torch.randint(lo, hi, shape, dtype=dt, device=dev, generator=g)
+
+    out = {}
+    x = rnd((128, 38, 38, 512))
+    y = torch.empty_like(x)
+    mult = torch.full((512,), 20.0 * 0.03 / 0.08, device=dev)
+    t = timed(lambda: q8.q8_l2norm(x, 0.03, 1e-10, mult, out=y))
+    out["l2norm"] = {"us": t * 1e6, "GB/s": 2 * x.numel() / t / 1e9, "frac": 2 * x.numel() / t / 1e9 / peak_gbs}
+    del x, y
+    N = 32
+    loc_np, conf_np = nets.detection_inputs(77, N)
+    priors = torch.from_numpy(nets.ssd300_priors()).to(dev)
+    loc, conf = torch.from_numpy(loc_np).to(dev), torch.from_numpy(conf_np).to(dev)
+    ws = torch.empty(q8.q8_detection_output_workspace_bytes(N, 8732, 21, 0, 400, 200), dtype=torch.uint8, device=dev)
+    rows = torch.empty((N, 200, 6), device=dev)
+    counts = torch.empty(N, dtype=torch.int32, device=dev)
+    src = [(loc, conf, 1)]
+    t = timed(lambda: q8.q8_detection_output(src, priors, nets.SSD300_VARIANCES, 21, workspace=ws, out=rows, counts=counts))
+    out["detection_output"] = {"batch": N, "us": t * 1e6, "images_per_s": N / t, "detections_per_image": float(counts.float().mean()),
+                               "launches": 3}
+    # the worst case for the per-class sort: flat logits, every box a candidate of every class
+    gen = np.random.default_rng(78)
+    conf = torch.from_numpy(gen.normal(0, 0.3, (N, 8732, 21)).astype(np.float32)).to(dev)
+    src = [(loc, conf, 1)]
+    t = timed(lambda: q8.q8_detection_output(src, priors, nets.SSD300_VARIANCES, 21, workspace=ws, out=rows, counts=counts))
+    out["detection_output_every_box_a_candidate"] = {"batch": N, "us": t * 1e6, "images_per_s": N / t}
+    del loc, conf, ws
+    blocks = {}
+    B = 64
+    for name, (H, Cin, Cmid, K, st) in {"res2a": (56, 64, 64, 256, 1), "res3a": (56, 256, 128, 512, 2), "res4a": (28, 512, 256, 1024, 2),
+                                        "res5a": (14, 1024, 512, 2048, 2)}.items():
+        Ho = H // st
+        xin, xmid = rnd((B, H, H, Cin)), rnd((B, Ho, Ho, Cmid))
+        w1, w2 = rnd((K, 1, 1, Cin), -128, 128, torch.int8), rnd((K, 1, 1, Cmid), -128, 128, torch.int8)
+        b1, b2 = rnd((K,), -1000, 1000, torch.int32), rnd((K,), -1000, 1000, torch.int32)
+        s = torch.tensor([1e-4], device=dev)
+        U8, S8, F32 = q8.Q8_U8, q8.Q8_S8, q8.Q8_F32
+        d1s = q8.make_conv_desc(B, H, H, Cin, K, 1, 1, (st, st), (0, 0), (1, 1), U8, U8, S8, False)
+        d2s = q8.make_conv_desc(B, Ho, Ho, Cmid, K, 1, 1, (1, 1), (0, 0), (1, 1), U8, S8, U8, True)
+        d1f = q8.make_conv_desc(B, H, H, Cin, K, 1, 1, (st, st), (0, 0), (1, 1), U8, U8, F32, False)
+        d2f = q8.make_conv_desc(B, Ho, Ho, Cmid, K, 1, 1, (1, 1), (0, 0), (1, 1), U8, U8, F32, False)
+        sc = torch.empty((B, Ho, Ho, K), dtype=torch.int8, device=dev)
+        yo = torch.empty((B, Ho, Ho, K), dtype=torch.uint8, device=dev)
+        fa, fb = torch.empty((B, Ho, Ho, K), device=dev), torch.empty((B, Ho, Ho, K), device=dev)
+
+        def int8_route():
+            q8.q8_conv2d(d1s, xin, w1, b1, s, None, 0.0, sc)
+            q8.q8_conv2d(d2s, xmid, w2, b2, s, sc, 0.5, yo)
+
+        def fp32_route():
+            q8.q8_conv2d(d1f, xin, w1, b1, s, None, 0.0, fa)
+            q8.q8_conv2d(d2f, xmid, w2, b2, s, None, 0.0, fb)
+            q8.q8_add_relu_quantize(fa, fb, 0.05, out=yo)
+
+        ti, tf = timed(int8_route), timed(fp32_route)
+        blocks[name] = {"int8_us": ti * 1e6, "fp32_route_us": tf * 1e6, "ratio": tf / ti,
+                        "int8_bytes": xin.numel() + xmid.numel() + 3 * yo.numel(),
+                        "fp32_route_bytes": xin.numel() + xmid.numel() + 17 * yo.numel()}
+        del xin, xmid, sc, yo, fa, fb
+    q8.q8_read_status()
+    out["fp32_route"] = {"batch": B, "blocks": blocks,
+                         "int8_us": sum(v["int8_us"] for v in blocks.values()),
+                         "fp32_route_us": sum(v["fp32_route_us"] for v in blocks.values())}
+    torch.cuda.empty_cache()
+    return out
 
 
 def main():
@@ -767,6 +865,8 @@ def main():
     ap.add_argument("--bandwidth-only", type=int, default=0, metavar="REPS",
                     help="run only the memory-bound kernels, REPS timed launches each, print their JSON and exit "
                          "(the command the ncu summary of these kernels is taken with)")
+    ap.add_argument("--ssd-tail-only", action="store_true",
+                    help="run only the SSD tail and the FP32-route comparison, print their JSON and exit")
     ap.add_argument("--skip-networks", "--skip-resnet50", dest="skip_networks", action="store_true",
                     help="leave out the whole-network numbers (ResNet-50, Inception-v3, SSD-300)")
     args = ap.parse_args()
@@ -776,6 +876,10 @@ def main():
         import torch
         print(json.dumps({"bandwidth_kernels": bandwidth_kernel_numbers(torch.device("cuda", 0), measured_peaks()["hbm_gbs"],
                                                                         reps=args.bandwidth_only)}), flush=True)
+        return
+    if args.ssd_tail_only:
+        import torch
+        print(json.dumps({"ssd_tail": ssd_tail_numbers(torch.device("cuda", 0), measured_peaks()["hbm_gbs"])}), flush=True)
         return
     if args.impl == "reference":
         run_reference(args)

@@ -305,11 +305,11 @@ int q8_avgpool2d(const void* x, int t, int N, int H, int W, int C, int kh, int k
  * ---------------------------------------------------------------------- */
 
 /* L2 normalisation across the channels of each pixel, on unsigned 8-bit codes:
- *   S = sum_c z_c^2 (integer),  d = sqrt(float(S) * (qx * qx) + eps),
- *   y_c = clamp(Round((float(z_c) * mult[c]) / d), 0, 255),   mult[c] = gamma_c qx / qy (formed by the caller).
+ *   S = sum_c z_c^2 (integer),  r = 1 / sqrt(float(S) * (qx * qx) + eps)   (one IEEE division per pixel),
+ *   y_c = clamp(Round((float(z_c) * mult[c]) * r), 0, 255),   mult[c] = gamma_c qx / qy (formed by the caller).
  * x, y: device [pixels][C] u8 (may not overlap); d_mult: device [C] fp32.  The fast path needs C % 4 == 0,
- * x and y 4-byte aligned and d_mult 16-byte aligned; anything else takes a scalar kernel.  0 / 0 (an all-zero
- * pixel with eps == 0) gives code 0.  Asynchronous on `stream`.
+ * x and y 4-byte aligned and d_mult 16-byte aligned; anything else takes a scalar kernel.  An all-zero pixel
+ * with eps == 0 gives code 0.  Asynchronous on `stream`.
  * Errors: Q8_ERR_INVALID_ARG (null pointer, C outside 1..65536), Q8_ERR_NONFINITE (qx not finite positive, eps
  * negative or not finite), Q8_ERR_CUDA. */
 int q8_l2norm(const void* x, size_t pixels, int C, float qx, float eps, const float* d_mult, void* y, void* stream);

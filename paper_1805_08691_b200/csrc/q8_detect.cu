@@ -19,51 +19,82 @@ namespace q8 {
 namespace {
 
 // ------------------------------------------------------------------------------------------ L2 normalisation
-//   S = sum_c z_c^2,  d = sqrt(float(S) * (q_x * q_x) + eps),  y_c = clamp(Round((float(z_c) * m_c) / d), 0, 255)
-__device__ __forceinline__ unsigned int l2_word(unsigned int w, const float4 m, float d) {
-  const float v0 = __fdiv_rn(__fmul_rn((float)(w & 0xffu), m.x), d);
-  const float v1 = __fdiv_rn(__fmul_rn((float)((w >> 8) & 0xffu), m.y), d);
-  const float v2 = __fdiv_rn(__fmul_rn((float)((w >> 16) & 0xffu), m.z), d);
-  const float v3 = __fdiv_rn(__fmul_rn((float)(w >> 24), m.w), d);
+//   S = sum_c z_c^2,  r = 1 / sqrt(float(S) * (q_x * q_x) + eps),  y_c = clamp(Round((float(z_c) * m_c) * r), 0, 255)
+__device__ __forceinline__ unsigned int l2_word(unsigned int w, const float4 m, float r) {
+  // byte -> float without a conversion instruction: 0x4B0000bb is 2^23 + b exactly
+  const float f0 = __fsub_rn(__uint_as_float(__byte_perm(w, 0x4B000000u, 0x7540u)), 8388608.0f);
+  const float f1 = __fsub_rn(__uint_as_float(__byte_perm(w, 0x4B000000u, 0x7541u)), 8388608.0f);
+  const float f2 = __fsub_rn(__uint_as_float(__byte_perm(w, 0x4B000000u, 0x7542u)), 8388608.0f);
+  const float f3 = __fsub_rn(__uint_as_float(__byte_perm(w, 0x4B000000u, 0x7543u)), 8388608.0f);
+  const float v0 = __fmul_rn(__fmul_rn(f0, m.x), r), v1 = __fmul_rn(__fmul_rn(f1, m.y), r);
+  const float v2 = __fmul_rn(__fmul_rn(f2, m.z), r), v3 = __fmul_rn(__fmul_rn(f3, m.w), r);
   unsigned int b0, b1, b2, b3;
   asm("cvt.rni.sat.u8.f32 %0, %1;" : "=r"(b0) : "f"(v0));
   asm("cvt.rni.sat.u8.f32 %0, %1;" : "=r"(b1) : "f"(v1));
   asm("cvt.rni.sat.u8.f32 %0, %1;" : "=r"(b2) : "f"(v2));
   asm("cvt.rni.sat.u8.f32 %0, %1;" : "=r"(b3) : "f"(v3));
-  return b0 | (b1 << 8) | (b2 << 16) | (b3 << 24);
+  return __byte_perm(__byte_perm(b0, b1, 0x0040u), __byte_perm(b2, b3, 0x0040u), 0x5410u);
 }
 
-// One warp per pixel, C a multiple of 4 and rows 4-byte aligned: a lane takes words lane, lane + 32, ...
-// (kept in registers for up to 1024 channels, re-read beyond that).
-constexpr int kL2Words = 8;  // words per lane held in registers: 8 * 32 * 4 = 1024 channels
+__device__ __forceinline__ float l2_recip(unsigned int s, float qx2, float eps) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  return __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fmul_rn((float)s, qx2), eps)));
+}
+
+// A warp takes two pixels per step (all loads of both are issued before the first sum is reduced), C a multiple of
+// 4 and rows 4-byte aligned: a lane takes words lane, lane + 32, ... of each pixel, kept in registers (kL2Words
+// words per lane: up to 512 channels; wider rows take the kernel below).
+constexpr int kL2Words = 4;
 __global__ void __launch_bounds__(256) l2norm_kernel(const unsigned int* __restrict__ x, size_t pixels, int cw, float qx2,
                                                      float eps, const float4* __restrict__ mult, unsigned int* __restrict__ y) {
   const int lane = threadIdx.x & 31;
   const size_t warp = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = ((size_t)gridDim.x * blockDim.x) >> 5;
-  for (size_t p = warp; p < pixels; p += nwarps) {
-    const unsigned int* row = x + p * (size_t)cw;
-    unsigned int w[kL2Words];
-    unsigned int s = 0;  // at most 65536 channels of 255^2: below 2^32
+  float4 m[kL2Words];
+#pragma unroll
+  for (int j = 0; j < kL2Words; ++j) m[j] = lane + 32 * j < cw ? __ldg(mult + lane + 32 * j) : make_float4(0.f, 0.f, 0.f, 0.f);
+  for (size_t p = 2 * warp; p < pixels; p += 2 * nwarps) {
+    const bool two = p + 1 < pixels;
+    const unsigned int* row0 = x + p * (size_t)cw;
+    const unsigned int* row1 = row0 + (two ? cw : 0);
+    unsigned int w0[kL2Words], w1[kL2Words];
 #pragma unroll
     for (int j = 0; j < kL2Words; ++j) {
       const int i = lane + 32 * j;
-      w[j] = i < cw ? __ldg(row + i) : 0u;
-      s = __dp4a(w[j], w[j], s);
+      w0[j] = i < cw ? __ldcs(row0 + i) : 0u;
+      w1[j] = i < cw ? __ldcs(row1 + i) : 0u;
     }
-    for (int i = lane + 32 * kL2Words; i < cw; i += 32) {
+    unsigned int s0 = 0, s1 = 0;  // at most 2048 channels of 255^2: far below 2^32
+#pragma unroll
+    for (int j = 0; j < kL2Words; ++j) { s0 = __dp4a(w0[j], w0[j], s0); s1 = __dp4a(w1[j], w1[j], s1); }
+    const float r0 = l2_recip(s0, qx2, eps), r1 = l2_recip(s1, qx2, eps);
+    unsigned int* out0 = y + p * (size_t)cw;
+#pragma unroll
+    for (int j = 0; j < kL2Words; ++j) {
+      const int i = lane + 32 * j;
+      if (i < cw) {
+        __stcs(out0 + i, l2_word(w0[j], m[j], r0));
+        if (two) __stcs(out0 + cw + i, l2_word(w1[j], m[j], r1));
+      }
+    }
+  }
+}
+
+// Rows wider than the registers of the kernel above hold (C % 4 == 0): one warp per pixel, the row is read twice.
+__global__ void __launch_bounds__(256) l2norm_wide_kernel(const unsigned int* __restrict__ x, size_t pixels, int cw, float qx2,
+                                                          float eps, const float4* __restrict__ mult, unsigned int* __restrict__ y) {
+  const int lane = threadIdx.x & 31;
+  const size_t warp = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = ((size_t)gridDim.x * blockDim.x) >> 5;
+  for (size_t p = warp; p < pixels; p += nwarps) {
+    const unsigned int* row = x + p * (size_t)cw;
+    unsigned int s = 0;  // at most 65536 channels of 255^2: below 2^32
+    for (int i = lane; i < cw; i += 32) {
       const unsigned int v = __ldg(row + i);
       s = __dp4a(v, v, s);
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    const float d = __fsqrt_rn(__fadd_rn(__fmul_rn((float)s, qx2), eps));
+    const float r = l2_recip(s, qx2, eps);
     unsigned int* out = y + p * (size_t)cw;
-#pragma unroll
-    for (int j = 0; j < kL2Words; ++j) {
-      const int i = lane + 32 * j;
-      if (i < cw) out[i] = l2_word(w[j], __ldg(mult + i), d);
-    }
-    for (int i = lane + 32 * kL2Words; i < cw; i += 32) out[i] = l2_word(__ldg(row + i), __ldg(mult + i), d);
+    for (int i = lane; i < cw; i += 32) out[i] = l2_word(__ldg(row + i), __ldg(mult + i), r);
   }
 }
 
@@ -75,10 +106,10 @@ __global__ void __launch_bounds__(256) l2norm_scalar_kernel(const unsigned char*
     const unsigned char* row = x + p * (size_t)C;
     unsigned long long s = 0;
     for (int c = 0; c < C; ++c) s += (unsigned int)row[c] * (unsigned int)row[c];
-    const float d = __fsqrt_rn(__fadd_rn(__fmul_rn((float)s, qx2), eps));
+    const float r = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(__fmul_rn((float)s, qx2), eps)));
     for (int c = 0; c < C; ++c) {
       unsigned int b;
-      asm("cvt.rni.sat.u8.f32 %0, %1;" : "=r"(b) : "f"(__fdiv_rn(__fmul_rn((float)row[c], mult[c]), d)));
+      asm("cvt.rni.sat.u8.f32 %0, %1;" : "=r"(b) : "f"(__fmul_rn(__fmul_rn((float)row[c], mult[c]), r)));
       y[p * (size_t)C + c] = (unsigned char)b;
     }
   }
@@ -350,11 +381,17 @@ int q8_l2norm(const void* x, size_t pixels, int C, float qx, float eps, const fl
   cudaStream_t s = as_stream(stream);
   const bool vec = C % 4 == 0 && (reinterpret_cast<uintptr_t>(x) & 3u) == 0 && (reinterpret_cast<uintptr_t>(y) & 3u) == 0 && aligned16(d_mult);
   if (vec) {
-    const size_t blocks = (pixels + 7) / 8;  // eight warps (pixels) per block
     const size_t cap = (size_t)sm_count() * 8;
-    l2norm_kernel<<<(unsigned)(blocks < cap ? blocks : cap), 256, 0, s>>>(static_cast<const unsigned int*>(x), pixels, C / 4, qx2, eps,
-                                                                            reinterpret_cast<const float4*>(d_mult), static_cast<unsigned int*>(y));
-    return check_launch("l2norm_kernel");
+    if (C / 4 <= 32 * kL2Words) {
+      const size_t blocks = (pixels + 15) / 16;  // eight warps of two pixels per block and step
+      l2norm_kernel<<<(unsigned)(blocks < cap ? blocks : cap), 256, 0, s>>>(static_cast<const unsigned int*>(x), pixels, C / 4, qx2, eps,
+                                                                              reinterpret_cast<const float4*>(d_mult), static_cast<unsigned int*>(y));
+      return check_launch("l2norm_kernel");
+    }
+    const size_t blocks = (pixels + 7) / 8;
+    l2norm_wide_kernel<<<(unsigned)(blocks < cap ? blocks : cap), 256, 0, s>>>(static_cast<const unsigned int*>(x), pixels, C / 4, qx2, eps,
+                                                                                 reinterpret_cast<const float4*>(d_mult), static_cast<unsigned int*>(y));
+    return check_launch("l2norm_wide_kernel");
   }
   const size_t blocks = (pixels + 255) / 256, cap = (size_t)sm_count() * 8;
   l2norm_scalar_kernel<<<(unsigned)(blocks < cap ? blocks : cap), 256, 0, s>>>(static_cast<const unsigned char*>(x), pixels, C, qx2, eps, d_mult,

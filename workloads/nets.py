@@ -321,7 +321,8 @@ def detection_inputs(seed: int, batch: int, priors: int = 8732, classes: int = 2
     g = rng(seed)
     loc = normal(g, (batch, priors, 4))
     conf = normal(g, (batch, priors, classes))
-    conf[..., 0] += 4.0                                         # background dominates, as in a trained detector
+    conf[..., 0] += 8.0                                         # background dominates, as in a trained detector:
+    #                                                             a few boxes per class and image pass a 0.01 threshold
     hot = g.random((batch, priors)) < peaked
     cls = g.integers(1, classes, (batch, priors))
     n_idx, p_idx = np.nonzero(hot)
