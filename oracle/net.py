@@ -125,6 +125,8 @@ def network_prepare(layers, folded, maxima, per_channel=False, sum_policy="max")
                 own[name] = final_factor(L.src[0])
             elif L.op == "concat":
                 own[name] = group_factor(root[name])
+            elif L.op == "l2norm":
+                own[name] = o.factor(maxima[name], 8)
             elif L.residual is not None and sum_policy == "post_sum":
                 own[name] = o.factor(maxima[name], 8)
             elif L.residual is not None:
@@ -174,6 +176,11 @@ def network_prepare(layers, folded, maxima, per_channel=False, sum_policy="max")
             info[L.name] = (t_in, q_in)
         elif L.op == "concat":
             info[L.name] = (t_in, group_factor(root[L.name]))
+        elif L.op == "l2norm":
+            assert t_in == o.U8, "L2 normalisation follows a ReLU"
+            q_y = final_factor(L.name)
+            prep[L.name] = {"mult": o.l2norm_mult(L.gamma, q_in, q_y), "eps": L.eps, "q_in": q_in}
+            info[L.name] = (o.U8, q_y)
         else:
             raise ValueError(L.op)
     return prep, info
@@ -197,4 +204,7 @@ def network_forward(layers, prep, info, x_f32, threads=1):
             out[L.name] = o.pool(x, "avg", L.k, L.stride, L.pad, L.ceil_mode)
         elif L.op == "concat":
             out[L.name] = o.concat([out[s] for s in L.src], [info[s][1] for s in L.src], info[L.name][1])
+        elif L.op == "l2norm":
+            d = prep[L.name]
+            out[L.name] = o.l2norm(x, d["q_in"], d["eps"], d["mult"])
     return out

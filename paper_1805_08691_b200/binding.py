@@ -354,26 +354,40 @@ def q8_detection_output_workspace_bytes(N, P, classes, background, nms_top_k, ke
     return n.value
 
 
+def _cell_view(t, what):
+    """(pointer, cell stride in floats, cells per image) of a CUDA fp32 tensor [N, cells..., values] whose cells lie a
+    fixed stride apart (a contiguous tensor, or a slice of the last dimension of one)."""
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == torch.float32 and t.dim() >= 2 and t.stride(-1) == 1):
+        raise TypeError(f"{what}: expected a CUDA fp32 tensor with unit stride in its last dimension")
+    if t.dim() == 2:
+        return t.data_ptr(), int(t.stride(0)), 1
+    stride = int(t.stride(-2))
+    for i in range(t.dim() - 2):
+        if t.shape[i] > 1 and t.stride(i) != t.stride(i + 1) * t.shape[i + 1]:
+            raise TypeError(f"{what}: cells are not a fixed stride apart")
+    cells = 1
+    for v in t.shape[1:-1]:
+        cells *= int(v)
+    return t.data_ptr(), stride, cells
+
+
 def q8_detection_output(sources, priors, variances, classes, background=0, conf_thresh=0.01, nms_thresh=0.45,
                         nms_top_k=400, keep_top_k=200, workspace=None, out=None, counts=None):
-    """sources: list of (loc, conf, boxes_per_cell) with loc [N, cells..., >= boxes*4] and conf [N, cells...,
-    >= boxes*classes] contiguous CUDA fp32 tensors (the last dimension is the cell stride), or of
-    (loc, conf, boxes_per_cell, loc_offset, conf_offset) where both views start that many floats into a cell of a
-    shared tensor.  priors: CUDA fp32 [P, 4].  Returns (rows [N, keep_top_k, 6], counts [N])."""
+    """sources: list of (loc, conf, boxes_per_cell) with loc [N, cells..., boxes * 4] and conf [N, cells...,
+    boxes * classes] CUDA fp32 tensors, contiguous or slices of the last dimension of a wider tensor (a merged
+    head).  priors: CUDA fp32 [P, 4].  Returns (rows [N, keep_top_k, 6], counts [N])."""
     N = int(sources[0][0].shape[0])
     n = len(sources)
     locp, confp = (C.c_void_p * n)(), (C.c_void_p * n)()
     lstr, cstr, cells, boxes = (C.c_int * n)(), (C.c_int * n)(), (C.c_int * n)(), (C.c_int * n)()
     P = 0
-    for i, src in enumerate(sources):
-        loc, conf, b = src[0], src[1], int(src[2])
-        lo, co = (int(src[3]), int(src[4])) if len(src) > 3 else (0, 0)
-        _dev(loc, "loc"), _dev(conf, "conf")
-        locp[i], confp[i] = loc.data_ptr() + 4 * lo, conf.data_ptr() + 4 * co
-        lstr[i], cstr[i] = int(loc.shape[-1]), int(conf.shape[-1])
-        cells[i] = loc.numel() // (N * int(loc.shape[-1]))
-        boxes[i] = b
-        P += cells[i] * b
+    for i, (loc, conf, b) in enumerate(sources):
+        locp[i], lstr[i], cells[i] = _cell_view(loc, "loc")
+        confp[i], cstr[i], ccells = _cell_view(conf, "conf")
+        if ccells != cells[i] or int(conf.shape[0]) != N or int(loc.shape[0]) != N:
+            raise ValueError("loc and conf of a source must cover the same cells of the same images")
+        boxes[i] = int(b)
+        P += cells[i] * int(b)
     dev = sources[0][0].device
     nbytes = q8_detection_output_workspace_bytes(N, P, classes, background, nms_top_k, keep_top_k)
     if workspace is None:

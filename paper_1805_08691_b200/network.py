@@ -32,6 +32,7 @@ for the fused residual sum; all tensor arithmetic runs in the library's kernels.
 """
 from typing import Dict, List
 
+import numpy as np
 import torch
 import torch.nn.functional as F
 
@@ -56,6 +57,7 @@ class QuantNetwork:
         self.maxima = maxima
         self.by_name = {L.name: L for L in layers}
         self.convs: Dict[str, pipeline.QuantConv] = {}
+        self.l2: Dict[str, tuple] = {}   # L2 normalisation layers: (input factor, eps, per-channel multipliers)
         self.bufs: Dict[str, torch.Tensor] = {}
         N, H, W, _ = in_shape
         first = next(L for L in layers if L.op == "conv")
@@ -106,6 +108,14 @@ class QuantNetwork:
                 self.info[L.name] = (t_in, q_in)
             elif L.op == "concat":
                 self.info[L.name] = (t_in, self._factor(L.name))
+            elif L.op == "l2norm":
+                if t_in != q8.Q8_U8:
+                    raise ValueError("L2 normalisation needs unsigned codes (it follows a ReLU)")
+                q_y = self._factor(L.name)
+                # gamma q_x / q_y formed in fp64 (a multiply, a division) and rounded once, per channel
+                mult = ((np.asarray(L.gamma, dtype=np.float64) * np.float64(q_in)) / np.float64(q_y)).astype(np.float32)
+                self.l2[L.name] = (float(q_in), float(L.eps), torch.from_numpy(mult).to(device))
+                self.info[L.name] = (q8.Q8_U8, q_y)
             else:
                 raise ValueError(L.op)
             dt = q8.TORCH_DTYPES[self.info[L.name][0]]
@@ -152,6 +162,8 @@ class QuantNetwork:
                 self.shape[L.name] = (n, P, Q, c)
             elif L.op == "concat":
                 self.shape[L.name] = (n, h, w_, sum(self.shape[s][3] for s in L.src))
+            elif L.op == "l2norm":
+                self.shape[L.name] = (n, h, w_, c)
             else:
                 raise ValueError(L.op)
 
@@ -200,6 +212,8 @@ class QuantNetwork:
             return self._factor(L.src[0])
         if L.op == "concat":
             return self._factor(name)
+        if L.op == "l2norm":
+            return q8.q8_factor(m[name], 8)
         if L.residual is not None and self.sum_policy == "post_sum":
             return q8.q8_factor(m[name], 8)       # calibrated on the tensor the layer emits
         if L.residual is not None:
@@ -362,6 +376,9 @@ class QuantNetwork:
             q8.q8_maxpool2d(x, L.k, L.stride, L.pad, L.ceil_mode, out=b[L.name])
         elif L.op == "avgpool":
             q8.q8_avgpool2d(x, L.k, L.stride, L.pad, L.ceil_mode, out=b[L.name])
+        elif L.op == "l2norm":
+            q_in, eps, mult = self.l2[L.name]
+            q8.q8_l2norm(x, q_in, eps, mult, out=b[L.name])
         elif L.op == "concat":
             for s in L.src:
                 if s in self.in_place or self.by_name[s].op == "concat":

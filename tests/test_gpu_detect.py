@@ -64,7 +64,7 @@ def _heads(loc, conf, splits, boxes_per_cell, merged):
         first += cells * b
         if merged:
             both = _cuda(np.concatenate([l, c], 2))
-            out.append((both, both, b, 0, b * 4))
+            out.append((both[..., :b * 4], both[..., b * 4:], b))
         else:
             out.append((_cuda(l), _cuda(c), b))
     return out

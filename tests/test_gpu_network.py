@@ -183,3 +183,27 @@ def test_resnet50_with_sparsity_removed_bit_exact(q8):
     got, want, ref, net = _run_both(q8, layers, hw=224, batch=2, calib_batches=2, seed=3000)
     logits, fp32 = got["fc1000"].cpu().numpy().reshape(2, -1), ref["fc1000"].reshape(2, -1)
     assert float(np.linalg.norm(logits - fp32) / np.linalg.norm(fp32)) < 0.5
+
+
+def test_ssd300_with_normalisation_and_detection_output(q8):
+    """SSD-300 as the detector defines it: the heads of conv4_3 read its L2-normalised copy, and the twelve head
+    tensors (merged per source map on the GPU) go through the detection output.  Every layer and every kept
+    detection bit-exact against the oracle at batch 2."""
+    layers = nets.ssd300(l2norm=True)
+    got, want, ref, net = _run_both(q8, layers, hw=300, batch=2, calib_batches=1, seed=5100, streams=3)
+    assert np.array_equal(got["conv4_3_norm"].cpu().numpy(), want["conv4_3_norm"])
+    srcs = [L.src[0] for L in layers if L.name.endswith("_mbox_loc")]
+    boxes = [L.conv.K // 4 for L in layers if L.name.endswith("_mbox_loc")]
+    classes = 21
+    loc = np.concatenate([want[s + "_mbox_loc"].reshape(2, -1, 4) for s in srcs], 1)
+    conf = np.concatenate([want[s + "_mbox_conf"].reshape(2, -1, classes) for s in srcs], 1)
+    assert loc.shape == (2, 8732, 4) and conf.shape == (2, 8732, classes)
+    priors = nets.ssd300_priors()
+    # random-init heads are nearly flat: a low threshold on purpose, so that suppression has work to do
+    kw = dict(conf_thresh=0.02, nms_thresh=0.45, nms_top_k=400, keep_top_k=200)
+    want_rows, want_counts = o.detection_output(loc, conf, priors, nets.SSD300_VARIANCES, **kw)
+    rows, counts = q8.q8_detection_output([(got[s + "_mbox_loc"], got[s + "_mbox_conf"], b) for s, b in zip(srcs, boxes)],
+                                          _cuda(priors), nets.SSD300_VARIANCES, classes, **kw)
+    q8.q8_read_status()
+    assert np.array_equal(counts.cpu().numpy(), want_counts) and want_counts.min() > 0
+    assert np.array_equal(rows.cpu().numpy(), want_rows)

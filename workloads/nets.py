@@ -20,7 +20,7 @@ from .synth import ConvSpec, make_conv, normal, rng
 @dataclass
 class Layer:
     name: str
-    op: str                      # "conv", "maxpool", "avgpool", "concat"
+    op: str                      # "conv", "maxpool", "avgpool", "concat", "l2norm"
     src: List[str]               # input tensor names ("input" = network input)
     conv: Optional[ConvSpec] = None
     residual: Optional[str] = None   # tensor added to the conv output before the ReLU (fused eltwise sum)
@@ -29,6 +29,8 @@ class Layer:
     stride: Tuple[int, int] = (1, 1)
     pad: Tuple[int, int] = (0, 0)
     ceil_mode: bool = False
+    gamma: Optional[np.ndarray] = None   # "l2norm": per-channel scale of the normalised vector
+    eps: float = 1e-10                   # "l2norm": added to the sum of squares
 
 
 def _pair(v):
@@ -171,11 +173,12 @@ def inception_v3(seed: int = 4000, classes: int = 1000) -> List[Layer]:
     return L
 
 
-def ssd300(seed: int = 5000, classes: int = 21) -> List[Layer]:
+def ssd300(seed: int = 5000, classes: int = 21, l2norm: bool = False) -> List[Layer]:
     """SSD-300 on VGG-16: the base network through conv5_3 (pool3 in ceil mode, pool5 3x3 stride 1), fc6 as
     a dilated 3x3 (dilation 6), fc7 as 1x1, four extra stages, and a 3x3 localisation and confidence head on
     each of the six source maps (38, 19, 10, 5, 3, 1; 4/6/6/6/4/4 boxes per cell, 8732 boxes).  Convolutions
-    carry a bias and no BN; head outputs are dequantized FP32.  No normalisation layer on conv4_3."""
+    carry a bias and no BN; head outputs are dequantized FP32.  l2norm: the heads of conv4_3 read its L2-normalised
+    copy (scale initialised around 20, as the detector's definition has it) instead of conv4_3 itself."""
     g = rng(seed)
     L: List[Layer] = []
 
@@ -194,6 +197,9 @@ def ssd300(seed: int = 5000, classes: int = 21) -> List[Layer]:
         if stage < 5:
             x = pool(f"pool{stage}", x, 2, 2, ceil_mode=(stage == 3))
     sources = [("conv4_3", 512, 4)]
+    if l2norm:
+        L.append(Layer("conv4_3_norm", "l2norm", ["conv4_3"], gamma=g.uniform(15.0, 25.0, 512).astype(np.float32)))
+        sources = [("conv4_3_norm", 512, 4)]
     x = pool("pool5", x, 3, 1, 1)
     x = conv("fc6", x, 512, 1024, 3, pad=6, dil=6)
     x = conv("fc7", x, 1024, 1024, 1)
@@ -255,6 +261,8 @@ def fp32_forward(layers: List[Layer], x: np.ndarray, folded: Dict[str, Tuple[np.
                 y = F.avg_pool2d(xin, L.k, L.stride, L.pad, ceil_mode=L.ceil_mode, count_include_pad=True)
             elif L.op == "concat":
                 y = torch.cat([out[s] for s in L.src], dim=1)
+            elif L.op == "l2norm":
+                y = xin / torch.sqrt((xin * xin).sum(1, keepdim=True) + L.eps) * _t(L.gamma, device).view(1, -1, 1, 1)
             else:
                 raise ValueError(L.op)
             out[L.name] = y
