@@ -271,14 +271,18 @@ def network_numbers(dev, name, reps=20):
     cfg = NETWORKS[name]
     hw = cfg["hw"]
     layers = getattr(nets, cfg["fn"])()
-    folded = {}
-    for L in layers:
-        if L.op != "conv":
-            continue
-        sp = L.conv
-        folded[L.name] = (q8.q8_fold_bn(cuda(sp.w), None, cuda(sp.gamma), cuda(sp.beta), cuda(sp.mean), cuda(sp.var), 1e-5)
-                          if sp.bn else (cuda(sp.w), cuda(sp.b)))
-    folded_np = {k: (w.cpu().numpy(), b.cpu().numpy()) for k, (w, b) in folded.items()}
+
+    def fold(ls):
+        f = {}
+        for L in ls:
+            if L.op != "conv":
+                continue
+            sp = L.conv
+            f[L.name] = (q8.q8_fold_bn(cuda(sp.w), None, cuda(sp.gamma), cuda(sp.beta), cuda(sp.mean), cuda(sp.var), 1e-5)
+                         if sp.bn else (cuda(sp.w), cuda(sp.b)))
+        return f, {k: (w.cpu().numpy(), b.cpu().numpy()) for k, (w, b) in f.items()}
+
+    folded, folded_np = fold(layers)
     acts = nets.fp32_forward(layers, nets.images(cfg["seed"] + 10, 2, hw), folded_np, device=dev)
     cal = pipeline.Calibrator(sorted(acts), device=dev)
     for k, v in acts.items():
@@ -311,23 +315,44 @@ def network_numbers(dev, name, reps=20):
         # quoted on the MACs of the original network)
         from paper_1805_08691_b200 import graph
         variants.append(("batch%d_sparsity_removed" % cfg["batch"], cfg["batch"], graph.remove_sparsity(layers)))
+    if name == "ssd300":
+        # the detector as the paper ran it: conv4_3 L2-normalised for its heads, detection output on the heads
+        variants.append(("batch%d_with_l2norm_and_detection_output" % cfg["batch"], cfg["batch"], nets.ssd300(l2norm=True)))
     for key, batch, net_layers in variants:
+        folded_v = folded
         if net_layers is not layers:
-            acts = nets.fp32_forward(net_layers, nets.images(cfg["seed"] + 10, 2, hw), folded_np, device=dev)
+            folded_v, folded_np_v = fold(net_layers)
+            acts = nets.fp32_forward(net_layers, nets.images(cfg["seed"] + 10, 2, hw), folded_np_v, device=dev)
             cal = pipeline.Calibrator(sorted(acts), device=dev)
             for k, v in acts.items():
                 cal.observe(k, cuda(v))
             maxima = cal.maxima()
             del acts
-        net = network.QuantNetwork(net_layers, folded, maxima, (batch, hw, hw, 3), device=dev,
+        net = network.QuantNetwork(net_layers, folded_v, maxima, (batch, hw, hw, 3), device=dev,
                                    streams=int(os.environ.get("Q8_BENCH_STREAMS", "4")))
         x = cuda(nets.images(cfg["seed"] + 1, batch, hw))
-        net.forward(x)
+        tail = None
+        if key.endswith("detection_output"):
+            srcs = [L.src[0] for L in net_layers if L.name.endswith("_mbox_loc")]
+            heads = [(net.outputs[s_ + "_mbox_loc"], net.outputs[s_ + "_mbox_conf"], net.by_name[s_ + "_mbox_loc"].conv.K // 4) for s_ in srcs]
+            priors = cuda(nets.ssd300_priors())
+            ws = torch.empty(q8.q8_detection_output_workspace_bytes(batch, 8732, 21, 0, 400, 200), dtype=torch.uint8, device=dev)
+            rows, counts = torch.empty((batch, 200, 6), device=dev), torch.empty(batch, dtype=torch.int32, device=dev)
+
+            def tail():
+                q8.q8_detection_output(heads, priors, nets.SSD300_VARIANCES, 21, workspace=ws, out=rows, counts=counts)
+
+        def run():
+            net.forward(x)
+            if tail is not None:
+                tail()
+
+        run()
         torch.cuda.synchronize()
         q8.q8_read_status()
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
-            net.forward(x)
+            run()
         for _ in range(3):
             g.replay()
         torch.cuda.synchronize()

@@ -232,47 +232,142 @@ __device__ __forceinline__ float iou(const float4 a, const float4 b) {
   return __fdiv_rn(inter, __fsub_rn(__fadd_rn(area_a, area_b), inter));
 }
 
-constexpr int kNmsThreads = 1024;
+constexpr int kNmsThreads = 512;     // per (image, class) block
+constexpr int kTopThreads = 1024;    // per image block
 constexpr int kMaxTopK = 512;        // candidates that enter the suppression of one class
-constexpr int kMaxSort = 16384;      // keys one block sorts in shared memory
+constexpr int kMaxSort = 16384;      // boxes per image; keys the per-image block sorts in shared memory
+constexpr int kSelBits = 11;         // key bits per histogram pass of the pre-selection
+constexpr int kSelBins = 1 << kSelBits;
+constexpr int kSelCap = 2048;        // keys handed to the per-class sort
 
-// One block per (image, class other than background).  Keys order candidates by probability, highest first, then by
-// box index: (~bits of the positive probability) << 32 | box.  Shared memory: keys[cap], then top[kMaxTopK] keys and
-// their boxes; the overlap bit matrix reuses the key area once the best candidates are copied out.
+// Warp 0 only: the first bin at which the running sum of hist reaches `need` (need <= the total), and the sum of
+// the bins before it.
+__device__ int select_bin(const int* hist, int need, int* below) {
+  const int lane = threadIdx.x & 31;
+  constexpr int kPer = kSelBins / 32;
+  int local = 0;
+  for (int j = 0; j < kPer; ++j) local += hist[lane * kPer + j];
+  int incl = local;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int v = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  const unsigned int reached = __ballot_sync(0xffffffffu, incl >= need);
+  const int src = reached ? __ffs(reached) - 1 : 31;
+  int bin = 0, bel = 0;
+  if (lane == src) {
+    int cum = incl - local, j = 0;
+    for (; j < kPer - 1; ++j) {
+      const int h = hist[lane * kPer + j];
+      if (cum + h >= need) break;
+      cum += h;
+    }
+    bin = lane * kPer + j;
+    bel = cum;
+  }
+  *below = __shfl_sync(0xffffffffu, bel, src);
+  return __shfl_sync(0xffffffffu, bin, src);
+}
+
+__device__ __forceinline__ unsigned long long nms_key(float s, int p) {
+  return ((unsigned long long)(~__float_as_uint(s)) << 32) | (unsigned int)p;
+}
+
+// One block per (image, class other than background).  Keys order candidates (probability > conf_thresh) by
+// probability, highest first, then by box index: (~bits of the positive probability) << 32 | box; they are unique.
+// Only the best top_k can matter.  The probabilities of the class (P floats, L2 resident) are read once per pass: the
+// first pass counts the candidates and fills a histogram of the leading kSelBits key bits; up to kSelCap candidates
+// are simply collected, more are narrowed by a radix selection (per pass: the bin in which the running count
+// reaches top_k; keys below it are in, keys in it go to the next pass over the next bits) until the keys at or below
+// the chosen prefix number at most kSelCap; with unique keys that ends at the latest when all 64 bits are fixed.
+// The collected keys are sorted (bitonic, shared memory), the best top_k and their boxes copied out, their overlaps
+// written as a bit matrix (over the sort area) and one warp walks the candidates in order.
 __global__ void __launch_bounds__(kNmsThreads) nms_class_kernel(const float4* __restrict__ boxes, const float* __restrict__ prob, int P,
                                                                 int classes, int background, float conf_thresh, float nms_thresh,
-                                                                int top_k, unsigned int key_bytes,
+                                                                int top_k, unsigned int work_bytes,
                                                                 unsigned long long* __restrict__ kept_keys,
                                                                 int* __restrict__ kept_count) {
-  // key_bytes: room for the keys of all P boxes and for top_k rows of the overlap matrix, whichever is larger
+  // work_bytes: room for kSelCap keys and for top_k rows of the overlap matrix, whichever is larger
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);
-  unsigned long long* top = reinterpret_cast<unsigned long long*>(smem_raw + key_bytes);
+  unsigned long long* work = reinterpret_cast<unsigned long long*>(smem_raw);
+  unsigned long long* top = reinterpret_cast<unsigned long long*>(smem_raw + work_bytes);
   float4* tbox = reinterpret_cast<float4*>(top + kMaxTopK);
+  int* hist = reinterpret_cast<int*>(tbox + kMaxTopK);
   unsigned int* mask = reinterpret_cast<unsigned int*>(smem_raw);
-  __shared__ int cnt;
+  __shared__ int cnt, sel_bin, sel_below, sel_in_bin, sel_cnt;
   const int n = blockIdx.y;
   int c = blockIdx.x;
   if (background >= 0 && c >= background) ++c;  // blockIdx.x runs over the foreground classes
-  if (threadIdx.x == 0) cnt = 0;
+  if (threadIdx.x == 0) { cnt = 0; sel_cnt = 0; }
+  for (int i = threadIdx.x; i < kSelBins; i += blockDim.x) hist[i] = 0;
   __syncthreads();
   const float* sc = prob + ((size_t)n * classes + c) * P;
-  for (int p = threadIdx.x; p < P; p += blockDim.x) {
-    const float s = sc[p];
-    if (s > conf_thresh) keys[atomicAdd(&cnt, 1)] = ((unsigned long long)(~__float_as_uint(s)) << 32) | (unsigned int)p;
+  for (int p0 = threadIdx.x; p0 < P; p0 += 4 * blockDim.x) {
+    float s[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) s[u] = p0 + u * blockDim.x < P ? sc[p0 + u * blockDim.x] : -1.0f;
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      if (s[u] > conf_thresh) {
+        atomicAdd(&cnt, 1);
+        atomicAdd(&hist[nms_key(s[u], 0) >> (64 - kSelBits)], 1);
+      }
   }
   __syncthreads();
-  const int m = cnt;
+  int m = cnt;
+  int shift = 64;                    // keys with (key >> shift) <= limit are collected; 64: all candidates
+  unsigned long long limit = 0;
+  if (m > kSelCap) {                 // (the whole block takes this branch or none of it does)
+    int need = top_k, accepted = 0;  // accepted: keys below the prefix chosen so far
+    int width = kSelBits;            // bits of the digit the histogram holds
+    shift = 64 - kSelBits;
+    for (;;) {
+      if (threadIdx.x < 32) {
+        int below;
+        const int b = select_bin(hist, need, &below);
+        if (threadIdx.x == 0) { sel_bin = b; sel_below = below; sel_in_bin = hist[b]; }
+      }
+      __syncthreads();
+      limit = (limit << width) | (unsigned int)sel_bin;
+      accepted += sel_below;
+      need -= sel_below;
+      m = accepted + sel_in_bin;
+      if (m <= kSelCap || shift == 0) break;
+      const int ns = shift >= kSelBits ? shift - kSelBits : 0;
+      width = shift - ns;
+      const unsigned int dmask = (1u << width) - 1u;
+      for (int i = threadIdx.x; i < kSelBins; i += blockDim.x) hist[i] = 0;
+      __syncthreads();
+      for (int p = threadIdx.x; p < P; p += blockDim.x) {
+        const float s = sc[p];
+        if (s > conf_thresh) {
+          const unsigned long long key = nms_key(s, p);
+          if ((key >> shift) == limit) atomicAdd(&hist[(unsigned int)(key >> ns) & dmask], 1);
+        }
+      }
+      __syncthreads();
+      shift = ns;
+    }
+  }
+  for (int p = threadIdx.x; p < P; p += blockDim.x) {
+    const float s = sc[p];
+    if (s > conf_thresh) {
+      const unsigned long long key = nms_key(s, p);
+      if (shift == 64 || (key >> shift) <= limit) work[atomicAdd(&sel_cnt, 1)] = key;
+    }
+  }
   int size = 1;
   while (size < m) size <<= 1;
-  for (int i = m + threadIdx.x; i < size; i += blockDim.x) keys[i] = ~0ull;
   __syncthreads();
-  bitonic_sort(keys, size);
+  for (int i = m + threadIdx.x; i < size; i += blockDim.x) work[i] = ~0ull;
+  __syncthreads();
+  bitonic_sort(work, size);
   const int k = m < top_k ? m : top_k;
   const float4* bx = boxes + (size_t)n * P;
   for (int i = threadIdx.x; i < k; i += blockDim.x) {
-    top[i] = keys[i];
-    tbox[i] = bx[(unsigned int)keys[i]];
+    top[i] = work[i];
+    tbox[i] = bx[(unsigned int)work[i]];
   }
   __syncthreads();
   const int W = (k + 31) >> 5;
@@ -306,7 +401,7 @@ __global__ void __launch_bounds__(kNmsThreads) nms_class_kernel(const float4* __
 
 // One block per image: the kept detections of all classes ordered by probability (ties: class, then box), the first
 // keep_top_k written as rows (class, probability, xmin, ymin, xmax, ymax); unused rows are zero.
-__global__ void __launch_bounds__(kNmsThreads) keep_top_kernel(const float4* __restrict__ boxes, const unsigned long long* __restrict__ kept_keys,
+__global__ void __launch_bounds__(kTopThreads) keep_top_kernel(const float4* __restrict__ boxes, const unsigned long long* __restrict__ kept_keys,
                                                                const int* __restrict__ kept_count, int P, int classes, int background,
                                                                int top_k, int keep_top_k, float* __restrict__ out,
                                                                int* __restrict__ counts) {
@@ -489,13 +584,11 @@ int q8_detection_output(int n_sources, const float* const* loc, const int* loc_s
   }
   const int fg = classes - (background >= 0 ? 1 : 0);
   {
-    int cap = 1;
-    while (cap < P) cap <<= 1;
     const unsigned int W = (unsigned)(nms_top_k + 31) / 32;
-    unsigned int key_bytes = (unsigned)cap * 8u;
-    if (key_bytes < (unsigned)nms_top_k * W * 4u) key_bytes = (unsigned)nms_top_k * W * 4u;
-    key_bytes = (key_bytes + 15u) & ~15u;
-    const size_t smem = (size_t)key_bytes + (size_t)kMaxTopK * (8 + 16);
+    unsigned int work_bytes = (unsigned)kSelCap * 8u;
+    if (work_bytes < (unsigned)nms_top_k * W * 4u) work_bytes = (unsigned)nms_top_k * W * 4u;
+    work_bytes = (work_bytes + 15u) & ~15u;
+    const size_t smem = (size_t)work_bytes + (size_t)kMaxTopK * (8 + 16) + (size_t)kSelBins * 4;
     const int dev = current_device();
     static std::atomic<size_t> configured[kMaxDevices];
     if (dev < 0 || configured[dev].load() < smem) {
@@ -504,7 +597,7 @@ int q8_detection_output(int n_sources, const float* const* loc, const int* loc_s
       if (dev >= 0) configured[dev].store(smem);
     }
     nms_class_kernel<<<dim3((unsigned)fg, (unsigned)N), kNmsThreads, smem, s>>>(boxes, prob, (int)P, classes, background, conf_thresh, nms_thresh,
-                                                                               nms_top_k, key_bytes, keys, kcount);
+                                                                               nms_top_k, work_bytes, keys, kcount);
     const int rc2 = check_launch("nms_class_kernel");
     if (rc2 != Q8_OK) return rc2;
   }
@@ -519,7 +612,7 @@ int q8_detection_output(int n_sources, const float* const* loc, const int* loc_s
       if (rc2 != Q8_OK) return rc2;
       if (dev >= 0) configured[dev].store(smem);
     }
-    keep_top_kernel<<<(unsigned)N, kNmsThreads, smem, s>>>(boxes, keys, kcount, (int)P, classes, background, nms_top_k, keep_top_k, d_out, d_counts);
+    keep_top_kernel<<<(unsigned)N, kTopThreads, smem, s>>>(boxes, keys, kcount, (int)P, classes, background, nms_top_k, keep_top_k, d_out, d_counts);
   }
   return check_launch("keep_top_kernel");
 }

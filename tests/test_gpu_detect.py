@@ -131,6 +131,20 @@ def test_detection_output_edge_cases(q8, case):
     _compare(q8, loc, conf, priors, [P], [1], **kw)
 
 
+@pytest.mark.parametrize("spread", [0.0, 1e-3, 0.5])
+def test_detection_output_many_candidates_with_equal_leading_bits(q8, spread):
+    """More candidates than the pre-selection hands to the sort: identical probabilities (the selection cannot
+    separate them and everything is sorted), probabilities that differ in their last bits only, and well spread
+    ones."""
+    g = np.random.default_rng(17)
+    P, classes = 4000, 3
+    x0, y0 = g.integers(0, 28, P) / 32.0, g.integers(0, 28, P) / 32.0
+    w, h = g.integers(1, 5, P) / 32.0, g.integers(1, 5, P) / 32.0
+    priors = np.stack([x0 + w / 2, y0 + h / 2, w, h], 1).astype(np.float32)
+    conf = (g.normal(0, 1, (2, P, classes)) * spread).astype(np.float32)
+    _compare(q8, np.zeros((2, P, 4), np.float32), conf, priors, [P], [1], conf_thresh=0.05, nms_top_k=300, keep_top_k=150)
+
+
 def test_detection_output_refuses_what_it_cannot_hold(q8):
     loc = torch.zeros((1, 20000, 4), device="cuda")
     conf = torch.zeros((1, 20000, 3), device="cuda")
