@@ -587,10 +587,25 @@ def run_ours(args):
         divs = [d for d in range(240, 0, -1) if args.steps % d == 0]
         chunk = next((d for d in divs if d % n_sets == 0), divs[0])
     replays_per_repeat = args.steps // chunk
+    # Steps work on different batches and are independent, so they may be in flight together: with
+    # --step-streams S step i is enqueued on stream i % S (every buffer set stays on one stream).  A step is still
+    # the whole block over one batch; the next batch's first kernel fills the SMs that the last kernel of this one
+    # leaves idle while it drains.
+    n_step_streams = max(1, min(args.step_streams, n_sets))
+    while n_sets % n_step_streams:
+        n_step_streams -= 1
+    side = [torch.cuda.Stream(device=dev) for _ in range(n_step_streams - 1)]
     timed = torch.cuda.CUDAGraph()
     with torch.cuda.graph(timed):
+        main = torch.cuda.current_stream()
+        for st in side:
+            st.wait_stream(main)
         for i in range(chunk):
-            blocks[i % n_sets](xs[i % n_sets], out=ys[i % n_sets])
+            st = main if i % n_step_streams == 0 else side[i % n_step_streams - 1]
+            with torch.cuda.stream(st):
+                blocks[i % n_sets](xs[i % n_sets], out=ys[i % n_sets])
+        for st in side:
+            main.wait_stream(st)
     # one graph per launch kind for the per-kernel durations: the same launch repeated over all buffer sets
     kreps = 8
     kinds = ["a", "bc"] if fused else ["a", "b", "c"]
@@ -757,7 +772,7 @@ def run_ours(args):
             "vs_baseline": None, "dtype": "s32", "data": "synthetic",
             "config": CONFIG,
             "timing": {"l2": "rotating %d buffer sets of %.0f MB (> 126 MB L2)" % (n_sets, set_bytes / 1e6),
-                       "launch": "CUDA graph of %d steps, %d replays per repeat" % (chunk, replays_per_repeat),
+                       "launch": "CUDA graph of %d steps on %d stream(s), %d replays per repeat" % (chunk, n_step_streams, replays_per_repeat),
                        "timed_repeats": repeats, "statistic": "median over the repeats of the time of K steps",
                        "ms_per_step_min": ms_min / args.steps, "timed_region_ms": ms_region},
             "clocks": clocks,
@@ -886,6 +901,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sets", type=int, default=6, help="rotating buffer sets (working set must exceed L2)")
+    ap.add_argument("--step-streams", type=int, default=2,
+                    help="streams the steps of the timed region alternate between (steps are independent batches)")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--bandwidth-only", type=int, default=0, metavar="REPS",
                     help="run only the memory-bound kernels, REPS timed launches each, print their JSON and exit "
