@@ -162,6 +162,7 @@ __device__ __forceinline__ float exp_fixed(float x) {
 }
 
 constexpr int kMaxSources = 8;
+constexpr int kRegClasses = 24;   // class counts up to this keep a box's logits in registers
 struct DetSources {
   const float* loc[kMaxSources];
   const float* conf[kMaxSources];
@@ -197,12 +198,32 @@ __global__ void __launch_bounds__(256) decode_softmax_kernel(const __grid_consta
     const float h = __fmul_rn(exp_fixed(__fmul_rn(v3, l[3])), pr.w);
     const float hw = __fmul_rn(w, 0.5f), hh = __fmul_rn(h, 0.5f);
     boxes[i] = make_float4(__fsub_rn(cx, hw), __fsub_rn(cy, hh), __fadd_rn(cx, hw), __fadd_rn(cy, hh));
-    float m = x[0];
-    for (int c = 1; c < classes; ++c) m = x[c] > m ? x[c] : m;
-    float sum = 0.0f;
-    for (int c = 0; c < classes; ++c) sum = __fadd_rn(sum, exp_fixed(__fsub_rn(x[c], m)));
-    for (int c = 0; c < classes; ++c)
-      prob[((size_t)n * classes + c) * P + p] = __fdiv_rn(exp_fixed(__fsub_rn(x[c], m)), sum);
+    float* pr_out = prob + (size_t)n * classes * P + p;
+    if (classes <= kRegClasses) {
+      // the logits and then the exponentials stay in registers: one exponential per class instead of two
+      float e[kRegClasses];
+#pragma unroll
+      for (int c = 0; c < kRegClasses; ++c) e[c] = c < classes ? x[c] : -FLT_MAX;
+      float m = e[0];
+#pragma unroll
+      for (int c = 1; c < kRegClasses; ++c) m = (c < classes && e[c] > m) ? e[c] : m;
+      float sum = 0.0f;
+#pragma unroll
+      for (int c = 0; c < kRegClasses; ++c)
+        if (c < classes) {
+          e[c] = exp_fixed(__fsub_rn(e[c], m));
+          sum = __fadd_rn(sum, e[c]);
+        }
+#pragma unroll
+      for (int c = 0; c < kRegClasses; ++c)
+        if (c < classes) pr_out[(size_t)c * P] = __fdiv_rn(e[c], sum);
+    } else {
+      float m = x[0];
+      for (int c = 1; c < classes; ++c) m = x[c] > m ? x[c] : m;
+      float sum = 0.0f;
+      for (int c = 0; c < classes; ++c) sum = __fadd_rn(sum, exp_fixed(__fsub_rn(x[c], m)));
+      for (int c = 0; c < classes; ++c) pr_out[(size_t)c * P] = __fdiv_rn(exp_fixed(__fsub_rn(x[c], m)), sum);
+    }
   }
 }
 
@@ -407,24 +428,18 @@ __global__ void __launch_bounds__(kTopThreads) keep_top_kernel(const float4* __r
                                                                int* __restrict__ counts) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);
-  __shared__ int cnt;
   const int n = blockIdx.x;
-  if (threadIdx.x == 0) cnt = 0;
-  __syncthreads();
+  int m = 0;  // every thread walks the class counts itself: no shared counter, no barrier per class
   for (int c = 0; c < classes; ++c) {
     if (c == background) continue;
     const int kc = kept_count[n * classes + c];
     const unsigned long long* kk = kept_keys + ((size_t)n * classes + c) * top_k;
-    __shared__ int base;
-    if (threadIdx.x == 0) { base = cnt; cnt += kc; }
-    __syncthreads();
     for (int i = threadIdx.x; i < kc; i += blockDim.x) {
       const unsigned long long key = kk[i];
-      keys[base + i] = (key & 0xffffffff00000000ull) | ((unsigned long long)c << 16) | (key & 0xffffull);
+      keys[m + i] = (key & 0xffffffff00000000ull) | ((unsigned long long)c << 16) | (key & 0xffffull);
     }
-    __syncthreads();
+    m += kc;
   }
-  const int m = cnt;
   int size = 1;
   while (size < m) size <<= 1;
   for (int i = m + threadIdx.x; i < size; i += blockDim.x) keys[i] = ~0ull;
