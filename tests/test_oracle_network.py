@@ -180,3 +180,35 @@ def test_per_channel_weight_factors():
     err_t = _rel(o.dequantize(out_t[last], info_t[last][1]), ref[last])
     err_c = _rel(o.dequantize(out_c[last], info_c[last][1]), ref[last])
     assert err_c < 0.12 and err_c <= err_t * 1.05
+
+
+def test_l2norm_layer_in_a_network_follows_fp32_and_keeps_its_structure():
+    """conv -> L2 normalisation -> two heads: the quantized run tracks the FP32 run, the normalised tensor is u8 at
+    its own calibrated factor, and dequantized it has per-pixel norms of about gamma (all channels equal here)."""
+    g = rng(91)
+    L = []
+    x = _conv(g, L, "c1", "input", 3, 32, 3, pad=1)
+    x = _conv(g, L, "c2", x, 32, 64, 3, pad=1)
+    L.append(Layer("c2_norm", "l2norm", [x], gamma=np.full(64, 20.0, np.float32)))
+    _conv(g, L, "head_a", "c2_norm", 64, 8, 3, pad=1, relu=False, bn=False, bias=True, f32_out=True)
+    _conv(g, L, "head_b", "c2_norm", 64, 12, 3, pad=1, relu=False, bn=False, bias=True, f32_out=True)
+    folded = _fold(L)
+    maxima = _calibrate(L, folded, 91, 2, 24)
+    prep, info = oracle_net.network_prepare(L, folded, maxima)
+    xin = nets.images(92, 2, 24)
+    got = oracle_net.network_forward(L, prep, info, xin, threads=2)
+    ref = nets.fp32_forward(L, xin, folded)
+    t, q = info["c2_norm"]
+    assert t == o.U8 and q == o.factor(maxima["c2_norm"], 8) and got["c2_norm"].dtype == np.uint8
+    deq = got["c2_norm"].astype(np.float64) * float(q)
+    norms = np.sqrt((deq ** 2).sum(-1))
+    live = np.sqrt((ref["c2"].astype(np.float64) ** 2).sum(-1)) > 1e-3
+    assert np.allclose(norms[live], 20.0, rtol=0.03)
+    assert _rel(deq, ref["c2_norm"]) < 0.05
+    for h in ("head_a", "head_b"):
+        assert _rel(got[h], ref[h]) < 0.1
+    # the SSD layer list with the option: one more layer, the conv4_3 heads read it
+    ssd = nets.ssd300(l2norm=True)
+    by = {x.name: x for x in ssd}
+    assert by["conv4_3_norm"].op == "l2norm" and by["conv4_3_norm_mbox_loc"].src == ["conv4_3_norm"] and by["pool4"].src == ["conv4_3"]
+    assert len(ssd) == len(nets.ssd300()) + 1 and nets.macs(ssd, 300) == nets.macs(nets.ssd300(), 300)
