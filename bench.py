@@ -10,7 +10,8 @@ between the two layers stays in shared memory).  Prints ONE JSON line (rank 0).
 
 * value      : int8 conv TOPS (2 * MACs / time), inputs resident in HBM, the K steps captured as one CUDA
                graph over rotating buffer sets whose total size exceeds L2; the graph is replayed until the
-               timed region lasts at least 0.25 s and the median time of a replay counts (timed_repeats).
+               timed region lasts at least 0.25 s and the median time of a replay counts (timed_repeats).  The
+               steps are independent batches and alternate between --step-streams streams (default 2).
 * e2e        : same metric with the u8 input of every step copied from pinned host memory and its u8 output
                copied back inside the timed region (three streams: the copies overlap the kernels).
 * roofline   : dominant kernel, algorithmic bytes / CUDA-event duration against the measured copy peak.
