@@ -932,16 +932,19 @@ __global__ void __launch_bounds__(256) pool3_strip_kernel(const uint4* __restric
 template <bool kSigned, bool kAvg, int kStride>
 void launch_pool3_strip(const void* x, int N, int H, int W, int cg, int pad_h, int pad_w, int P, int Q, float inv, void* y,
                         cudaStream_t s) {
+  // One strip per thread and a block per 256 strips: with a grid capped at the resident blocks, a tensor of 1.3
+  // times that many strips ran two rounds with the second a third full.  Four output rows per strip: two and eight
+  // were both measured slower for stride 2 (0.585 and 0.58 against 0.64 of the copy bandwidth).
   constexpr int kRows = 4;
   const int strips = (P + kRows - 1) / kRows;
   if (kStride == 1) {
     const unsigned int total = (unsigned int)((size_t)N * strips * ((Q + 1) / 2) * cg);
-    pool3_strip2_kernel<kSigned, kAvg, kRows><<<grid_for(total, 256, 8), 256, 0, s>>>(
+    pool3_strip2_kernel<kSigned, kAvg, kRows><<<(total + 255u) / 256u, 256, 0, s>>>(
         static_cast<const uint4*>(x), H, W, cg, pad_h, pad_w, P, Q, strips, inv, total, static_cast<uint4*>(y));
     return;
   }
   const unsigned int total = (unsigned int)((size_t)N * strips * Q * cg);
-  pool3_strip_kernel<kSigned, kAvg, kStride, kRows><<<grid_for(total, 256, 8), 256, 0, s>>>(
+  pool3_strip_kernel<kSigned, kAvg, kStride, kRows><<<(total + 255u) / 256u, 256, 0, s>>>(
       static_cast<const uint4*>(x), H, W, cg, pad_h, pad_w, P, Q, strips, inv, total, static_cast<uint4*>(y));
 }
 
